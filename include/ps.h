@@ -1,0 +1,242 @@
+/* ps.h -- C interface of the placement-semantics sweep library (CUDA, sm_100a).
+ *
+ * The library evaluates, on one GPU, the derivation rules of "Placement
+ * Semantics for Distributed Deep Learning" over a design space that is
+ * enumerated on the device, never stored:
+ *
+ *   a point = (model shape, device count N, factorisation N = T*K*D into tensor,
+ *              pipeline and data degrees, activation variant, tensor-axis
+ *              activation variant, one of the five modes R,S,S*,M,O for each of
+ *              Theta, Omega, G, A on the data axis)
+ *
+ * and for every point yields, as exact unsigned 64-bit integers,
+ *
+ *   mem         per-device GPU bytes                      (Theorem 1)
+ *   comm_paper  per-step bytes priced by the paper         (Theorem 2, Corollary 1)
+ *   comm_ext    per-step bytes the execution model moves that Theorem 2 does
+ *               not price (re-replication, offload gathers, tensor/pipeline
+ *               traffic; Proposition 1 names the per-layer collectives)
+ *   host        per-step bytes over the host link (mode O, Definition 1 eq. (5))
+ *   flags       gradient integrity (Theorem 3), state consistency (Theorem 4),
+ *               composition validity (Theorems 6-7, Proposition 1, Remark 4)
+ *               and their reasons.
+ *
+ * There is no floating point anywhere.  Shards are element-granular with the
+ * boundaries of Definition 1 eq. (2); the per-device figure is the largest
+ * shard, ceil(E/n); a ring reduce-scatter or all-gather (Section 2.3) moves
+ * E - floor(E/n) elements on its busiest device; an all-reduce twice that.
+ *
+ * Conventions.  Every function returns 0 (PS_OK) or a negative PS_E_* code and
+ * never aborts.  "device pointer" = memory of the context's GPU, owned by the
+ * caller; "host pointer" = ordinary host memory.  All device work is enqueued
+ * on the stream the context borrows; outputs are valid once the caller has
+ * synchronised that stream (or called ps_status).  Kernels never trap: a
+ * kernel that detects an inconsistency sets a status word that ps_status and
+ * every later call report as PS_E_DEVICE.
+ */
+#ifndef PS_H_
+#define PS_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ------------------------------------------------------------------ codes */
+enum {
+  PS_OK = 0,
+  PS_E_NULLPTR = -1,       /* a required pointer is null                         */
+  PS_E_ALIGN = -2,         /* a device pointer is not aligned to its element     */
+  PS_E_RANGE = -3,         /* a size, shape or count is outside the stated range */
+  PS_E_BADINDEX = -4,      /* [first, first+count) leaves the space              */
+  PS_E_TRUNCATED = -5,     /* an output held fewer entries than were found       */
+  PS_E_CUDA = -6,          /* a CUDA runtime call failed                          */
+  PS_E_UNIMPLEMENTED = -7,
+  PS_E_DEVICE = -8,        /* a kernel reported an inconsistency (status word)   */
+  PS_E_CAPACITY = -9       /* an internal fixed-size list overflowed             */
+};
+
+/* placement modes of Definition 1 */
+enum { PS_MODE_R = 0, PS_MODE_S = 1, PS_MODE_SG = 2 /* S* */, PS_MODE_M = 3, PS_MODE_O = 4 };
+
+/* A placement specification (Definition 2) as a code:
+ *   code = pi_Theta + 5*pi_Omega + 25*pi_G + 125*pi_A        (0..624)
+ * Table 2's rows: DP 0, ZeRO-1 5, ZeRO-2 30, ZeRO-3/FSDP 32, ZeRO-Offload 49,
+ * tensor parallel (S,S,S,S) 156, pipeline parallel (S,S,S,R) 31. */
+#define PS_CODE_TP_SEQPAR 156
+#define PS_CODE_TP 31
+#define PS_CODE_PP 31
+
+/* flags */
+enum {
+  PS_F_GI = 1u << 0,          /* gradient integrity (Theorem 3)                      */
+  PS_F_SC = 1u << 1,          /* state consistency (Theorem 4)                       */
+  PS_F_CV = 1u << 2,          /* composition valid = bits 4..7 all set and T*K*D = N */
+  PS_F_FEASIBLE = 1u << 3,    /* mem <= capacity (only where a capacity is given)    */
+  PS_F_T_DIV_HEADS = 1u << 4, /* T divides the head count                            */
+  PS_F_K_DIV_LAYERS = 1u << 5,/* K divides the layer count                           */
+  PS_F_TP_LE_MAX = 1u << 6,   /* T <= tp_max_valid (Proposition 1: TP stays in-node) */
+  PS_F_AXIS_FORM = 1u << 7,   /* model axes have Table 2's forms                     */
+  PS_F_THETA_AVAIL = 1u << 8, /* every replica can obtain all parameters             */
+  PS_F_ACT_AVAIL = 1u << 9,   /* every replica has its own activations for backward  */
+  PS_F_GRAD_COVER = 1u << 10, /* reduced gradients reach every element that is updated */
+  PS_F_USES_HOST = 1u << 11,  /* some state is offloaded                             */
+  PS_F_PAPER_PRICED = 1u << 12/* Theorem 2 prices all data-axis traffic of this point */
+};
+
+enum { PS_COMM_PAPER = 0, PS_COMM_PAPER_PLUS_EXT = 1 };
+enum { PS_REDUCE_PARETO = 0, PS_REDUCE_TOPK = 1 };
+
+#define PS_NO_LIMIT UINT64_MAX
+#define PS_TOPK_MAX 128          /* largest max_entries of a top-k sweep            */
+#define PS_FRONTIER_INTERNAL 256 /* longest frontier one block can hold (see sweep) */
+
+/* ------------------------------------------------------------------ types */
+typedef struct ps_ctx ps_ctx;     /* opaque: device, borrowed stream, scratch memory      */
+typedef struct ps_space ps_space; /* opaque: device copy of the model table + enumeration */
+
+/* One model, 48 bytes (Section 2.1, Remark 1, Definition 3).
+ * Ranges: layers <= 2^10, hidden <= 2^16, heads <= 2^16, vocab <= 2^24,
+ * seq <= 2^17, micro_batch <= 2^10, widths 1..16, parameter count <= 2^46,
+ * stored activations <= 2^58 bytes; all >= 1.  Outside: PS_E_RANGE. */
+typedef struct {
+  uint64_t param_elems_override; /* 0: P = 12*L*H^2 + V*H (Section 2.1); else P    */
+  uint32_t layers, hidden, heads, vocab, seq, micro_batch;
+  uint8_t w_param, w_grad, w_opt, w_act; /* bytes per element; Remark 1: 2, 2, 12, 2 */
+  uint8_t unit_from_shape;       /* 1: reconstruction unit = 12*H^2 elements (Def. 3); 0: none */
+  uint8_t act_enabled;           /* 0: |A| = 0 ("excluding activations", Example 3)  */
+  uint8_t pad[10];
+} ps_model_shape;
+
+/* The design space.  Linear index order: model-major; then N in the order
+ * given; then factorisations (T ascending, then K ascending) over all T | N,
+ * T <= t_enum_max, K | N/T, K <= k_enum_max, D = N/(T*K), independent of the
+ * model; then the activation variant; then the tensor-axis variant; then the
+ * data-axis code, fastest, written in base |mode_mask| over the allowed modes
+ * in ascending order with the Theta digit fastest. */
+typedef struct {
+  const ps_model_shape* models; /* host pointer, copied by ps_space_create            */
+  uint32_t n_models;            /* 1 .. 2^20                                           */
+  const uint32_t* n_values;     /* host pointer, copied; each 1 .. 2^24                */
+  uint32_t n_n;                 /* 1 .. 64                                             */
+  uint32_t t_enum_max;          /* >= 1                                                */
+  uint32_t k_enum_max;          /* >= 1                                                */
+  uint32_t tp_max_valid;        /* T above this clears PS_F_TP_LE_MAX                  */
+  uint32_t n_act_variants;      /* 1: activations stored; 2: {stored, full checkpointing} */
+  uint32_t n_tpa_variants;      /* 1: tensor axis shards activations (pi_A = S);
+                                   2: {S, R}                                            */
+  uint32_t mode_mask;           /* bit m set: mode m allowed on the data axis; != 0    */
+  uint32_t tp_coll_per_layer;   /* all-reduces per layer per step on the tensor axis, <= 64 */
+} ps_space_desc;
+
+/* survivors of a filter: mem <= cap_bytes, host <= host_cap and every bit of
+ * require_flags set (PS_F_FEASIBLE in require_flags is implied by the cap). */
+typedef struct {
+  uint64_t host_cap;      /* PS_NO_LIMIT for none                                  */
+  uint32_t require_flags;
+  uint32_t comm_kind;     /* objective of the sweeps: PS_COMM_PAPER or ..._PLUS_EXT */
+  uint64_t cap_bytes;     /* ps_eval_batch only; the sweeps take their own list     */
+} ps_filter;
+
+/* structure-of-arrays outputs of ps_eval_batch: device pointers, any may be
+ * null (skipped); u64 arrays 8-byte aligned (16 preferred), flags 4-byte. */
+typedef struct {
+  uint64_t *mem, *comm_paper, *comm_ext, *host;
+  uint32_t* flags;
+} ps_out_soa;
+
+/* one entry of a frontier or top-k list, 40 bytes */
+typedef struct {
+  uint64_t mem, comm, host, idx;
+  uint32_t flags, pad;
+} ps_front_entry;
+
+/* a decoded point; device rank layout is rank = (d*K + k)*T + t (Remark 4:
+ * tensor innermost, pipeline in the middle, data outermost; Theorem 6(1)) */
+typedef struct {
+  uint32_t model, N, T, K, D, act_variant, tpa_variant;
+  uint16_t code_dp, code_tp, code_pp, pad;
+} ps_point;
+
+/* ------------------------------------------------------------------ context */
+/* Create a context on `device` that enqueues on `cuda_stream` (a cudaStream_t
+ * passed as void*, borrowed, may be null = default stream).  Allocates a small
+ * scratch area that later calls grow on demand. */
+int ps_create(ps_ctx** out, int device, void* cuda_stream);
+void ps_destroy(ps_ctx* ctx);
+/* Synchronise the stream and return PS_OK or the first error a kernel
+ * recorded since the last call of ps_status (which also clears it). */
+int ps_status(ps_ctx* ctx);
+const char* ps_strerror(int code);
+
+/* ------------------------------------------------------------------ space */
+/* Validate the description, enumerate the factorisations of every N on the
+ * host, copy the shape table to the device and derive the per-model records
+ * there (Section 2.1, Remark 1, Definition 3).  The space keeps no table of
+ * points.  Points per model must stay below 2^32. */
+int ps_space_create(ps_ctx* ctx, const ps_space_desc* desc, ps_space** out);
+void ps_space_destroy(ps_space* space);
+/* Replace the shape table (same n_models) from host memory: one asynchronous
+ * copy plus the derivation kernel on the context's stream.  `models` must stay
+ * valid until the stream has passed the copy (pinned memory makes it truly
+ * asynchronous). */
+int ps_space_set_models(ps_space* space, const ps_model_shape* models, uint32_t n_models);
+uint64_t ps_space_size(const ps_space* space);
+uint64_t ps_space_points_per_model(const ps_space* space);
+/* host-side decoding of a linear index (for reports) */
+int ps_space_decode(const ps_space* space, uint64_t idx, ps_point* out);
+
+/* ------------------------------------------------------------------ hot path */
+/* Evaluate points [first, first+count) (Theorems 1-4, 6-7).
+ *  filter == NULL: materialise -- out.X[i] belongs to point first+i.
+ *  filter != NULL: stream compaction -- the survivors are written densely in
+ *    index order; d_idx_out (device, may be null) receives their indices,
+ *    *d_n_out (device scalar, required) their number; flags carry
+ *    PS_F_FEASIBLE.  Outputs need room for `count` elements in the worst case.
+ * count may be 0. */
+int ps_eval_batch(ps_ctx* ctx, const ps_space* space, uint64_t first, uint64_t count,
+                  const ps_filter* filter, ps_out_soa out, uint64_t* d_idx_out,
+                  uint64_t* d_n_out);
+
+/* Sweep the whole space and reduce it per (model, capacity).
+ *  PS_REDUCE_PARETO: the distinct non-dominated (mem, comm) pairs among the
+ *    survivors, both minimised (the trade-off of Corollary 1), each represented
+ *    by its smallest linear index, sorted by mem ascending.
+ *  PS_REDUCE_TOPK: the max_entries (<= PS_TOPK_MAX) smallest survivors by
+ *    (comm, mem, idx).
+ * d_out is [n_models][n_caps][max_entries] (device, 8-byte aligned); unused
+ * slots are zeroed.  d_counts[n_models][n_caps] (device) receives the true
+ * frontier length, or for top-k the number of survivors, even when that
+ * exceeds max_entries.  A frontier longer than PS_FRONTIER_INTERNAL inside one
+ * block makes ps_status return PS_E_CAPACITY.  n_caps <= 8. */
+int ps_sweep_pareto(ps_ctx* ctx, const ps_space* space, const ps_filter* filter,
+                    const uint64_t* caps_bytes /* host */, uint32_t n_caps, uint32_t reduce_kind,
+                    uint32_t max_entries, ps_front_entry* d_out, uint32_t* d_counts);
+
+/* One composition with arbitrary per-axis codes (Definition 5): N devices as
+ * T x K x D, code_tp on the tensor axis, code_pp on the pipeline axis, code_dp
+ * on the data axis (each 0..624).  Evaluated on the device; h_out (host) is
+ * filled before the call returns (this call synchronises).  The numbers assume
+ * Table 2's forms on the model axes, the tensor-axis activation mode taken from
+ * code_tp; PS_F_AXIS_FORM says whether the given codes have those forms (an
+ * axis of degree 1 is not looked at).  idx of the entry is 0. */
+int ps_check_composition(ps_ctx* ctx, const ps_model_shape* shape /* host */, uint32_t N,
+                         uint32_t T, uint32_t K, uint32_t D, uint16_t code_tp, uint16_t code_pp,
+                         uint16_t code_dp, uint32_t act_variant, uint64_t cap_bytes,
+                         uint32_t tp_max_valid, uint32_t tp_coll_per_layer, uint32_t comm_kind,
+                         ps_front_entry* h_out);
+
+/* ------------------------------------------------------------------ measurement */
+/* Integer-pipe microbenchmark: `blocks` x 256 threads each run `iters` rounds
+ * of 8 independent 32-bit add/logic chains of 16 operations.  Returns through
+ * *thread_ops the number of 32-bit thread operations issued; the caller times
+ * the stream.  d_sink (device, >= 4 bytes) receives a value that depends on
+ * every chain. */
+int ps_int_peak(ps_ctx* ctx, uint32_t blocks, uint32_t iters, uint32_t* d_sink,
+                uint64_t* thread_ops);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PS_H_ */

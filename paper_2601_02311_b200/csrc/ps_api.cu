@@ -1,0 +1,498 @@
+// The C interface: argument validation, host-side enumeration of the
+// factorisations, scratch management and kernel launches.  No arithmetic of the
+// method happens on the host; every evaluation runs in the kernels.
+#include <cuda_runtime.h>
+#include <stdlib.h>
+#include <string.h>
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "ps.h"
+#include "ps_device.cuh"
+#include "ps_internal.h"
+
+struct ps_ctx {
+  int device;
+  cudaStream_t stream;
+  void* scratch;
+  size_t scratch_bytes;
+  u32* d_status;
+  u32* h_status;      // pinned
+  int sm_count;
+};
+
+struct ps_space {
+  ps_ctx* ctx;
+  ps_space_desc desc;             // pointers inside are not kept
+  std::vector<u32> n_values;
+  std::vector<Fact> facts;        // all N concatenated
+  std::vector<u32> fact_begin;    // per N, offset into facts (n_n + 1 entries)
+  std::vector<u32> modes;         // allowed modes ascending
+  ps_model_shape* d_shapes;
+  ModelRec* d_recs;
+  Fact* d_facts;
+  SpaceDev dev;
+};
+
+namespace {
+
+#define CUDA_OK(call)                         \
+  do {                                        \
+    if ((call) != cudaSuccess) return PS_E_CUDA; \
+  } while (0)
+
+struct DeviceGuard {
+  int prev;
+  bool ok;
+  explicit DeviceGuard(int dev) : prev(-1), ok(false) {
+    if (cudaGetDevice(&prev) != cudaSuccess) return;
+    ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// the supported ranges of a shape (the same limits the derivation kernel checks)
+bool shape_in_range(const ps_model_shape& s, u32 tp_coll) {
+  if (s.layers < 1 || s.layers > (1u << 10)) return false;
+  if (s.hidden < 1 || s.hidden > (1u << 16)) return false;
+  if (s.heads < 1 || s.heads > (1u << 16)) return false;
+  if (s.vocab < 1 || s.vocab > (1u << 24)) return false;
+  if (s.seq < 1 || s.seq > (1u << 17)) return false;
+  if (s.micro_batch < 1 || s.micro_batch > (1u << 10)) return false;
+  const uint8_t w[4] = {s.w_param, s.w_grad, s.w_opt, s.w_act};
+  for (int i = 0; i < 4; ++i)
+    if (w[i] < 1 || w[i] > 16) return false;
+  if (tp_coll > 64) return false;
+  typedef unsigned __int128 u128;
+  const u128 L = s.layers, H = s.hidden, V = s.vocab, S = s.seq, b = s.micro_batch, a = s.heads;
+  const u128 P = s.param_elems_override ? (u128)s.param_elems_override : 12 * L * H * H + V * H;
+  if (P < 1 || P > ((u128)1 << 46)) return false;
+  if (S * b * H > ((u128)1 << 40)) return false;
+  if (s.act_enabled) {
+    const u128 A0 = L * (34 * S * b * H + 5 * a * S * S * b);
+    if (A0 > ((u128)1 << 58)) return false;
+  } else if (5 * a * S * S * b > ((u128)1 << 58)) {
+    return false;
+  }
+  return true;
+}
+
+int ensure_scratch(ps_ctx* ctx, size_t bytes) {
+  if (bytes <= ctx->scratch_bytes) return PS_OK;
+  CUDA_OK(cudaStreamSynchronize(ctx->stream));
+  if (ctx->scratch) CUDA_OK(cudaFree(ctx->scratch));
+  ctx->scratch = nullptr;
+  ctx->scratch_bytes = 0;
+  size_t want = (bytes + (size_t(1) << 20) - 1) & ~((size_t(1) << 20) - 1);
+  CUDA_OK(cudaMalloc(&ctx->scratch, want));
+  ctx->scratch_bytes = want;
+  return PS_OK;
+}
+
+// a kernel-reported problem seen by an earlier status copy
+int pending_device_error(ps_ctx* ctx) {
+  const u32 st = *ctx->h_status;
+  if (st & ST_LIST_OVERFLOW) return PS_E_CAPACITY;
+  if (st) return PS_E_DEVICE;
+  return PS_OK;
+}
+
+int enqueue_status_copy(ps_ctx* ctx) {
+  CUDA_OK(cudaMemcpyAsync(ctx->h_status, ctx->d_status, sizeof(u32), cudaMemcpyDeviceToHost, ctx->stream));
+  return PS_OK;
+}
+
+u32 pick_chunks(const ps_ctx* ctx, const ps_space* sp) {
+  // enough blocks for about eight waves of four resident blocks per SM
+  const u64 target = (u64)ctx->sm_count * 4 * 8;
+  u64 c = (target + sp->dev.n_models - 1) / sp->dev.n_models;
+  if (c < 1) c = 1;
+  if (c > SWEEP_MAX_CHUNKS) c = SWEEP_MAX_CHUNKS;
+  const u64 by_units = (sp->dev.n_facts + SWEEP_WARPS - 1) / SWEEP_WARPS;   // a unit per warp at least
+  if (c > by_units) c = by_units;
+  if (c < 1) c = 1;
+  return (u32)c;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* ps_strerror(int code) {
+  switch (code) {
+    case PS_OK: return "ok";
+    case PS_E_NULLPTR: return "a required pointer is null";
+    case PS_E_ALIGN: return "a device pointer is misaligned";
+    case PS_E_RANGE: return "a size, shape or count is outside the supported range";
+    case PS_E_BADINDEX: return "the index window leaves the space";
+    case PS_E_TRUNCATED: return "an output was too short";
+    case PS_E_CUDA: return "a CUDA runtime call failed";
+    case PS_E_UNIMPLEMENTED: return "not implemented";
+    case PS_E_DEVICE: return "a kernel reported an inconsistency";
+    case PS_E_CAPACITY: return "an internal fixed-size list overflowed";
+    default: return "unknown error";
+  }
+}
+
+int ps_create(ps_ctx** out, int device, void* cuda_stream) {
+  if (!out) return PS_E_NULLPTR;
+  *out = nullptr;
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev < 1) return PS_E_CUDA;
+  if (device < 0 || device >= n_dev) return PS_E_RANGE;
+  DeviceGuard guard(device);
+  if (!guard.ok) return PS_E_CUDA;
+  ps_ctx* ctx = new (std::nothrow) ps_ctx();
+  if (!ctx) return PS_E_CUDA;
+  ctx->device = device;
+  ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+  ctx->scratch = nullptr;
+  ctx->scratch_bytes = 0;
+  ctx->d_status = nullptr;
+  ctx->h_status = nullptr;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return PS_E_CUDA; }
+  ctx->sm_count = prop.multiProcessorCount;
+  if (cudaMalloc(&ctx->d_status, sizeof(u32)) != cudaSuccess ||
+      cudaMallocHost(&ctx->h_status, sizeof(u32)) != cudaSuccess ||
+      cudaMemsetAsync(ctx->d_status, 0, sizeof(u32), ctx->stream) != cudaSuccess) {
+    ps_destroy(ctx);
+    return PS_E_CUDA;
+  }
+  *ctx->h_status = 0;
+  if (ensure_scratch(ctx, size_t(8) << 20) != PS_OK) { ps_destroy(ctx); return PS_E_CUDA; }
+  *out = ctx;
+  return PS_OK;
+}
+
+void ps_destroy(ps_ctx* ctx) {
+  if (!ctx) return;
+  DeviceGuard guard(ctx->device);
+  cudaStreamSynchronize(ctx->stream);
+  if (ctx->scratch) cudaFree(ctx->scratch);
+  if (ctx->d_status) cudaFree(ctx->d_status);
+  if (ctx->h_status) cudaFreeHost(ctx->h_status);
+  delete ctx;
+}
+
+int ps_status(ps_ctx* ctx) {
+  if (!ctx) return PS_E_NULLPTR;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return PS_E_CUDA;
+  CUDA_OK(cudaMemcpyAsync(ctx->h_status, ctx->d_status, sizeof(u32), cudaMemcpyDeviceToHost, ctx->stream));
+  CUDA_OK(cudaStreamSynchronize(ctx->stream));
+  const int rc = pending_device_error(ctx);
+  if (rc != PS_OK) {
+    *ctx->h_status = 0;
+    CUDA_OK(cudaMemsetAsync(ctx->d_status, 0, sizeof(u32), ctx->stream));
+    CUDA_OK(cudaStreamSynchronize(ctx->stream));
+  }
+  return rc;
+}
+
+// ------------------------------------------------------------------ space
+int ps_space_create(ps_ctx* ctx, const ps_space_desc* desc, ps_space** out) {
+  if (!ctx || !desc || !out || !desc->models || !desc->n_values) return PS_E_NULLPTR;
+  *out = nullptr;
+  if (desc->n_models < 1 || desc->n_models > (1u << 20)) return PS_E_RANGE;
+  if (desc->n_n < 1 || desc->n_n > 64) return PS_E_RANGE;
+  if (desc->t_enum_max < 1 || desc->k_enum_max < 1) return PS_E_RANGE;
+  if (desc->n_act_variants < 1 || desc->n_act_variants > 2) return PS_E_RANGE;
+  if (desc->n_tpa_variants < 1 || desc->n_tpa_variants > 2) return PS_E_RANGE;
+  if ((desc->mode_mask & 0x1Fu) == 0 || (desc->mode_mask & ~0x1Fu)) return PS_E_RANGE;
+  if (desc->tp_coll_per_layer > 64) return PS_E_RANGE;
+  for (u32 i = 0; i < desc->n_n; ++i)
+    if (desc->n_values[i] < 1 || desc->n_values[i] > (1u << 24)) return PS_E_RANGE;
+  for (u32 i = 0; i < desc->n_models; ++i)
+    if (!shape_in_range(desc->models[i], desc->tp_coll_per_layer)) return PS_E_RANGE;
+
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return PS_E_CUDA;
+  ps_space* sp = new (std::nothrow) ps_space();
+  if (!sp) return PS_E_CUDA;
+  sp->ctx = ctx;
+  sp->desc = *desc;
+  sp->desc.models = nullptr;
+  sp->desc.n_values = nullptr;
+  sp->d_shapes = nullptr;
+  sp->d_recs = nullptr;
+  sp->d_facts = nullptr;
+  sp->n_values.assign(desc->n_values, desc->n_values + desc->n_n);
+  // all (T, K) with T | N, K | N/T inside the enumeration limits: T ascending, then K
+  for (u32 i = 0; i < desc->n_n; ++i) {
+    sp->fact_begin.push_back((u32)sp->facts.size());
+    const u32 N = desc->n_values[i];
+    std::vector<u32> sorted;                      // divisors of N, ascending
+    for (u32 d = 1; (u64)d * d <= N; ++d)
+      if (N % d == 0) { sorted.push_back(d); if (d != N / d) sorted.push_back(N / d); }
+    std::sort(sorted.begin(), sorted.end());
+    for (u32 T : sorted) {
+      if (T > desc->t_enum_max) break;
+      const u32 rest = N / T;
+      for (u32 K : sorted) {
+        if (K > desc->k_enum_max || K > rest) break;
+        if (rest % K) continue;
+        sp->facts.push_back(Fact{N, T, K, rest / K});
+      }
+    }
+    if (sp->facts.size() > (size_t(1) << 20)) { delete sp; return PS_E_RANGE; }
+  }
+  sp->fact_begin.push_back((u32)sp->facts.size());
+  if (sp->facts.empty()) { delete sp; return PS_E_RANGE; }
+  u32 modemap = 0, nm = 0;
+  for (u32 m = 0; m < 5; ++m)
+    if (desc->mode_mask & (1u << m)) { modemap |= m << (4 * nm); sp->modes.push_back(m); ++nm; }
+  SpaceDev& d = sp->dev;
+  d.n_models = desc->n_models;
+  d.n_facts = (u32)sp->facts.size();
+  d.nv = desc->n_act_variants;
+  d.nt = desc->n_tpa_variants;
+  d.nvt = d.nv * d.nt;
+  d.nm = nm;
+  d.modemap = modemap;
+  d.n3 = nm * nm * nm;
+  d.n_codes = d.n3 * nm;
+  d.tp_max_valid = desc->tp_max_valid;
+  d.tp_coll = desc->tp_coll_per_layer;
+  const u64 ppm = (u64)d.n_facts * d.nvt * d.n_codes;
+  if (ppm >= ((u64)1 << 32)) { delete sp; return PS_E_RANGE; }
+  d.ppm = ppm;
+
+  bool ok = cudaMalloc(&sp->d_shapes, sizeof(ps_model_shape) * (size_t)desc->n_models) == cudaSuccess &&
+            cudaMalloc(&sp->d_recs, sizeof(ModelRec) * (size_t)desc->n_models) == cudaSuccess &&
+            cudaMalloc(&sp->d_facts, sizeof(Fact) * sp->facts.size()) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(sp->d_facts, sp->facts.data(), sizeof(Fact) * sp->facts.size(),
+                             cudaMemcpyHostToDevice, ctx->stream) == cudaSuccess;
+  if (!ok) { ps_space_destroy(sp); return PS_E_CUDA; }
+  d.recs = sp->d_recs;
+  d.facts = sp->d_facts;
+  int rc = ps_space_set_models(sp, desc->models, desc->n_models);
+  if (rc == PS_OK && cudaStreamSynchronize(ctx->stream) != cudaSuccess) rc = PS_E_CUDA;
+  if (rc != PS_OK) { ps_space_destroy(sp); return rc; }
+  *out = sp;
+  return PS_OK;
+}
+
+int ps_space_set_models(ps_space* sp, const ps_model_shape* models, uint32_t n_models) {
+  if (!sp || !models) return PS_E_NULLPTR;
+  if (n_models != sp->dev.n_models) return PS_E_RANGE;
+  for (u32 i = 0; i < n_models; ++i)
+    if (!shape_in_range(models[i], sp->dev.tp_coll)) return PS_E_RANGE;
+  ps_ctx* ctx = sp->ctx;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return PS_E_CUDA;
+  CUDA_OK(cudaMemcpyAsync(sp->d_shapes, models, sizeof(ps_model_shape) * (size_t)n_models,
+                          cudaMemcpyHostToDevice, ctx->stream));
+  CUDA_OK(launch_model_derive(sp->d_shapes, sp->d_recs, n_models, ctx->d_status, ctx->stream));
+  return PS_OK;
+}
+
+void ps_space_destroy(ps_space* sp) {
+  if (!sp) return;
+  DeviceGuard guard(sp->ctx->device);
+  cudaStreamSynchronize(sp->ctx->stream);
+  if (sp->d_shapes) cudaFree(sp->d_shapes);
+  if (sp->d_recs) cudaFree(sp->d_recs);
+  if (sp->d_facts) cudaFree(sp->d_facts);
+  delete sp;
+}
+
+uint64_t ps_space_size(const ps_space* sp) { return sp ? sp->dev.ppm * sp->dev.n_models : 0; }
+uint64_t ps_space_points_per_model(const ps_space* sp) { return sp ? sp->dev.ppm : 0; }
+
+int ps_space_decode(const ps_space* sp, uint64_t idx, ps_point* out) {
+  if (!sp || !out) return PS_E_NULLPTR;
+  if (idx >= ps_space_size(sp)) return PS_E_BADINDEX;
+  const SpaceDev& d = sp->dev;
+  out->model = (u32)(idx / d.ppm);
+  u64 r = idx % d.ppm;
+  const u64 per_unit = (u64)d.nvt * d.n_codes;
+  const Fact& f = sp->facts[(size_t)(r / per_unit)];
+  r %= per_unit;
+  out->N = f.N; out->T = f.T; out->K = f.K; out->D = f.D;
+  const u32 vt = (u32)(r / d.n_codes);
+  u32 code = (u32)(r % d.n_codes);
+  out->act_variant = vt / d.nt;
+  out->tpa_variant = vt % d.nt;
+  u32 full = 0, weight = 1;
+  for (int s = 0; s < 4; ++s) {
+    full += weight * sp->modes[code % d.nm];
+    code /= d.nm;
+    weight *= 5;
+  }
+  out->code_dp = (uint16_t)full;
+  out->code_tp = out->tpa_variant == 0 ? PS_CODE_TP_SEQPAR : PS_CODE_TP;
+  out->code_pp = PS_CODE_PP;
+  out->pad = 0;
+  return PS_OK;
+}
+
+// ------------------------------------------------------------------ batch evaluation
+int ps_eval_batch(ps_ctx* ctx, const ps_space* sp, uint64_t first, uint64_t count,
+                  const ps_filter* filter, ps_out_soa out, uint64_t* d_idx_out, uint64_t* d_n_out) {
+  if (!ctx || !sp) return PS_E_NULLPTR;
+  if (sp->ctx != ctx) return PS_E_RANGE;
+  const u64 size = ps_space_size(sp);
+  if (first > size || count > size - first) return PS_E_BADINDEX;
+  if (filter && !d_n_out) return PS_E_NULLPTR;
+  if (!aligned(out.mem, 8) || !aligned(out.comm_paper, 8) || !aligned(out.comm_ext, 8) ||
+      !aligned(out.host, 8) || !aligned(out.flags, 4) || !aligned(d_idx_out, 8) || !aligned(d_n_out, 8))
+    return PS_E_ALIGN;
+  if (filter && filter->comm_kind > PS_COMM_PAPER_PLUS_EXT) return PS_E_RANGE;
+  int rc = pending_device_error(ctx);
+  if (rc != PS_OK) return rc;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return PS_E_CUDA;
+  if (count == 0) {
+    if (filter) CUDA_OK(cudaMemsetAsync(d_n_out, 0, sizeof(u64), ctx->stream));
+    return PS_OK;
+  }
+  EvalArgs a;
+  memset(&a, 0, sizeof(a));
+  a.first = first;
+  a.count = count;
+  a.first_group = first / sp->dev.n_codes;
+  const u64 last_group = (first + count - 1) / sp->dev.n_codes;
+  const u64 n_groups = last_group - a.first_group + 1;
+  if (n_groups > (u64)0x7fffffff) return PS_E_RANGE;
+  a.n_tiles = (u32)n_groups;
+  a.out = out;
+  a.idx_out = d_idx_out;
+  a.n_out = d_n_out;
+  a.status = ctx->d_status;
+  if (!filter) {
+    CUDA_OK(launch_eval_materialise(sp->dev, a, ctx->stream));
+  } else {
+    a.has_filter = 1;
+    a.cap_bytes = filter->cap_bytes;
+    a.host_cap = filter->host_cap;
+    a.require_flags = filter->require_flags & ~(u32)PS_F_FEASIBLE;
+    const size_t off_bytes = (sizeof(u32) * n_groups + 15) & ~size_t(15);
+    rc = ensure_scratch(ctx, off_bytes + sizeof(u64) * n_groups);
+    if (rc != PS_OK) return rc;
+    a.tile_count = static_cast<u32*>(ctx->scratch);
+    a.tile_offset = reinterpret_cast<u64*>(static_cast<char*>(ctx->scratch) + off_bytes);
+    CUDA_OK(launch_eval_count(sp->dev, a, ctx->stream));
+    CUDA_OK(launch_tile_scan(a, ctx->stream));
+    CUDA_OK(launch_eval_write(sp->dev, a, ctx->stream));
+  }
+  return enqueue_status_copy(ctx);
+}
+
+// ------------------------------------------------------------------ sweeps
+int ps_sweep_pareto(ps_ctx* ctx, const ps_space* sp, const ps_filter* filter,
+                    const uint64_t* caps_bytes, uint32_t n_caps, uint32_t reduce_kind,
+                    uint32_t max_entries, ps_front_entry* d_out, uint32_t* d_counts) {
+  if (!ctx || !sp || !filter || !caps_bytes || !d_out || !d_counts) return PS_E_NULLPTR;
+  if (sp->ctx != ctx) return PS_E_RANGE;
+  if (n_caps < 1 || n_caps > PS_MAX_CAPS || max_entries < 1) return PS_E_RANGE;
+  if (reduce_kind != PS_REDUCE_PARETO && reduce_kind != PS_REDUCE_TOPK) return PS_E_RANGE;
+  if (reduce_kind == PS_REDUCE_TOPK && max_entries > PS_TOPK_MAX) return PS_E_RANGE;
+  if (filter->comm_kind > PS_COMM_PAPER_PLUS_EXT) return PS_E_RANGE;
+  if (!aligned(d_out, 8) || !aligned(d_counts, 4)) return PS_E_ALIGN;
+  int rc = pending_device_error(ctx);
+  if (rc != PS_OK) return rc;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return PS_E_CUDA;
+
+  const u32 n_chunks = pick_chunks(ctx, sp);
+  const size_t slots = (size_t)sp->dev.n_models * n_chunks;
+  const size_t partial_bytes = slots * SWEEP_LIST_CAP * sizeof(PartialEntry);
+  rc = ensure_scratch(ctx, partial_bytes + slots * sizeof(uint2));
+  if (rc != PS_OK) return rc;
+  SweepArgs s;
+  memset(&s, 0, sizeof(s));
+  s.host_cap = filter->host_cap;
+  s.require_flags = filter->require_flags & ~(u32)PS_F_FEASIBLE;
+  s.comm_kind = filter->comm_kind;
+  s.k_keep = reduce_kind == PS_REDUCE_TOPK ? max_entries : 0;
+  s.partial = static_cast<PartialEntry*>(ctx->scratch);
+  s.partial_n = reinterpret_cast<uint2*>(static_cast<char*>(ctx->scratch) + partial_bytes);
+  s.status = ctx->d_status;
+  MergeArgs m;
+  memset(&m, 0, sizeof(m));
+  m.partial = s.partial;
+  m.partial_n = s.partial_n;
+  m.n_chunks = n_chunks;
+  m.n_caps_total = n_caps;
+  m.max_entries = max_entries;
+  m.k_keep = s.k_keep;
+  m.comm_kind = filter->comm_kind;
+  m.out = d_out;
+  m.counts = d_counts;
+  m.status = ctx->d_status;
+  if (reduce_kind == PS_REDUCE_PARETO) {
+    u64 cap_max = 0;
+    for (u32 c = 0; c < n_caps; ++c) { m.caps[c] = caps_bytes[c]; if (caps_bytes[c] > cap_max) cap_max = caps_bytes[c]; }
+    s.cap_max = cap_max;
+    m.n_caps = n_caps;
+    CUDA_OK(launch_sweep(PS_REDUCE_PARETO, sp->dev, s, n_chunks, ctx->stream));
+    CUDA_OK(launch_sweep_merge(PS_REDUCE_PARETO, sp->dev, m, ctx->stream));
+  } else {
+    for (u32 c = 0; c < n_caps; ++c) {
+      s.cap_max = caps_bytes[c];
+      m.caps[0] = caps_bytes[c];
+      m.n_caps = 1;
+      m.cap_index = c;
+      CUDA_OK(launch_sweep(PS_REDUCE_TOPK, sp->dev, s, n_chunks, ctx->stream));
+      CUDA_OK(launch_sweep_merge(PS_REDUCE_TOPK, sp->dev, m, ctx->stream));
+    }
+  }
+  return enqueue_status_copy(ctx);
+}
+
+// ------------------------------------------------------------------ one composition
+int ps_check_composition(ps_ctx* ctx, const ps_model_shape* shape, uint32_t N, uint32_t T,
+                         uint32_t K, uint32_t D, uint16_t code_tp, uint16_t code_pp,
+                         uint16_t code_dp, uint32_t act_variant, uint64_t cap_bytes,
+                         uint32_t tp_max_valid, uint32_t tp_coll_per_layer, uint32_t comm_kind,
+                         ps_front_entry* h_out) {
+  if (!ctx || !shape || !h_out) return PS_E_NULLPTR;
+  if (N < 1 || N > (1u << 24) || T < 1 || T > (1u << 24) || K < 1 || K > (1u << 24) || D < 1 ||
+      D > (1u << 24))
+    return PS_E_RANGE;
+  if (code_tp > 624 || code_pp > 624 || code_dp > 624 || act_variant > 1 ||
+      comm_kind > PS_COMM_PAPER_PLUS_EXT)
+    return PS_E_RANGE;
+  if (!shape_in_range(*shape, tp_coll_per_layer)) return PS_E_RANGE;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return PS_E_CUDA;
+  int rc = ensure_scratch(ctx, 1024);
+  if (rc != PS_OK) return rc;
+  char* base = static_cast<char*>(ctx->scratch);
+  ps_model_shape* d_shape = reinterpret_cast<ps_model_shape*>(base);
+  ModelRec* d_rec = reinterpret_cast<ModelRec*>(base + 256);
+  ps_front_entry* d_out = reinterpret_cast<ps_front_entry*>(base + 512);
+  CUDA_OK(cudaMemcpyAsync(d_shape, shape, sizeof(ps_model_shape), cudaMemcpyHostToDevice, ctx->stream));
+  CUDA_OK(launch_model_derive(d_shape, d_rec, 1, ctx->d_status, ctx->stream));
+  // Table 2: tensor axis (S,S,S,S) or (S,S,S,R), pipeline axis (S,S,S,R); an axis
+  // of degree 1 is absent.  Activation mode of the tensor axis: digit 3 of its code.
+  const bool tp_form = (T == 1) || code_tp == PS_CODE_TP_SEQPAR || code_tp == PS_CODE_TP;
+  const bool pp_form = (K == 1) || code_pp == PS_CODE_PP;
+  const u32 tau = ((code_tp / 125) % 5 == PS_MODE_S) ? 0 : 1;
+  CUDA_OK(launch_check_point(d_rec, Fact{N, T, K, D}, act_variant, tau, code_dp, tp_max_valid,
+                             tp_coll_per_layer, (tp_form && pp_form) ? 1 : 0, comm_kind, cap_bytes,
+                             d_out, ctx->stream));
+  CUDA_OK(cudaMemcpyAsync(h_out, d_out, sizeof(ps_front_entry), cudaMemcpyDeviceToHost, ctx->stream));
+  CUDA_OK(cudaStreamSynchronize(ctx->stream));
+  return PS_OK;
+}
+
+// ------------------------------------------------------------------ measurement
+int ps_int_peak(ps_ctx* ctx, uint32_t blocks, uint32_t iters, uint32_t* d_sink, uint64_t* thread_ops) {
+  if (!ctx || !d_sink || !thread_ops) return PS_E_NULLPTR;
+  if (blocks < 1 || blocks > (1u << 20) || iters < 1) return PS_E_RANGE;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return PS_E_CUDA;
+  CUDA_OK(launch_int_peak(blocks, iters, d_sink, ctx->stream));
+  *thread_ops = (u64)blocks * 256 * iters * 128;   // 8 rounds x 8 chains x 2 operations
+  return PS_OK;
+}
+
+}  // extern "C"

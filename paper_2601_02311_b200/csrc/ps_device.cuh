@@ -1,0 +1,229 @@
+// Device-side data structures and arithmetic shared by the kernels of the
+// placement-semantics sweep.  Everything is unsigned integer arithmetic.
+#pragma once
+#include <stdint.h>
+#include "ps.h"
+
+typedef uint64_t u64;
+typedef uint32_t u32;
+
+// ---------------------------------------------------------------- records
+// What one model contributes to the formulas; derived on the device from a
+// ps_model_shape (Section 2.1, Remark 1, Definition 3).  96 bytes, 16-aligned.
+struct __align__(16) ModelRec {
+  u64 P;        // parameter elements
+  u64 unit;     // reconstruction unit in elements (Definition 3), 0 = none
+  u64 A[2];     // activation bytes of one replica: stored / full checkpointing
+  u64 UA[2];    // one layer of them
+  u64 Sbh;      // elements of one layer-boundary tensor, S*b*H
+  u32 L, heads;
+  u32 wT, wO, wG, wA;  // bytes per element of Theta, Omega, G, activation elements
+  u32 ok;       // 1 if the shape was within the supported ranges
+  u32 pad[3];
+};
+static_assert(sizeof(ModelRec) == 96, "model record is 96 bytes");
+
+// One factorisation N = T*K*D.  The list of all factorisations of all N of a
+// space (model independent, at most a few thousand entries) is the only
+// enumeration table that exists.
+struct __align__(16) Fact {
+  u32 N, T, K, D;
+};
+
+// The space as the kernels see it (passed by value).
+struct SpaceDev {
+  const ModelRec* recs;
+  const Fact* facts;
+  u64 ppm;            // points per model = n_facts * nvt * n_codes
+  u32 n_models;
+  u32 n_facts;        // factorisations of all N together ("units" per model)
+  u32 nv, nt, nvt;    // activation variants, tensor-axis variants, product
+  u32 nm;             // allowed modes on the data axis
+  u32 modemap;        // digit d -> mode, 4 bits each, ascending modes
+  u32 n_codes;        // nm^4
+  u32 n3;             // nm^3
+  u32 tp_max_valid, tp_coll;
+};
+
+enum : u32 {
+  SET_SHARDLIKE = (1u << PS_MODE_S) | (1u << PS_MODE_SG),
+  SET_TRANSIENT = (1u << PS_MODE_SG) | (1u << PS_MODE_M),
+  SET_UPDATE_ON_SHARD = (1u << PS_MODE_S) | (1u << PS_MODE_SG) | (1u << PS_MODE_O),
+  SET_THETA_ALWAYS = (1u << PS_MODE_R) | (1u << PS_MODE_SG) | (1u << PS_MODE_O),
+  SET_GRAD_FULL = (1u << PS_MODE_R) | (1u << PS_MODE_SG) | (1u << PS_MODE_M),
+  SET_ACT_OWN = (1u << PS_MODE_R) | (1u << PS_MODE_M) | (1u << PS_MODE_O),
+  SET_M_OR_O = (1u << PS_MODE_M) | (1u << PS_MODE_O)
+};
+
+__device__ __forceinline__ bool in_set(u32 set, u32 mode) { return (set >> mode) & 1u; }
+__device__ __forceinline__ u32 digit_mode(u32 modemap, u32 digit) { return (modemap >> (4 * digit)) & 7u; }
+
+// ---------------------------------------------------------------- division
+// Divisors are degrees (< 2^24).  Powers of two, the common case, are shifts;
+// the branch is uniform wherever a warp works on one factorisation.
+__device__ __forceinline__ u64 div_floor(u64 a, u32 d) {
+  if ((d & (d - 1)) == 0) return a >> (31 - __clz(d));
+  return a / d;
+}
+__device__ __forceinline__ u64 div_ceil(u64 a, u32 d) { return div_floor(a + (d - 1), d); }
+
+// ---------------------------------------------------------------- per factorisation
+// Quantities that depend on (model, T, K, D) only.  Remark 4: the tensor split
+// is innermost, the pipeline split next, the data axis outermost.  Both model
+// axes shard Theta, Omega and G (Table 2).
+struct UnitBase {
+  u64 E2;     // elements of Theta (= Omega = G) left on one (t, k) position
+  u64 sh;     // largest data-axis shard of them, ceil(E2 / D)   (eq. (2))
+  u64 x;      // ring volume over the data axis, E2 - floor(E2 / D)  (Section 2.3)
+  u64 u;      // reconstruction unit after the tensor split
+  u64 tp_x;   // ring volume of a boundary tensor over the tensor axis
+  u64 sbh_t;  // ceil(Sbh / T)
+  u32 lps;    // layers per pipeline stage, ceil(L / K)
+  u32 cv;     // PS_F_CV and its reason bits (axis form assumed)
+  bool d1;    // D == 1
+};
+
+__device__ __forceinline__ UnitBase unit_base(const ModelRec& r, const Fact& f, u32 tp_max_valid,
+                                              bool axis_form) {
+  UnitBase b;
+  u64 E1 = div_ceil(r.P, f.T);
+  b.E2 = div_ceil(E1, f.K);
+  u64 q = div_floor(b.E2, f.D);
+  b.sh = q + ((q * f.D != b.E2) ? 1 : 0);
+  b.x = b.E2 - q;
+  b.u = div_ceil(r.unit, f.T);
+  u64 qs = div_floor(r.Sbh, f.T);
+  b.tp_x = r.Sbh - qs;
+  b.sbh_t = qs + ((qs * f.T != r.Sbh) ? 1 : 0);
+  u32 ql = (u32)div_floor((u64)r.L, f.K);
+  bool k_layers = (ql * f.K == r.L);
+  b.lps = ql + (k_layers ? 0 : 1);
+  u32 qh = (u32)div_floor((u64)r.heads, f.T);
+  bool t_heads = (qh * f.T == r.heads);
+  bool tp_le = f.T <= tp_max_valid;
+  bool whole = ((u64)f.T * f.K * f.D == (u64)f.N);
+  u32 cv = (t_heads ? PS_F_T_DIV_HEADS : 0) | (k_layers ? PS_F_K_DIV_LAYERS : 0) |
+           (tp_le ? PS_F_TP_LE_MAX : 0) | (axis_form ? PS_F_AXIS_FORM : 0);
+  if (t_heads && k_layers && tp_le && axis_form && whole) cv |= PS_F_CV;
+  b.cv = cv;
+  b.d1 = (f.D == 1);
+  return b;
+}
+
+// Activations of one replica for variant v (stored / checkpointed) when the
+// tensor axis shards them (tau = 0, sequence parallel) or not (tau = 1); the
+// pipeline axis leaves them whole (Table 2).  Bytes.
+struct ActBase {
+  u64 EA, shA, uA;
+};
+__device__ __forceinline__ ActBase act_base(const ModelRec& r, const Fact& f, u32 v, u32 tau) {
+  ActBase a;
+  a.EA = tau == 0 ? div_ceil(r.A[v], f.T) : r.A[v];
+  a.uA = tau == 0 ? div_ceil(r.UA[v], f.T) : r.UA[v];
+  a.shA = div_ceil(a.EA, f.D);
+  return a;
+}
+
+// tensor-axis and pipeline-axis traffic per step (not priced by Theorem 2):
+// per layer of a stage, tp_coll all-reduces of a boundary tensor over T
+// devices; one boundary tensor forward and one backward between stages
+__device__ __forceinline__ u64 model_axis_traffic(const ModelRec& r, const Fact& f,
+                                                  const UnitBase& b, u32 tau, u32 tp_coll) {
+  u64 tp = (u64)b.lps * tp_coll * 2 * b.tp_x * r.wA;
+  u64 pp = (f.K > 1) ? 2 * (tau == 0 ? b.sbh_t : r.Sbh) * r.wA : 0;
+  return tp + pp;
+}
+
+// Theorem 1: persistent plus transient elements of a state under mode pi
+__device__ __forceinline__ u64 mu_elems(u32 pi, u64 full, u64 shard, u64 unit) {
+  u64 p = (pi == PS_MODE_R) ? full : (in_set(SET_SHARDLIKE, pi) ? shard : 0);
+  u64 t = in_set(SET_TRANSIENT, pi) ? unit : 0;
+  return p + t;
+}
+
+// ---------------------------------------------------------------- one point
+struct PointOut {
+  u64 mem, comm_paper, comm_ext, host;
+  u32 flags;  // without PS_F_FEASIBLE
+};
+
+// flags of a point from its four modes; ext_data_zero says whether the data
+// axis moves nothing beyond Theorem 2's terms
+__device__ __forceinline__ u32 point_flags(u32 th, u32 om, u32 gr, u32 ac, bool d1, u32 cv,
+                                           bool ext_data_zero) {
+  bool omega_full = (om == PS_MODE_R) || (d1 && in_set(SET_SHARDLIKE, om));
+  bool theta_avail = in_set(SET_THETA_ALWAYS, th) || (th == PS_MODE_S && d1) ||
+                     (th == PS_MODE_M && omega_full);
+  bool act_avail = d1 || in_set(SET_ACT_OWN, ac);
+  bool grad_cover = d1 || in_set(SET_UPDATE_ON_SHARD, om) || in_set(SET_GRAD_FULL, gr);
+  bool sc = (om != PS_MODE_M);
+  u32 modes_seen = (1u << th) | (1u << om) | (1u << gr) | (1u << ac);
+  bool uses_host = (modes_seen >> PS_MODE_O) & 1u;
+  bool priced = ext_data_zero && !(modes_seen & SET_M_OR_O);
+  u32 fl = cv;
+  if (theta_avail && act_avail && grad_cover) fl |= PS_F_GI;
+  if (sc) fl |= PS_F_SC;
+  if (theta_avail) fl |= PS_F_THETA_AVAIL;
+  if (act_avail) fl |= PS_F_ACT_AVAIL;
+  if (grad_cover) fl |= PS_F_GRAD_COVER;
+  if (uses_host) fl |= PS_F_USES_HOST;
+  if (priced) fl |= PS_F_PAPER_PRICED;
+  return fl;
+}
+
+// The whole evaluation of one point, with nothing hoisted.  Used where single
+// points are needed (ps_check_composition, re-deriving host bytes and flags of
+// the few entries a sweep emits).
+__device__ __forceinline__ PointOut eval_point(const ModelRec& r, const Fact& f, u32 v, u32 tau,
+                                               u32 th, u32 om, u32 gr, u32 ac, u32 tp_max_valid,
+                                               u32 tp_coll, bool axis_form) {
+  UnitBase b = unit_base(r, f, tp_max_valid, axis_form);
+  ActBase a = act_base(r, f, v, tau);
+  PointOut o;
+  o.mem = r.wT * mu_elems(th, b.E2, b.sh, b.u) + r.wO * mu_elems(om, b.E2, b.sh, b.u) +
+          r.wG * mu_elems(gr, b.E2, b.sh, b.u) + mu_elems(ac, a.EA, a.shA, a.uA);
+  u64 xT = b.x * r.wT, xO = b.x * r.wO, xG = b.x * r.wG;
+  // Theorem 2
+  o.comm_paper = (gr == PS_MODE_R ? 2 * xG : 0) + (gr == PS_MODE_S ? xG : 0) +
+                 (th == PS_MODE_SG ? 2 * xT : 0);
+  bool on_shard = in_set(SET_UPDATE_ON_SHARD, om);
+  u64 ext = 0;
+  if (th == PS_MODE_O) ext += 2 * xT;
+  if (th == PS_MODE_R && on_shard) ext += xT;
+  if (gr == PS_MODE_SG) ext += 2 * xG;
+  if (gr == PS_MODE_M) ext += on_shard ? xG : 2 * xG;
+  if (gr == PS_MODE_O) ext += xG;
+  if (om == PS_MODE_SG) ext += xO;
+  o.comm_ext = ext + model_axis_traffic(r, f, b, tau, tp_coll);
+  o.host = (th == PS_MODE_O ? 3 * b.sh * r.wT : 0) + (om == PS_MODE_O ? 2 * b.sh * r.wO : 0) +
+           (gr == PS_MODE_O ? 2 * b.sh * r.wG : 0) + (ac == PS_MODE_O ? 2 * a.EA : 0);
+  o.flags = point_flags(th, om, gr, ac, b.d1, b.cv, ext == 0);
+  return o;
+}
+
+// linear index within a model -> unit, variant, digits of the data-axis code
+struct LocalPoint {
+  u32 unit, v, tau, dth, dom, dgr, dac;
+};
+__device__ __forceinline__ LocalPoint decode_local(const SpaceDev& sp, u32 lidx) {
+  LocalPoint p;
+  u32 per_unit = sp.nvt * sp.n_codes;
+  p.unit = lidx / per_unit;
+  u32 r = lidx - p.unit * per_unit;
+  u32 vt = r / sp.n_codes;
+  u32 code = r - vt * sp.n_codes;
+  p.v = vt / sp.nt;
+  p.tau = vt - p.v * sp.nt;
+  p.dth = code % sp.nm; code /= sp.nm;
+  p.dom = code % sp.nm; code /= sp.nm;
+  p.dgr = code % sp.nm;
+  p.dac = code / sp.nm;
+  return p;
+}
+
+// status word bits set by kernels
+enum : u32 {
+  ST_BAD_SHAPE = 1u << 0,      // a model shape outside the supported ranges
+  ST_LIST_OVERFLOW = 1u << 1,  // a per-warp or per-block list was too short
+  ST_SELF_CHECK = 1u << 2      // an emitted entry did not re-evaluate to itself
+};

@@ -1,0 +1,85 @@
+// Host-visible declarations shared by the translation units of the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include "ps.h"
+#include "ps_device.cuh"
+
+// ---- sweep
+#define SWEEP_WARPS 8
+#define SWEEP_LIST_CAP 128        /* entries of a warp's list and of a block's partial list */
+#define SWEEP_MAX_CHUNKS 16       /* blocks per model                                        */
+#define MERGE_CAP (SWEEP_MAX_CHUNKS * SWEEP_LIST_CAP)
+#define SWEEP_MAX_PER_THREAD 8    /* MERGE_CAP / threads per block                           */
+#define PS_MAX_CAPS 8
+
+struct PartialEntry {
+  u64 a, b;   // Pareto: (mem, comm); top-k: (comm, mem)
+  u32 i;      // point index within the model
+  u32 pad;
+};
+
+struct SweepArgs {
+  u64 cap_max;          // survivors need mem <= cap_max
+  u64 host_cap;
+  u32 require_flags;    // without PS_F_FEASIBLE
+  u32 comm_kind;
+  u32 k_keep;           // top-k: entries kept
+  PartialEntry* partial;   // [n_models * n_chunks][SWEEP_LIST_CAP]
+  uint2* partial_n;        // [n_models * n_chunks]: (entries, survivors)
+  u32* status;
+};
+
+struct MergeArgs {
+  const PartialEntry* partial;
+  const uint2* partial_n;
+  u64 caps[PS_MAX_CAPS];
+  u32 n_chunks;
+  u32 n_caps;           // capacities this launch emits
+  u32 n_caps_total;     // capacities of the output layout
+  u32 cap_index;        // top-k: which capacity this launch is for
+  u32 max_entries;
+  u32 k_keep;
+  u32 comm_kind;
+  ps_front_entry* out;
+  u32* counts;
+  u32* status;
+};
+
+cudaError_t launch_sweep(int kind, const SpaceDev& sp, const SweepArgs& a, u32 n_chunks,
+                         cudaStream_t stream);
+cudaError_t launch_sweep_merge(int kind, const SpaceDev& sp, const MergeArgs& a, cudaStream_t stream);
+
+// ---- batch evaluation
+#define EVAL_THREADS 256
+#define EVAL_GROUPS_PER_TILE 8    /* a tile = this many consecutive groups of n_codes points */
+
+struct EvalArgs {
+  u64 first, count;         // the window
+  u64 first_group;          // global group index of the tile 0's first group
+  u32 n_tiles;
+  // filter (compaction modes)
+  u64 cap_bytes, host_cap;
+  u32 require_flags;        // without PS_F_FEASIBLE
+  u32 has_filter;
+  ps_out_soa out;
+  u64* idx_out;
+  u64* n_out;
+  // compaction scratch
+  u32* tile_count;          // [n_tiles] survivors of each tile
+  u64* tile_offset;         // [n_tiles] exclusive prefix
+  u32* status;
+};
+
+cudaError_t launch_eval_materialise(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream);
+cudaError_t launch_eval_count(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream);
+cudaError_t launch_tile_scan(const EvalArgs& a, cudaStream_t stream);
+cudaError_t launch_eval_write(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream);
+
+// ---- small kernels
+cudaError_t launch_model_derive(const ps_model_shape* d_shapes, ModelRec* d_recs, u32 n,
+                                u32* status, cudaStream_t stream);
+cudaError_t launch_check_point(const ModelRec* d_rec, Fact f, u32 v, u32 tau, u32 code_dp,
+                               u32 tp_max_valid, u32 tp_coll, u32 axis_form, u32 comm_kind,
+                               u64 cap_bytes, ps_front_entry* d_out, cudaStream_t stream);
+cudaError_t launch_int_peak(u32 blocks, u32 iters, u32* d_sink, cudaStream_t stream);

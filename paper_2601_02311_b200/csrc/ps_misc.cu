@@ -1,0 +1,121 @@
+// Small kernels: model-table derivation, single-point evaluation, integer-pipe
+// microbenchmark.
+#include "ps_device.cuh"
+#include "ps_internal.h"
+
+namespace {
+
+// Section 2.1: P = 12 L H^2 + V H; Definition 3: unit = 12 H^2 elements;
+// Remark 1: byte widths.  Activations of one replica (the paper gives no
+// formula; this is the per-layer count of the selective-recomputation analysis
+// it cites for sequence parallelism): 34 S b H + 5 a S^2 b bytes stored,
+// 2 S b H with full checkpointing.
+__global__ void k_model_derive(const ps_model_shape* __restrict__ shapes, ModelRec* __restrict__ recs,
+                               u32 n, u32* status) {
+  const u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  // 48-byte shape as three 16-byte loads
+  ps_model_shape s;
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(shapes + i);
+    uint4* dst = reinterpret_cast<uint4*>(&s);
+    dst[0] = __ldg(src); dst[1] = __ldg(src + 1); dst[2] = __ldg(src + 2);
+  }
+  bool ok = s.layers >= 1 && s.layers <= (1u << 10) && s.hidden >= 1 && s.hidden <= (1u << 16) &&
+            s.heads >= 1 && s.heads <= (1u << 16) && s.vocab >= 1 && s.vocab <= (1u << 24) &&
+            s.seq >= 1 && s.seq <= (1u << 17) && s.micro_batch >= 1 && s.micro_batch <= (1u << 10) &&
+            s.w_param >= 1 && s.w_param <= 16 && s.w_grad >= 1 && s.w_grad <= 16 &&
+            s.w_opt >= 1 && s.w_opt <= 16 && s.w_act >= 1 && s.w_act <= 16;
+  ModelRec r;
+  const u64 L = s.layers, H = s.hidden, V = s.vocab, S = s.seq, b = s.micro_batch, a = s.heads;
+  r.P = s.param_elems_override ? s.param_elems_override : 12 * L * H * H + V * H;
+  r.unit = s.unit_from_shape ? 12 * H * H : 0;
+  r.Sbh = S * b * H;                              // <= 2^43 here; supported up to 2^40
+  ok = ok && r.Sbh <= ((u64)1 << 40);
+  // per-layer activation bytes; 5 a S^2 b can reach 2^63, so bound it first
+  const u64 attn_unit = a * S;                    // <= 2^33
+  const u64 attn_rest = S * b;                    // <= 2^27
+  ok = ok && attn_unit <= (((u64)1 << 58) / 5) / attn_rest;
+  u64 per_layer = 0, per_layer_ckpt = 0;
+  if (ok && s.act_enabled) {
+    per_layer = 34 * r.Sbh + 5 * attn_unit * attn_rest;
+    per_layer_ckpt = 2 * r.Sbh;
+    ok = ok && per_layer <= ((u64)1 << 58) / L;
+  }
+  ok = ok && r.P >= 1 && r.P <= ((u64)1 << 46);
+  r.A[0] = ok ? L * per_layer : 0;
+  r.A[1] = ok ? L * per_layer_ckpt : 0;
+  r.UA[0] = ok ? per_layer : 0;
+  r.UA[1] = ok ? per_layer_ckpt : 0;
+  r.L = s.layers;
+  r.heads = s.heads;
+  r.wT = s.w_param; r.wO = s.w_opt; r.wG = s.w_grad; r.wA = s.w_act;
+  r.ok = ok ? 1 : 0;
+  r.pad[0] = r.pad[1] = r.pad[2] = 0;
+  if (!ok) {
+    // keep every later division and product harmless
+    r.P = 1; r.unit = 0; r.Sbh = 1; r.L = 1; r.heads = 1;
+    r.wT = r.wO = r.wG = r.wA = 1;
+    atomicOr(status, ST_BAD_SHAPE);
+  }
+  recs[i] = r;
+}
+
+__global__ void k_check_point(const ModelRec* rec, Fact f, u32 v, u32 tau, u32 code_dp,
+                              u32 tp_max_valid, u32 tp_coll, u32 axis_form, u32 comm_kind,
+                              u64 cap_bytes, ps_front_entry* out) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  const u32 th = code_dp % 5, om = (code_dp / 5) % 5, gr = (code_dp / 25) % 5, ac = (code_dp / 125) % 5;
+  const PointOut p = eval_point(*rec, f, v, tau, th, om, gr, ac, tp_max_valid, tp_coll, axis_form != 0);
+  ps_front_entry e;
+  e.mem = p.mem;
+  e.comm = comm_kind == PS_COMM_PAPER ? p.comm_paper : p.comm_paper + p.comm_ext;
+  e.host = p.host;
+  e.idx = 0;
+  e.flags = p.flags | (p.mem <= cap_bytes ? PS_F_FEASIBLE : 0);
+  e.pad = 0;
+  *out = e;
+}
+
+// 8 independent chains per thread; each round applies to every chain an add
+// and an xor with loop-carried values the compiler cannot fold, so a round is
+// 16 independent-across-chains 32-bit operations and a chain's operations are
+// dependent (8 chains hide the pipe latency).
+__global__ void __launch_bounds__(256) k_int_peak(u32 iters, u32* sink) {
+  u32 c0 = threadIdx.x, c1 = c0 + 1, c2 = c0 + 2, c3 = c0 + 3, c4 = c0 + 4, c5 = c0 + 5,
+      c6 = c0 + 6, c7 = c0 + 7;
+  u32 k = blockIdx.x | 1u, m = (blockIdx.x << 7) | 5u;
+  for (u32 it = 0; it < iters; ++it) {
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      c0 += k; c1 += k; c2 += k; c3 += k; c4 += k; c5 += k; c6 += k; c7 += k;
+      c0 ^= m; c1 ^= m; c2 ^= m; c3 ^= m; c4 ^= m; c5 ^= m; c6 ^= m; c7 ^= m;
+    }
+    k += it;
+    m ^= k;
+  }
+  const u32 r = c0 ^ c1 ^ c2 ^ c3 ^ c4 ^ c5 ^ c6 ^ c7;
+  if (r == 0x9e3779b9u) atomicAdd(sink, r);   // practically never; keeps the chains alive
+  if (threadIdx.x == 0 && blockIdx.x == 0) atomicAdd(sink, r & 1u);
+}
+
+}  // namespace
+
+cudaError_t launch_model_derive(const ps_model_shape* d_shapes, ModelRec* d_recs, u32 n, u32* status,
+                                cudaStream_t stream) {
+  k_model_derive<<<(n + 127) / 128, 128, 0, stream>>>(d_shapes, d_recs, n, status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_check_point(const ModelRec* d_rec, Fact f, u32 v, u32 tau, u32 code_dp,
+                               u32 tp_max_valid, u32 tp_coll, u32 axis_form, u32 comm_kind,
+                               u64 cap_bytes, ps_front_entry* d_out, cudaStream_t stream) {
+  k_check_point<<<1, 32, 0, stream>>>(d_rec, f, v, tau, code_dp, tp_max_valid, tp_coll, axis_form,
+                                      comm_kind, cap_bytes, d_out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_int_peak(u32 blocks, u32 iters, u32* d_sink, cudaStream_t stream) {
+  k_int_peak<<<blocks, 256, 0, stream>>>(iters, d_sink);
+  return cudaGetLastError();
+}

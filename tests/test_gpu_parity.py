@@ -1,0 +1,288 @@
+"""Bit-exact parity of the CUDA library (through its C interface) with the CPU
+oracle on the same seeded inputs.  Everything is an integer or a boolean, so
+the tolerance is zero."""
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+from paper_2601_02311_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+FIELDS = ("mem", "comm_paper", "comm_ext", "host", "flags")
+VALID = O.F_GI | O.F_SC | O.F_CV
+
+
+@pytest.fixture(scope="module")
+def ps():
+    import paper_2601_02311_b200.ps as ps_mod
+    return ps_mod
+
+
+@pytest.fixture(scope="module")
+def ctx(ps):
+    c = ps.Context(0)
+    yield c
+    c.close()
+
+
+def both(ctx, space):
+    return ctx.space(space), O.Space(space)
+
+
+def assert_same_arrays(got, want, what=""):
+    for k in want:
+        if k not in got:
+            continue
+        g, w = np.asarray(got[k]), np.asarray(want[k])
+        assert g.shape == w.shape, (what, k, g.shape, w.shape)
+        if not np.array_equal(g, w):
+            bad = np.nonzero(g != w)[0]
+            raise AssertionError(f"{what} {k}: {len(bad)} mismatches, first at {bad[0]}: "
+                                 f"gpu {g[bad[0]]} oracle {w[bad[0]]}")
+
+
+def assert_same_sweep(got, want, model_slice=slice(None)):
+    ge, gc = got
+    we, wc = want
+    assert np.array_equal(gc[model_slice], wc[model_slice]), (gc[model_slice], wc[model_slice])
+    g, w = ge[model_slice], we[model_slice]
+    for name in ("mem", "comm", "host", "idx", "flags"):
+        if not np.array_equal(g[name], w[name]):
+            bad = np.argwhere(g[name] != w[name])[0]
+            raise AssertionError(f"{name} differs at {tuple(bad)}: gpu {g[name][tuple(bad)]} "
+                                 f"oracle {w[name][tuple(bad)]}")
+
+
+# ------------------------------------------------------------------ worked example
+def test_worked_example_all_outputs(ctx):
+    for name in ("C0", "C0b"):
+        gs, os_ = both(ctx, synth.config(name))
+        assert gs.size == os_.size == 4375
+        assert_same_arrays(gs.eval_batch(0, 4375), os_.eval_range(0, 4375), name)
+
+
+def test_worked_example_printed_values(ctx):
+    """The numbers the paper prints, straight from the kernels."""
+    gs = ctx.space(synth.config("C0"))
+    r = gs.eval_batch(0, 4375)
+    n8 = 3 * 625
+    assert int(r["mem"][n8 + 0]) == 1_120_000_000_000        # Example 3, data parallel
+    assert int(r["mem"][n8 + 32]) == 140_000_000_000         # Example 3, ZeRO-3 at N = 8
+    assert int(r["comm_paper"][n8 + 0]) == 245_000_000_000   # Example 4
+    assert int(r["comm_paper"][n8 + 32]) == 367_500_000_000  # Example 4
+    for ni in range(1, 7):
+        b = ni * 625
+        assert 2 * int(r["comm_paper"][b + 32]) == 3 * int(r["comm_paper"][b + 0])
+
+
+# ------------------------------------------------------------------ materialise
+@pytest.mark.parametrize("name,n_models", [("C1", 6), ("C2", 2), ("C3", 1)])
+def test_materialise_whole_small_space(ctx, name, n_models):
+    gs, os_ = both(ctx, synth.config(name, n_models=n_models))
+    n = gs.size
+    assert n == os_.size
+    assert_same_arrays(gs.eval_batch(0, n), os_.eval_range(0, n), name)
+
+
+def test_materialise_ragged_windows(ctx):
+    """Windows that start and end inside groups, one shorter than a group, one
+    of a single point, one empty, one ending at the last point of the space."""
+    gs, os_ = both(ctx, synth.config("C2", n_models=3))
+    n = gs.size
+    for first, count in [(1, 77), (255, 2), (256 * 5 + 13, 256 * 9 + 200), (n - 1000, 1000),
+                         (n - 1, 1), (12345, 0), (n, 0), (100_000, 300_001)]:
+        got = gs.eval_batch(first, count)
+        want = os_.eval_range(first, count)
+        assert_same_arrays(got, want, f"window {first}+{count}")
+
+
+def test_materialise_subset_of_outputs(ctx):
+    gs, os_ = both(ctx, synth.config("C1", n_models=2))
+    got = gs.eval_batch(500, 20000, fields=("mem", "flags"))
+    want = os_.eval_range(500, 20000)
+    assert set(got) == {"mem", "flags"}
+    assert_same_arrays(got, want)
+
+
+def test_awkward_device_counts_and_mode_mask(ctx):
+    """N that are primes or have repeated factors, T and K not powers of two,
+    three allowed modes (27 + 54 = 81 codes per group)."""
+    space = synth.ragged_space(21)
+    gs, os_ = both(ctx, space)
+    n = gs.size
+    assert n == os_.size
+    assert_same_arrays(gs.eval_batch(0, n), os_.eval_range(0, n), "ragged")
+    for idx in list(range(0, n, 997)) + [n - 1]:
+        assert gs.decode(idx) == os_.decode(idx)
+
+
+def test_single_mode_space(ctx):
+    """mode_mask with one bit: one point per group."""
+    space = synth.ragged_space(5, n_models=2)
+    space["mode_mask"] = 0b00100
+    gs, os_ = both(ctx, space)
+    n = gs.size
+    assert_same_arrays(gs.eval_batch(0, n), os_.eval_range(0, n), "single mode")
+
+
+# ------------------------------------------------------------------ compaction
+@pytest.mark.parametrize("cap_gb,require,host_cap", [(80, VALID, O.NO_LIMIT), (192, O.F_GI | O.F_SC, 10 ** 10),
+                                                     (10 ** 6, 0, O.NO_LIMIT), (0, 0, O.NO_LIMIT)])
+def test_compaction_in_index_order(ctx, cap_gb, require, host_cap):
+    gs, os_ = both(ctx, synth.config("C3", n_models=2))
+    first, count = 4321, 700_001
+    filt = dict(cap_bytes=cap_gb * synth.GB, require_flags=require, host_cap=host_cap)
+    got = gs.compact(first, count, filt)
+    want = os_.compact_range(first, count, filt)
+    assert len(got["idx"]) == len(want["idx"])
+    assert_same_arrays(got, want, "compaction")
+
+
+def test_compaction_c2_under_80gb(ctx):
+    gs, os_ = both(ctx, synth.config("C2", n_models=4))
+    n = gs.size
+    filt = dict(cap_bytes=80 * synth.GB, require_flags=VALID)
+    got = gs.compact(0, n, filt)
+    want = os_.compact_range(0, n, filt)
+    assert_same_arrays(got, want, "C2 compaction")
+    assert np.all(got["flags"] & O.F_FEASIBLE)
+
+
+# ------------------------------------------------------------------ sweeps
+@pytest.mark.parametrize("comm_kind", [O.COMM_PAPER, O.COMM_PAPER_PLUS_EXT])
+@pytest.mark.parametrize("host_cap", [0, 16 * synth.GB, O.NO_LIMIT])
+def test_pareto_c3_sample(ctx, ps, comm_kind, host_cap):
+    space = synth.config("C3", n_models=5)
+    gs, os_ = both(ctx, space)
+    filt = dict(require_flags=VALID, comm_kind=comm_kind, host_cap=host_cap)
+    caps = [80 * synth.GB, 192 * synth.GB]
+    got = gs.sweep(filt, caps, ps.REDUCE_PARETO, 64)
+    want = os_.sweep(filt, caps, O.KIND_PARETO, 64, n_threads=8)
+    assert_same_sweep(got, want)
+
+
+def test_pareto_many_caps_unsorted_and_truncated(ctx, ps):
+    """Capacities in arbitrary order; an output shorter than the frontier still
+    gets the true length in counts."""
+    space = synth.config("C3", n_models=3)
+    gs, os_ = both(ctx, space)
+    filt = dict(require_flags=VALID, host_cap=0)
+    caps = [192 * synth.GB, 8 * synth.GB, 10 ** 15, 1, 40 * synth.GB]
+    got = gs.sweep(filt, caps, ps.REDUCE_PARETO, 3)
+    want = os_.sweep(filt, caps, O.KIND_PARETO, 3, n_threads=8)
+    assert want[1].max() > 3
+    assert_same_sweep(got, want)
+
+
+def test_pareto_without_requirements(ctx, ps):
+    """No required flags: invalid compositions compete too, ties are everywhere."""
+    space = synth.config("C2", n_models=2)
+    gs, os_ = both(ctx, space)
+    filt = dict(require_flags=0, comm_kind=O.COMM_PAPER)
+    caps = [192 * synth.GB]
+    assert_same_sweep(gs.sweep(filt, caps, ps.REDUCE_PARETO, 128),
+                      os_.sweep(filt, caps, O.KIND_PARETO, 128, n_threads=8))
+
+
+def test_pareto_worked_example_ties(ctx, ps):
+    """Activations excluded: the 625 codes collapse to 125 results, so the
+    smallest-index rule decides every entry."""
+    gs, os_ = both(ctx, synth.config("C0"))
+    for comm_kind in (0, 1):
+        filt = dict(require_flags=O.F_GI | O.F_SC, comm_kind=comm_kind, host_cap=0)
+        caps = [80 * synth.GB, 2000 * synth.GB]
+        assert_same_sweep(gs.sweep(filt, caps, ps.REDUCE_PARETO, 64),
+                          os_.sweep(filt, caps, O.KIND_PARETO, 64))
+
+
+def test_pareto_ragged_space(ctx, ps):
+    space = synth.ragged_space(33, n_models=4)
+    gs, os_ = both(ctx, space)
+    rec = O.model_record(space["models"][0:1])
+    caps = [16 * rec["P"] // 7, 16 * rec["P"]]
+    for require in (VALID, O.F_GI | O.F_SC, 0):
+        filt = dict(require_flags=require, host_cap=rec["P"])
+        assert_same_sweep(gs.sweep(filt, caps, ps.REDUCE_PARETO, 96),
+                          os_.sweep(filt, caps, O.KIND_PARETO, 96, n_threads=4))
+
+
+@pytest.mark.parametrize("k", [64, 7, 128])
+def test_topk_c4_sample(ctx, ps, k):
+    space = synth.config("C4", n_models=3)
+    gs, os_ = both(ctx, space)
+    filt = dict(require_flags=VALID)
+    caps = [192 * synth.GB]
+    assert_same_sweep(gs.sweep(filt, caps, ps.REDUCE_TOPK, k),
+                      os_.sweep(filt, caps, O.KIND_TOPK, k, n_threads=8))
+
+
+def test_topk_two_caps_host_cap_and_few_survivors(ctx, ps):
+    space = synth.ragged_space(8, n_models=3)
+    gs, os_ = both(ctx, space)
+    rec = O.model_record(space["models"][0:1])
+    filt = dict(require_flags=VALID, host_cap=0, comm_kind=O.COMM_PAPER)
+    caps = [rec["P"], 20 * rec["P"]]
+    got = gs.sweep(filt, caps, ps.REDUCE_TOPK, 64)
+    want = os_.sweep(filt, caps, O.KIND_TOPK, 64, n_threads=4)
+    assert want[1].min() < 64        # some (model, cap) has fewer survivors than slots
+    assert_same_sweep(got, want)
+
+
+def test_sweeps_are_deterministic(ctx, ps):
+    space = synth.config("C3", n_models=4)
+    gs = ctx.space(space)
+    filt = dict(require_flags=VALID, host_cap=16 * synth.GB)
+    a = gs.sweep(filt, [80 * synth.GB, 192 * synth.GB], ps.REDUCE_PARETO, 64)
+    b = gs.sweep(filt, [80 * synth.GB, 192 * synth.GB], ps.REDUCE_PARETO, 64)
+    assert a[0].tobytes() == b[0].tobytes() and a[1].tobytes() == b[1].tobytes()
+
+
+# ------------------------------------------------------------------ single compositions
+def test_check_composition_matches_oracle(ctx):
+    rng = np.random.default_rng(0)
+    shapes = synth.zoo(6, 77)
+    for trial in range(200):
+        shape = shapes[trial % 6:trial % 6 + 1]
+        T = int(rng.choice([1, 2, 3, 4, 8, 16]))
+        K = int(rng.choice([1, 2, 3, 5, 8]))
+        D = int(rng.choice([1, 2, 7, 64]))
+        N = T * K * D if trial % 5 else T * K * D + 1
+        code_tp = int(rng.choice([156, 31, 0, 32, 624]))
+        code_pp = int(rng.choice([31, 31, 156, 5]))
+        code_dp = int(rng.integers(0, 625))
+        args = (N, T, K, D, code_tp, code_pp, code_dp)
+        kw = dict(act_variant=trial % 2, cap_bytes=80 * synth.GB, comm_kind=trial % 2)
+        assert ctx.check_composition(shape, *args, **kw) == O.check_composition(shape, *args, **kw)
+
+
+def test_decode_matches_oracle(ctx):
+    space = synth.config("C4", n_models=3)
+    gs, os_ = both(ctx, space)
+    rng = np.random.default_rng(1)
+    for idx in rng.integers(0, gs.size, 300):
+        assert gs.decode(int(idx)) == os_.decode(int(idx))
+
+
+# ------------------------------------------------------------------ errors
+def test_argument_errors(ctx, ps):
+    space = synth.config("C1", n_models=1)
+    gs = ctx.space(space)
+    with pytest.raises(ps.PsError) as e:
+        gs.eval_batch(gs.size - 5, 6)
+    assert e.value.code == ps.E_BADINDEX
+    bad = dict(space)
+    bad["mode_mask"] = 0
+    with pytest.raises(ps.PsError) as e:
+        ctx.space(bad)
+    assert e.value.code == ps.E_RANGE
+    huge = synth.zoo(1, 3)
+    huge["hidden"] = 1 << 20
+    bad = dict(space, models=huge)
+    with pytest.raises(ps.PsError) as e:
+        ctx.space(bad)
+    assert e.value.code == ps.E_RANGE
+    with pytest.raises(ps.PsError) as e:
+        gs.sweep(dict(), [1], ps.REDUCE_TOPK, ps.TOPK_MAX + 1)
+    assert e.value.code == ps.E_RANGE
+    assert ctx.status() == ps.OK
