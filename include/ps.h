@@ -182,6 +182,9 @@ void ps_space_destroy(ps_space* space);
  * valid until the stream has passed the copy (pinned memory makes it truly
  * asynchronous). */
 int ps_space_set_models(ps_space* space, const ps_model_shape* models, uint32_t n_models);
+/* Run the derivation kernel again on the shape table already resident on the
+ * device (Section 2.1, Remark 1, Definition 3); no host memory is touched. */
+int ps_space_rederive(ps_space* space);
 uint64_t ps_space_size(const ps_space* space);
 uint64_t ps_space_points_per_model(const ps_space* space);
 /* host-side decoding of a linear index (for reports) */

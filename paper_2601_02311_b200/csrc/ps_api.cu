@@ -293,6 +293,15 @@ int ps_space_set_models(ps_space* sp, const ps_model_shape* models, uint32_t n_m
   return PS_OK;
 }
 
+int ps_space_rederive(ps_space* sp) {
+  if (!sp) return PS_E_NULLPTR;
+  ps_ctx* ctx = sp->ctx;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return PS_E_CUDA;
+  CUDA_OK(launch_model_derive(sp->d_shapes, sp->d_recs, sp->dev.n_models, ctx->d_status, ctx->stream));
+  return PS_OK;
+}
+
 void ps_space_destroy(ps_space* sp) {
   if (!sp) return;
   DeviceGuard guard(sp->ctx->device);

@@ -37,7 +37,7 @@ ENTRY_DTYPE = np.dtype([("mem", "<u8"), ("comm", "<u8"), ("host", "<u8"), ("idx"
                         ("flags", "<u4"), ("pad", "<u4")])
 
 EXPORTS = ("ps_create", "ps_destroy", "ps_status", "ps_strerror", "ps_space_create",
-           "ps_space_destroy", "ps_space_set_models", "ps_space_size",
+           "ps_space_destroy", "ps_space_set_models", "ps_space_rederive", "ps_space_size",
            "ps_space_points_per_model", "ps_space_decode", "ps_eval_batch", "ps_sweep_pareto",
            "ps_check_composition", "ps_int_peak")
 
@@ -78,6 +78,7 @@ _lib.ps_space_create.argtypes = [C.c_void_p, C.POINTER(_SpaceDesc), C.POINTER(C.
 _lib.ps_space_destroy.argtypes = [C.c_void_p]
 _lib.ps_space_destroy.restype = None
 _lib.ps_space_set_models.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32]
+_lib.ps_space_rederive.argtypes = [C.c_void_p]
 _lib.ps_space_size.argtypes = [C.c_void_p]
 _lib.ps_space_size.restype = C.c_uint64
 _lib.ps_space_points_per_model.argtypes = [C.c_void_p]
@@ -211,6 +212,9 @@ class Space:
             models_host = np.ascontiguousarray(models_host)
             ptr, n = models_host.ctypes.data, len(models_host)
         _check(_lib.ps_space_set_models(self._h, ptr, n), "ps_space_set_models")
+
+    def rederive(self) -> None:
+        _check(_lib.ps_space_rederive(self._h), "ps_space_rederive")
 
     # ---- ps_eval_batch
     def eval_batch_into(self, first: int, count: int, out: dict, filt: dict | None = None,
