@@ -54,7 +54,9 @@ enum {
   PS_E_CUDA = -6,          /* a CUDA runtime call failed                          */
   PS_E_UNIMPLEMENTED = -7,
   PS_E_DEVICE = -8,        /* a kernel reported an inconsistency (status word)   */
-  PS_E_CAPACITY = -9       /* an internal fixed-size list overflowed             */
+  PS_E_CAPACITY = -9,      /* an internal fixed-size list overflowed             */
+  PS_E_NOALLOC_LIMIT = -10 /* the window is too large for ps_eval_compact_noalloc's
+                              fixed scratch array (PS_NOALLOC_MAX_GROUPS groups)  */
 };
 
 /* placement modes of Definition 1 */
@@ -229,6 +231,38 @@ int ps_check_composition(ps_ctx* ctx, const ps_model_shape* shape /* host */, ui
                          uint16_t code_dp, uint32_t act_variant, uint64_t cap_bytes,
                          uint32_t tp_max_valid, uint32_t tp_coll_per_layer, uint32_t comm_kind,
                          ps_front_entry* h_out);
+
+/* The filter-and-compact form of ps_eval_batch for callers that cannot
+ * allocate device memory.  (The paper has no counterpart: this is a property of
+ * the library, not of the method.)
+ *
+ * Who needs it: a program whose GPU memory is wholly owned by another
+ * allocator -- a training framework's caching pool, or a serving process that
+ * has handed every byte to its cache -- where a raw cudaMalloc from a library
+ * can fail or fragment that pool; and a loop that cannot afford the implicit
+ * device-wide synchronisation of cudaFree/cudaMalloc.  ps_eval_batch may do
+ * both when its scratch has to grow.  This function never calls cudaMalloc,
+ * cudaFree or any allocating routine: its two scratch tables (a survivor count
+ * and a prefix sum per group of |mode_mask|^4 consecutive points) sit in a
+ * fixed 1.5 MiB array inside the library image, which every GPU that loads the
+ * library holds until the process ends.
+ *
+ * Arguments, outputs, order of the survivors and error behaviour are those of
+ * ps_eval_batch with a non-null filter (which is required here).  Limits and
+ * rules of its own:
+ *  - the window may touch at most PS_NOALLOC_MAX_GROUPS groups, else
+ *    PS_E_NOALLOC_LIMIT is returned and nothing is enqueued;
+ *  - the first call on each device looks up the array's device address (with
+ *    that device made current); make that first call before any stream
+ *    capture is begun;
+ *  - all calls on a device share the one array, and it keeps the previous
+ *    call's contents (the function clears what it is about to use): two calls
+ *    whose kernels overlap on the GPU -- different streams, or different
+ *    contexts on the same device -- race on it.  Serialise them. */
+#define PS_NOALLOC_MAX_GROUPS 131072
+int ps_eval_compact_noalloc(ps_ctx* ctx, const ps_space* space, uint64_t first, uint64_t count,
+                            const ps_filter* filter, ps_out_soa out, uint64_t* d_idx_out,
+                            uint64_t* d_n_out);
 
 /* ------------------------------------------------------------------ measurement */
 /* Integer-pipe microbenchmark: `blocks` x 256 threads each run `iters` rounds

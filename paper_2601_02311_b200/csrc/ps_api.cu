@@ -12,29 +12,6 @@
 #include "ps_device.cuh"
 #include "ps_internal.h"
 
-struct ps_ctx {
-  int device;
-  cudaStream_t stream;
-  void* scratch;
-  size_t scratch_bytes;
-  u32* d_status;
-  u32* h_status;      // pinned
-  int sm_count;
-};
-
-struct ps_space {
-  ps_ctx* ctx;
-  ps_space_desc desc;             // pointers inside are not kept
-  std::vector<u32> n_values;
-  std::vector<Fact> facts;        // all N concatenated
-  std::vector<u32> fact_begin;    // per N, offset into facts (n_n + 1 entries)
-  std::vector<u32> modes;         // allowed modes ascending
-  ps_model_shape* d_shapes;
-  ModelRec* d_recs;
-  Fact* d_facts;
-  SpaceDev dev;
-};
-
 namespace {
 
 #define CUDA_OK(call)                         \
@@ -136,6 +113,8 @@ const char* ps_strerror(int code) {
     case PS_E_UNIMPLEMENTED: return "not implemented";
     case PS_E_DEVICE: return "a kernel reported an inconsistency";
     case PS_E_CAPACITY: return "an internal fixed-size list overflowed";
+    case PS_E_NOALLOC_LIMIT:
+      return "the window needs more scratch than the no-allocation entry point's fixed array holds";
     default: return "unknown error";
   }
 }

@@ -5,6 +5,31 @@
 #include "ps.h"
 #include "ps_device.cuh"
 
+// ---- the opaque handles of ps.h
+#include <vector>
+struct ps_ctx {
+  int device;
+  cudaStream_t stream;
+  void* scratch;
+  size_t scratch_bytes;
+  u32* d_status;
+  u32* h_status;      // pinned
+  int sm_count;
+};
+
+struct ps_space {
+  ps_ctx* ctx;
+  ps_space_desc desc;             // pointers inside are not kept
+  std::vector<u32> n_values;
+  std::vector<Fact> facts;        // all N concatenated
+  std::vector<u32> fact_begin;    // per N, offset into facts (n_n + 1 entries)
+  std::vector<u32> modes;         // allowed modes ascending
+  ps_model_shape* d_shapes;
+  ModelRec* d_recs;
+  Fact* d_facts;
+  SpaceDev dev;
+};
+
 // ---- sweep
 #define SWEEP_WARPS 8
 #define SWEEP_LIST_CAP 128        /* entries of a warp's list and of a block's partial list */

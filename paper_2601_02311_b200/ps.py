@@ -24,6 +24,8 @@ _lib = C.CDLL(LIB_PATH)
 OK = 0
 E_NULLPTR, E_ALIGN, E_RANGE, E_BADINDEX, E_TRUNCATED, E_CUDA, E_UNIMPLEMENTED, E_DEVICE, E_CAPACITY = \
     -1, -2, -3, -4, -5, -6, -7, -8, -9
+E_NOALLOC_LIMIT = -10
+NOALLOC_MAX_GROUPS = 131072
 F_GI, F_SC, F_CV, F_FEASIBLE = 1, 2, 4, 8
 F_T_DIV_HEADS, F_K_DIV_LAYERS, F_TP_LE_MAX, F_AXIS_FORM = 16, 32, 64, 128
 F_THETA_AVAIL, F_ACT_AVAIL, F_GRAD_COVER, F_USES_HOST, F_PAPER_PRICED = 256, 512, 1024, 2048, 4096
@@ -39,7 +41,7 @@ ENTRY_DTYPE = np.dtype([("mem", "<u8"), ("comm", "<u8"), ("host", "<u8"), ("idx"
 EXPORTS = ("ps_create", "ps_destroy", "ps_status", "ps_strerror", "ps_space_create",
            "ps_space_destroy", "ps_space_set_models", "ps_space_rederive", "ps_space_size",
            "ps_space_points_per_model", "ps_space_decode", "ps_eval_batch", "ps_sweep_pareto",
-           "ps_check_composition", "ps_int_peak")
+           "ps_check_composition", "ps_int_peak", "ps_eval_compact_noalloc")
 
 
 class _SpaceDesc(C.Structure):
@@ -86,6 +88,7 @@ _lib.ps_space_points_per_model.restype = C.c_uint64
 _lib.ps_space_decode.argtypes = [C.c_void_p, C.c_uint64, C.POINTER(_Point)]
 _lib.ps_eval_batch.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.POINTER(_Filter),
                                _OutSoa, C.c_void_p, C.c_void_p]
+_lib.ps_eval_compact_noalloc.argtypes = _lib.ps_eval_batch.argtypes
 _lib.ps_sweep_pareto.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(_Filter), C.c_void_p,
                                  C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p]
 _lib.ps_check_composition.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32,
@@ -256,6 +259,17 @@ class Space:
         res = {name: _to_unsigned(v[:k]) for name, v in out.items()}
         res["idx"] = _to_unsigned(idx[:k])
         return res
+
+    def compact_noalloc_into(self, first: int, count: int, out: dict, filt: dict,
+                             idx_out: torch.Tensor | None, n_out: torch.Tensor):
+        """ps_eval_compact_noalloc: same contract as the filtered eval_batch_into, but the
+        library allocates nothing (fixed scratch; at most NOALLOC_MAX_GROUPS groups per
+        call; calls on one device must not overlap)."""
+        soa = _OutSoa(*(None if out.get(k) is None else out[k].data_ptr()
+                        for k in ("mem", "comm_paper", "comm_ext", "host", "flags")))
+        f = _mk_filter(filt)
+        _check(_lib.ps_eval_compact_noalloc(self.ctx._h, self._h, first, count, C.byref(f), soa,
+                                            _dptr(idx_out), _dptr(n_out)), "ps_eval_compact_noalloc")
 
     # ---- ps_sweep_pareto
     def sweep_into(self, filt: dict, caps, kind: int, max_entries: int, d_out: torch.Tensor,
