@@ -91,7 +91,7 @@ enum { PS_COMM_PAPER = 0, PS_COMM_PAPER_PLUS_EXT = 1 };
 enum { PS_REDUCE_PARETO = 0, PS_REDUCE_TOPK = 1 };
 
 #define PS_NO_LIMIT UINT64_MAX
-#define PS_TOPK_MAX 128          /* largest max_entries of a top-k sweep            */
+#define PS_TOPK_MAX 64           /* largest max_entries of a top-k sweep            */
 #define PS_FRONTIER_INTERNAL 256 /* longest frontier one block can hold (see sweep) */
 
 /* ------------------------------------------------------------------ types */

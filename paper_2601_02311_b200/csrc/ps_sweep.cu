@@ -4,9 +4,13 @@
 // of its factorisations ("units"); its warps take units round-robin.  For a
 // unit the warp computes the shard quantities once (all divisions), writes
 // small per-mode tables to its shared-memory slice, and then walks the
-// placement codes: a lane owns a (Theta, Omega, G) triple, keeps that triple's
-// partial sums in registers and visits the activation variants and activation
-// modes with adds, compares and selects only.
+// placement codes: a lane owns up to four (Theta, Omega, G) triples for the
+// whole kernel (their modes and the activation digits their flags allow never
+// change), keeps each triple's own bytes, communication and host bytes in
+// registers and visits the activation variants and activation digits.  Because
+// the activation bytes of a (variant, digit) are the same for every triple, the
+// capacity test of a point is one 64-bit compare of the triple's bytes against a
+// per-(variant, digit) bound; the sum is formed only for candidates.
 //
 // Reductions.  Every warp keeps a private sorted list in shared memory
 // (Pareto staircase or top-k), tests its candidates against it lane-parallel
@@ -26,15 +30,23 @@ constexpr int LIST_CAP = SWEEP_LIST_CAP;       // entries per warp list / per pa
 constexpr int BLOCK_CAP = WARPS * LIST_CAP;    // union of the warps' lists
 constexpr u64 U64MAX = ~0ull;
 
-// per-warp tables, rebuilt for every unit (all u64)
+// per-warp tables, rebuilt for every unit.  One entry per (state, mode): what
+// that state contributes to memory, to the objective communication and to the
+// host-link bytes (Theorem 1, Theorem 2 plus unpriced traffic, mode O).
+struct __align__(16) ModeEntry {
+  u64 mem, comm, host, pad;
+};
 struct WarpTables {
-  u64 mem[3][5];       // state (Theta, Omega, G) x mode: bytes of Theorem 1
-  u64 c_theta[2][5];   // [update on shard][mode]: objective communication terms
-  u64 c_omega[5];
-  u64 c_grad[2][5];
-  u64 act[4][5];       // variant (v, tau) x activation mode: bytes
-  u64 act_host[4];     // host bytes when activations are offloaded
-  u64 c_axis[4];       // tensor + pipeline traffic of the variant (0 if not in the objective)
+  ModeEntry theta[2][5];   // [update committed on a shard][mode]
+  ModeEntry omega[5];
+  ModeEntry grad[2][5];
+  // per activation variant vt = (v, tau) and slot k: k is the activation digit
+  // (top-k) or the rank of the digit by activation bytes, ascending (Pareto)
+  u64 bound[4][5];         // a triple whose own bytes are below this fits the capacity
+  u64 act[4][5];           // activation bytes of the slot
+  u32 digit[4][5];         // activation digit of the slot
+  u64 host_bound[4];       // a triple whose own host bytes are below this may offload activations
+  u64 c_axis[4];           // tensor + pipeline traffic of the variant (0 if not in the objective)
 };
 
 struct Key {
@@ -56,22 +68,8 @@ struct WarpList {
 };
 
 // Pareto staircase: a = mem ascending, b = comm strictly descending.
-// Is (m, c, idx) dominated by, or a later duplicate of, an entry?  Per lane.
-__device__ __forceinline__ bool pareto_rejects(const WarpList& w, u64 m, u64 c, u32 idx) {
-  int lo = 0, hi = w.n;
-  while (lo < hi) {               // number of entries with mem <= m
-    int mid = (lo + hi) >> 1;
-    if (w.a[mid] <= m) lo = mid + 1; else hi = mid;
-  }
-  if (lo == 0) return false;
-  u64 ec = w.b[lo - 1];           // smallest comm among entries with mem <= m
-  if (ec < c) return true;
-  if (ec > c) return false;
-  return w.a[lo - 1] < m || w.i[lo - 1] < idx;
-}
-
 // warp-cooperative insertion; all lanes hold the same (m, c, idx)
-__device__ __forceinline__ void pareto_insert(WarpList& w, u64 m, u64 c, u32 idx, int lane,
+__device__ __noinline__ void pareto_insert(WarpList& w, u64 m, u64 c, u32 idx, int lane,
                                               u32* status) {
   constexpr int PER = LIST_CAP / 32;
   u64 ea[PER], eb[PER];
@@ -116,37 +114,54 @@ __device__ __forceinline__ void pareto_insert(WarpList& w, u64 m, u64 c, u32 idx
   __syncwarp();
 }
 
-// top-k list: keys ascending, at most k entries
-__device__ __forceinline__ void topk_insert(WarpList& w, const Key& key, int k_keep, int lane,
-                                            Key& threshold) {
-  constexpr int PER = LIST_CAP / 32;
-  Key e[PER];
-  int below = 0;
-#pragma unroll
-  for (int k = 0; k < PER; ++k) {
-    int p = lane + 32 * k;
-    bool valid = p < w.n;
-    e[k].a = valid ? w.a[p] : U64MAX;
-    e[k].b = valid ? w.b[p] : U64MAX;
-    e[k].i = valid ? w.i[p] : 0xffffffffu;
-    below += __popc(__ballot_sync(0xffffffffu, valid && key_less(e[k], key)));
-  }
-  if (below >= k_keep) return;                         // (cannot happen after the threshold test)
+// Top-k list of a warp: entries [0, n) are unordered candidates that were below
+// the threshold when they arrived.  When the list is full the warp sorts it,
+// keeps the k smallest and tightens the threshold to the k-th; until the first
+// such compaction the threshold is "everything".  A stale threshold only lets
+// extra candidates in, never keeps a wanted one out.
+__device__ __noinline__ void topk_compact(WarpList& w, int k_keep, int lane, Key& threshold) {
+  for (int p = w.n + lane; p < LIST_CAP; p += 32) { w.a[p] = U64MAX; w.b[p] = U64MAX; w.i[p] = 0xffffffffu; }
   __syncwarp();
-  int n_new = min(w.n + 1, k_keep);
+  for (int k = 2; k <= LIST_CAP; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
 #pragma unroll
-  for (int k = 0; k < PER; ++k) {
-    int p = lane + 32 * k;
-    if (p < w.n && p >= below && p + 1 < k_keep) {
-      w.a[p + 1] = e[k].a; w.b[p + 1] = e[k].b; w.i[p + 1] = e[k].i;
+      for (int e = 0; e < LIST_CAP / 64; ++e) {
+        const int t = lane + 32 * e;                       // pair number
+        const int p = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+        const int q = p | j;
+        const Key x{w.a[p], w.b[p], w.i[p]}, y{w.a[q], w.b[q], w.i[q]};
+        const bool up = (p & k) == 0;
+        if (key_less(y, x) == up) {
+          w.a[p] = y.a; w.b[p] = y.b; w.i[p] = y.i;
+          w.a[q] = x.a; w.b[q] = x.b; w.i[q] = x.i;
+        }
+      }
+      __syncwarp();
     }
   }
-  if (lane == 0) { w.a[below] = key.a; w.b[below] = key.b; w.i[below] = key.i; }
-  w.n = n_new;
-  __syncwarp();
+  w.n = min(w.n, k_keep);
   if (w.n == k_keep) {
     threshold.a = w.a[k_keep - 1]; threshold.b = w.b[k_keep - 1]; threshold.i = w.i[k_keep - 1];
   }
+  __syncwarp();
+}
+
+// every lane may bring one candidate
+__device__ __forceinline__ void topk_append(WarpList& w, bool cand, const Key& key, int k_keep,
+                                            int lane, Key& threshold) {
+  u32 votes = __ballot_sync(0xffffffffu, cand);
+  if (votes == 0) return;
+  if (w.n + __popc(votes) > LIST_CAP) {
+    topk_compact(w, k_keep, lane, threshold);
+    cand = cand && key_less(key, threshold);
+    votes = __ballot_sync(0xffffffffu, cand);
+  }
+  if (cand) {
+    const int p = w.n + __popc(votes & ((1u << lane) - 1u));
+    w.a[p] = key.a; w.b[p] = key.b; w.i[p] = key.i;
+  }
+  w.n += __popc(votes);
+  __syncwarp();
 }
 
 // ------------------------------------------------------------------ block sort / prune
@@ -226,12 +241,50 @@ struct SweepShared {
   int scount[THREADS];
   int warp_n[WARPS];
   u32 warp_survivors[WARPS];
+  u32 next_unit;
   ModelRec rec;
 };
 
 // ------------------------------------------------------------------ the sweep
-template <int KIND>
-__global__ void __launch_bounds__(THREADS) k_sweep(SpaceDev sp, SweepArgs args) {
+// bits of a triple's static description
+enum : u32 {
+  T_THETA_AVAIL = 1u << 0, T_GRAD_COVER = 1u << 1, T_SC = 1u << 2, T_HOST = 1u << 3,
+  T_M_OR_O = 1u << 4, T_EXT0 = 1u << 5
+};
+
+__device__ __forceinline__ u32 triple_bits(u32 th, u32 om, u32 gr, bool d1) {
+  const bool on_shard = in_set(SET_UPDATE_ON_SHARD, om);
+  const bool omega_full = (om == PS_MODE_R) || (d1 && in_set(SET_SHARDLIKE, om));
+  const bool theta_avail = in_set(SET_THETA_ALWAYS, th) || (th == PS_MODE_S && d1) ||
+                           (th == PS_MODE_M && omega_full);
+  const bool grad_cover = d1 || on_shard || in_set(SET_GRAD_FULL, gr);
+  const u32 seen = (1u << th) | (1u << om) | (1u << gr);
+  // data-axis traffic beyond Theorem 2: none with a single replica (nothing moves)
+  const bool ext0 = d1 || !((th == PS_MODE_O) || (th == PS_MODE_R && on_shard) ||
+                            in_set((1u << PS_MODE_SG) | SET_M_OR_O, gr) || om == PS_MODE_SG);
+  return (theta_avail ? T_THETA_AVAIL : 0) | (grad_cover ? T_GRAD_COVER : 0) |
+         (om != PS_MODE_M ? T_SC : 0) | ((seen >> PS_MODE_O) & 1u ? T_HOST : 0) |
+         ((seen & SET_M_OR_O) ? T_M_OR_O : 0) | (ext0 ? T_EXT0 : 0);
+}
+
+// which activation digits give a point with every required flag, for a triple
+// with static bits `tb` (the composition bits are checked per unit)
+__device__ __forceinline__ u32 allowed_act_digits(u32 tb, u32 req, u32 all, u32 own, u32 is_o, u32 not_mo) {
+  u32 ok = all;
+  if ((req & PS_F_SC) && !(tb & T_SC)) ok = 0;
+  if ((req & PS_F_THETA_AVAIL) && !(tb & T_THETA_AVAIL)) ok = 0;
+  if ((req & PS_F_GRAD_COVER) && !(tb & T_GRAD_COVER)) ok = 0;
+  if (req & PS_F_GI) ok &= ((tb & T_THETA_AVAIL) && (tb & T_GRAD_COVER)) ? own : 0;
+  if (req & PS_F_ACT_AVAIL) ok &= own;
+  if (req & PS_F_USES_HOST) ok &= (tb & T_HOST) ? all : is_o;
+  if (req & PS_F_PAPER_PRICED) ok &= ((tb & T_EXT0) && !(tb & T_M_OR_O)) ? not_mo : 0;
+  return ok;
+}
+
+template <int KIND, int NM>
+__global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs args) {
+  constexpr int N2 = NM * NM, N3 = NM * NM * NM, NC = N3 * NM;
+  constexpr int R = (N3 + 31) / 32;                 // triples per lane
   extern __shared__ __align__(16) unsigned char smem_raw[];
   SweepShared& sh = *reinterpret_cast<SweepShared*>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -240,8 +293,11 @@ __global__ void __launch_bounds__(THREADS) k_sweep(SpaceDev sp, SweepArgs args) 
   // stage the model record with 16-byte loads (6 x 16 B)
   if (tid < (int)(sizeof(ModelRec) / 16))
     reinterpret_cast<uint4*>(&sh.rec)[tid] = reinterpret_cast<const uint4*>(&sp.recs[model])[tid];
+  const u32 u_begin = (u32)(((u64)blockIdx.x * sp.n_facts) / gridDim.x);
+  const u32 u_end = (u32)(((u64)(blockIdx.x + 1) * sp.n_facts) / gridDim.x);
+  if (tid == 0) sh.next_unit = u_begin + WARPS;
   __syncthreads();
-  const ModelRec rec = sh.rec;
+  const ModelRec& rec = sh.rec;
 
   WarpTables& tb = sh.tables[warp];
   WarpList list{sh.list_a + warp * LIST_CAP, sh.list_b + warp * LIST_CAP,
@@ -249,24 +305,55 @@ __global__ void __launch_bounds__(THREADS) k_sweep(SpaceDev sp, SweepArgs args) 
   const int k_keep = (int)args.k_keep;
   Key threshold{U64MAX, U64MAX, 0xffffffffu};
   u32 survivors = 0;
+  u64 dom_m = U64MAX, dom_c = U64MAX;               // Pareto: a point known to be a survivor
 
   const u32 req = args.require_flags;
   const bool ext_in_objective = args.comm_kind == PS_COMM_PAPER_PLUS_EXT;
-  const u32 per_unit = sp.nvt * sp.n_codes;
-  const u32 u_begin = (u32)(((u64)chunk * sp.n_facts) / n_chunks);
-  const u32 u_end = (u32)(((u64)(chunk + 1) * sp.n_facts) / n_chunks);
+  const u32 nvt = sp.nvt;
+  const u32 per_unit = nvt * NC;
+  // capacities as exclusive bounds (memory and host bytes stay below 2^63)
+  const u64 cap_x = min(args.cap_max, (u64)1 << 62) + 1;
+  const u64 host_x = min(args.host_cap, (u64)1 << 62) + 1;
+  constexpr u32 CV_BITS = PS_F_CV | PS_F_T_DIV_HEADS | PS_F_K_DIV_LAYERS | PS_F_TP_LE_MAX | PS_F_AXIS_FORM;
+  const u32 req_cv = req & CV_BITS;
 
-  for (u32 unit = u_begin + warp; unit < u_end; unit += WARPS) {
+  // activation-digit classes (Theorem 3: a replica needs its own activations)
+  u32 all = (1u << NM) - 1u, own = 0, is_o = 0, not_mo = 0;
+#pragma unroll
+  for (int d = 0; d < NM; ++d) {
+    const u32 ac = digit_mode(sp.modemap, d);
+    if (in_set(SET_ACT_OWN, ac)) own |= 1u << d;
+    if (ac == PS_MODE_O) is_o |= 1u << d;
+    if (!in_set(SET_M_OR_O, ac)) not_mo |= 1u << d;
+  }
+
+  // this lane's triples: modes, table offsets and allowed digits are the same for every unit
+  u32 t_local[R];      // triple number (0 if the lane has none in this round)
+  u32 t_modes[R];      // th | om << 3 | gr << 6 | on_shard << 9
+  u32 t_allowed[R];    // allowed activation digits: bits 0..4 for D > 1, bits 8..12 for D = 1
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const u32 t = lane + 32 * r;
+    const bool live = t < (u32)N3;
+    const u32 tt = live ? t : 0;
+    const u32 th = digit_mode(sp.modemap, tt % NM), om = digit_mode(sp.modemap, (tt / NM) % NM),
+              gr = digit_mode(sp.modemap, tt / N2);
+    t_local[r] = tt;
+    t_modes[r] = th | (om << 3) | (gr << 6) | (in_set(SET_UPDATE_ON_SHARD, om) ? 1u << 9 : 0);
+    const u32 a_many = allowed_act_digits(triple_bits(th, om, gr, false), req, all, own, is_o, not_mo);
+    const u32 a_one = allowed_act_digits(triple_bits(th, om, gr, true), req, all, all, is_o, not_mo);
+    t_allowed[r] = live ? (a_many | (a_one << 8)) : 0;
+  }
+
+  // warps take the block's units in turn: the first one by warp number, then
+  // whichever is next when they finish (their work differs with the candidates)
+  for (u32 unit = u_begin + warp; unit < u_end;) {
     const Fact f = sp.facts[unit];
     const UnitBase ub = unit_base(rec, f, sp.tp_max_valid, true);
-    const u64 hostT = 3 * ub.sh * rec.wT, hostO = 2 * ub.sh * rec.wO, hostG = 2 * ub.sh * rec.wG;
     __syncwarp();
     if (lane < 5) {
       const u32 pi = lane;
       const u64 pe = mu_elems(pi, ub.E2, ub.sh, ub.u);
-      tb.mem[0][pi] = rec.wT * pe;
-      tb.mem[1][pi] = rec.wO * pe;
-      tb.mem[2][pi] = rec.wG * pe;
       const u64 xT = ub.x * rec.wT, xO = ub.x * rec.wO, xG = ub.x * rec.wG;
       // Theorem 2's terms, plus (if asked for) the traffic it does not price
       u64 ct0 = (pi == PS_MODE_SG) ? 2 * xT : 0, ct1 = ct0, co = 0;
@@ -278,97 +365,166 @@ __global__ void __launch_bounds__(THREADS) k_sweep(SpaceDev sp, SweepArgs args) 
         if (pi == PS_MODE_M) { cg0 += 2 * xG; cg1 += xG; }
         if (pi == PS_MODE_O) { cg0 += xG; cg1 += xG; }
       }
-      tb.c_theta[0][pi] = ct0; tb.c_theta[1][pi] = ct1;
-      tb.c_omega[pi] = co;
-      tb.c_grad[0][pi] = cg0; tb.c_grad[1][pi] = cg1;
-      for (u32 v = 0; v < sp.nv; ++v)
-        for (u32 tau = 0; tau < sp.nt; ++tau) {
-          const ActBase ab = act_base(rec, f, v, tau);
-          tb.act[v * sp.nt + tau][pi] = mu_elems(pi, ab.EA, ab.shA, ab.uA);
-          if (pi == 0) {
-            tb.act_host[v * sp.nt + tau] = 2 * ab.EA;
-            tb.c_axis[v * sp.nt + tau] =
-                ext_in_objective ? model_axis_traffic(rec, f, ub, tau, sp.tp_coll) : 0;
-          }
+      const bool off = (pi == PS_MODE_O);
+      const u64 hT = off ? 3 * ub.sh * rec.wT : 0, hO = off ? 2 * ub.sh * rec.wO : 0,
+                hG = off ? 2 * ub.sh * rec.wG : 0;
+      tb.theta[0][pi] = ModeEntry{rec.wT * pe, ct0, hT, 0};
+      tb.theta[1][pi] = ModeEntry{rec.wT * pe, ct1, hT, 0};
+      tb.omega[pi] = ModeEntry{rec.wO * pe, co, hO, 0};
+      tb.grad[0][pi] = ModeEntry{rec.wG * pe, cg0, hG, 0};
+      tb.grad[1][pi] = ModeEntry{rec.wG * pe, cg1, hG, 0};
+    }
+    {
+      // lane (vt, d): activation bytes of digit d under variant vt, and the bound
+      // a triple's own bytes must stay below for the sum to fit the capacity
+      const u32 vt = lane / NM, d = lane - vt * NM;
+      const bool mine = vt < nvt;
+      const u32 v = mine ? vt / sp.nt : 0, tau = mine ? vt - v * sp.nt : 0;
+      const ActBase ab = act_base(rec, f, v, tau);
+      const u32 ac = digit_mode(sp.modemap, d);
+      const u64 am = mu_elems(ac, ab.EA, ab.shA, ab.uA);
+      const u64 bound = am < cap_x ? cap_x - am : 0;
+      u32 slot = d;
+      if (KIND == PS_REDUCE_PARETO) {
+        // rank of this digit among its variant's digits by (bytes, digit)
+        slot = 0;
+#pragma unroll
+        for (int o = 0; o < NM; ++o) {
+          const u64 other = __shfl_sync(0xffffffffu, am, (vt * NM + o) & 31);
+          if (mine && (other < am || (other == am && (u32)o < d))) ++slot;
         }
+      }
+      if (mine) {
+        tb.bound[vt][slot] = bound;
+        tb.act[vt][slot] = am;
+        tb.digit[vt][slot] = d;
+        if (d == 0) {
+          const u64 ah = 2 * ab.EA;                            // offload after fwd, reload for bwd
+          tb.host_bound[vt] = ah < host_x ? host_x - ah : 0;
+          tb.c_axis[vt] = ext_in_objective ? model_axis_traffic(rec, f, ub, tau, sp.tp_coll) : 0;
+        }
+      }
     }
     __syncwarp();
 
+    // the lane's triples for this unit: own bytes, own communication, allowed digits
+    const bool unit_ok = (ub.cv & req_cv) == req_cv;
+    const u32 a_shift = ub.d1 ? 8 : 0;
+    u64 mem3[R], comm3[R], host3[R];
+    u32 allowed[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const u32 tm = t_modes[r];
+      const u32 th = tm & 7u, om = (tm >> 3) & 7u, gr = (tm >> 6) & 7u, rho = (tm >> 9) & 1u;
+      const ModeEntry et = tb.theta[rho][th], eo = tb.omega[om], eg = tb.grad[rho][gr];
+      mem3[r] = et.mem + eo.mem + eg.mem;
+      comm3[r] = et.comm + eo.comm + eg.comm;
+      host3[r] = et.host + eo.host + eg.host;
+      allowed[r] = (unit_ok && host3[r] < host_x) ? ((t_allowed[r] >> a_shift) & all) : 0;
+    }
     const u32 unit_first = unit * per_unit;      // index of the unit's first point in the model
-    for (u32 t0 = 0; t0 < sp.n3; t0 += 32) {
-      const u32 t = t0 + lane;
-      const bool live = t < sp.n3;
-      const u32 tt = live ? t : 0;
-      const u32 dth = tt % sp.nm, dom = (tt / sp.nm) % sp.nm, dgr = tt / (sp.nm * sp.nm);
-      const u32 th = digit_mode(sp.modemap, dth), om = digit_mode(sp.modemap, dom),
-                gr = digit_mode(sp.modemap, dgr);
-      const u32 on_shard = in_set(SET_UPDATE_ON_SHARD, om) ? 1 : 0;
-      const u64 mem3 = tb.mem[0][th] + tb.mem[1][om] + tb.mem[2][gr];
-      const u64 comm3 = tb.c_theta[on_shard][th] + tb.c_omega[om] + tb.c_grad[on_shard][gr];
-      const u64 host3 = (th == PS_MODE_O ? hostT : 0) + (om == PS_MODE_O ? hostO : 0) +
-                        (gr == PS_MODE_O ? hostG : 0);
-      // which activation modes give a point that has every required flag
-      u32 ok_modes = 0;
-      if (live) {
-        // data-axis traffic beyond Theorem 2 (needed for the paper-priced flag only)
-        const bool ext0 = ub.d1 || !((th == PS_MODE_O) || (th == PS_MODE_R && on_shard) ||
-                                     in_set((1u << PS_MODE_SG) | SET_M_OR_O, gr) || om == PS_MODE_SG);
-        for (u32 da = 0; da < sp.nm; ++da) {
-          const u32 ac = digit_mode(sp.modemap, da);
-          const u32 fl = point_flags(th, om, gr, ac, ub.d1, ub.cv, ext0);
-          if ((fl & req) == req) ok_modes |= 1u << da;
-        }
-      }
-      const bool host3_ok = host3 <= args.host_cap;
 
-      for (u32 vt = 0; vt < sp.nvt; ++vt) {
-        const u64 comm = comm3 + tb.c_axis[vt];
-        const u32 vt_first = unit_first + vt * sp.n_codes + tt;   // + da * n3
-        if (KIND == PS_REDUCE_PARETO) {
-          // same communication for the nm activation modes: the smallest memory
-          // (first on ties) is the only one that can be on the frontier
-          u64 best = U64MAX;
-          u32 best_da = 0;
-          for (u32 da = 0; da < sp.nm; ++da) {
-            const u32 ac = digit_mode(sp.modemap, da);
-            const u64 mem = mem3 + tb.act[vt][ac];
-            const bool host_ok = (ac == PS_MODE_O) ? (host3 + tb.act_host[vt] <= args.host_cap) : host3_ok;
-            if (((ok_modes >> da) & 1u) && host_ok && mem < best) { best = mem; best_da = da; }
-          }
-          const u32 idx = vt_first + best_da * sp.n3;
-          bool cand = best <= args.cap_max;
-          if (cand) cand = !pareto_rejects(list, best, comm, idx);
-          u32 pending = __ballot_sync(0xffffffffu, cand);
-          while (pending) {
-            const int src = __ffs(pending) - 1;
-            pending &= pending - 1;
-            const u64 m = __shfl_sync(0xffffffffu, best, src);
-            const u64 c = __shfl_sync(0xffffffffu, comm, src);
-            const u32 ix = __shfl_sync(0xffffffffu, idx, src);
-            pareto_insert(list, m, c, ix, lane, args.status);
-          }
-        } else {
-          for (u32 da = 0; da < sp.nm; ++da) {
-            const u32 ac = digit_mode(sp.modemap, da);
-            const u64 mem = mem3 + tb.act[vt][ac];
-            const bool host_ok = (ac == PS_MODE_O) ? (host3 + tb.act_host[vt] <= args.host_cap) : host3_ok;
-            const bool pass = ((ok_modes >> da) & 1u) && host_ok && mem <= args.cap_max;
-            survivors += pass ? 1 : 0;
-            const Key key{comm, mem, vt_first + da * sp.n3};
-            u32 pending = __ballot_sync(0xffffffffu, pass && key_less(key, threshold));
+    for (u32 vt = 0; vt < nvt; ++vt) {
+      const u64 c_axis = tb.c_axis[vt], host_bound = tb.host_bound[vt];
+      u32 allow_vt[R];
+      u64 comm[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        comm[r] = comm3[r] + c_axis;
+        // offloading activations adds host bytes: drop that digit if they do not fit
+        allow_vt[r] = (host3[r] < host_bound) ? allowed[r] : (allowed[r] & ~is_o);
+      }
+      const u32 vt_first = unit_first + vt * NC;
+
+      if (KIND == PS_REDUCE_PARETO) {
+        // For a triple and variant the communication is the same for all NM
+        // activation digits, so only the fitting digit with the least bytes
+        // (lowest digit on ties) can be on the frontier: slots are ordered so.
+        u32 best[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) best[r] = NM;
+#pragma unroll
+        for (int k = NM - 1; k >= 0; --k) {
+          const u64 bound = tb.bound[vt][k];
+          const u32 dg = tb.digit[vt][k];
+#pragma unroll
+          for (int r = 0; r < R; ++r)
+            if (mem3[r] < bound && ((allow_vt[r] >> dg) & 1u)) best[r] = k;
+        }
+        bool some = false;
+#pragma unroll
+        for (int r = 0; r < R; ++r) some = some || best[r] < (u32)NM;
+        if (__any_sync(0xffffffffu, some))
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          const bool has = best[r] < (u32)NM;
+          const u32 k = has ? best[r] : 0;
+          const u64 m = mem3[r] + tb.act[vt][k];
+          const u64 c = comm[r];
+          const u32 idx = vt_first + t_local[r] + tb.digit[vt][k] * N3;
+          // cheap test first: strictly dominated by a point already known to survive
+          bool cand = has && !(dom_m <= m && dom_c <= c && (dom_m != m || dom_c != c));
+          if (__any_sync(0xffffffffu, cand)) {
+            if (cand) {
+              int lo = 0, hi = list.n;
+              while (lo < hi) {               // entries with mem <= m
+                const int mid = (lo + hi) >> 1;
+                if (list.a[mid] <= m) lo = mid + 1; else hi = mid;
+              }
+              if (lo > 0) {
+                const u64 em = list.a[lo - 1], ec = list.b[lo - 1];
+                if (ec < c || (ec == c && (em < m || list.i[lo - 1] < idx))) {
+                  cand = false;
+                  dom_m = em; dom_c = ec;
+                }
+              }
+            }
+            u32 pending = __ballot_sync(0xffffffffu, cand);
             while (pending) {
               const int src = __ffs(pending) - 1;
               pending &= pending - 1;
-              Key k;
-              k.a = __shfl_sync(0xffffffffu, key.a, src);
-              k.b = __shfl_sync(0xffffffffu, key.b, src);
-              k.i = __shfl_sync(0xffffffffu, key.i, src);
-              if (key_less(k, threshold)) topk_insert(list, k, k_keep, lane, threshold);
+              const u64 pm = __shfl_sync(0xffffffffu, m, src);
+              const u64 pc = __shfl_sync(0xffffffffu, c, src);
+              const u32 pi = __shfl_sync(0xffffffffu, idx, src);
+              pareto_insert(list, pm, pc, pi, lane, args.status);
             }
+          }
+        }
+      } else {
+        bool above[R];                         // communication already above the k-th smallest
+#pragma unroll
+        for (int r = 0; r < R; ++r) above[r] = comm[r] > threshold.a;
+        u32 hot = 0;                           // digits with a survivor that may enter the list
+#pragma unroll
+        for (int d = 0; d < NM; ++d) {
+          const u64 bound = tb.bound[vt][d];
+          bool any = false;
+#pragma unroll
+          for (int r = 0; r < R; ++r) {
+            const bool pass = mem3[r] < bound && ((allow_vt[r] >> d) & 1u);
+            survivors += pass ? 1u : 0u;
+            any = any || (pass && !above[r]);
+          }
+          if (__any_sync(0xffffffffu, any)) hot |= 1u << d;
+        }
+#pragma unroll 1
+        while (hot) {
+          const u32 d = __ffs(hot) - 1;
+          hot &= hot - 1;
+          const u64 bound = tb.bound[vt][d], am = tb.act[vt][d];
+#pragma unroll
+          for (int r = 0; r < R; ++r) {
+            const bool pass = mem3[r] < bound && ((allow_vt[r] >> d) & 1u);
+            const Key key{comm[r], mem3[r] + am, vt_first + t_local[r] + d * N3};
+            topk_append(list, pass && key_less(key, threshold), key, k_keep, lane, threshold);
           }
         }
       }
     }
+    // next unit
+    u32 nxt = 0;
+    if (lane == 0) nxt = atomicAdd(&sh.next_unit, 1u);
+    unit = __shfl_sync(0xffffffffu, nxt, 0);
   }
 
   // ---- block-level merge of the warps' lists
@@ -511,21 +667,31 @@ __global__ void __launch_bounds__(THREADS) k_sweep_merge(SpaceDev sp, MergeArgs 
 size_t sweep_shared_bytes() { return sizeof(SweepShared); }
 size_t merge_shared_bytes() { return sizeof(MergeShared); }
 
+template <int KIND, int NM>
+static cudaError_t launch_sweep_t(const SpaceDev& sp, const SweepArgs& a, u32 n_chunks, cudaStream_t stream) {
+  dim3 grid(n_chunks, sp.n_models);
+  const size_t smem = sizeof(SweepShared);
+  cudaError_t e = cudaFuncSetAttribute(k_sweep<KIND, NM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  k_sweep<KIND, NM><<<grid, THREADS, smem, stream>>>(sp, a);
+  return cudaGetLastError();
+}
+
+template <int KIND>
+static cudaError_t launch_sweep_k(const SpaceDev& sp, const SweepArgs& a, u32 n_chunks, cudaStream_t stream) {
+  switch (sp.nm) {
+    case 1: return launch_sweep_t<KIND, 1>(sp, a, n_chunks, stream);
+    case 2: return launch_sweep_t<KIND, 2>(sp, a, n_chunks, stream);
+    case 3: return launch_sweep_t<KIND, 3>(sp, a, n_chunks, stream);
+    case 4: return launch_sweep_t<KIND, 4>(sp, a, n_chunks, stream);
+    default: return launch_sweep_t<KIND, 5>(sp, a, n_chunks, stream);
+  }
+}
+
 cudaError_t launch_sweep(int kind, const SpaceDev& sp, const SweepArgs& a, u32 n_chunks,
                          cudaStream_t stream) {
-  dim3 grid(n_chunks, sp.n_models);
-  size_t smem = sizeof(SweepShared);
-  cudaError_t e;
-  if (kind == PS_REDUCE_PARETO) {
-    e = cudaFuncSetAttribute(k_sweep<PS_REDUCE_PARETO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    k_sweep<PS_REDUCE_PARETO><<<grid, THREADS, smem, stream>>>(sp, a);
-  } else {
-    e = cudaFuncSetAttribute(k_sweep<PS_REDUCE_TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    k_sweep<PS_REDUCE_TOPK><<<grid, THREADS, smem, stream>>>(sp, a);
-  }
-  return cudaGetLastError();
+  return kind == PS_REDUCE_PARETO ? launch_sweep_k<PS_REDUCE_PARETO>(sp, a, n_chunks, stream)
+                                  : launch_sweep_k<PS_REDUCE_TOPK>(sp, a, n_chunks, stream);
 }
 
 cudaError_t launch_sweep_merge(int kind, const SpaceDev& sp, const MergeArgs& a, cudaStream_t stream) {

@@ -33,7 +33,7 @@ F_VALID = F_GI | F_SC | F_CV
 COMM_PAPER, COMM_PAPER_PLUS_EXT = 0, 1
 REDUCE_PARETO, REDUCE_TOPK = 0, 1
 NO_LIMIT = (1 << 64) - 1
-TOPK_MAX = 128
+TOPK_MAX = 64
 
 ENTRY_DTYPE = np.dtype([("mem", "<u8"), ("comm", "<u8"), ("host", "<u8"), ("idx", "<u8"),
                         ("flags", "<u4"), ("pad", "<u4")])

@@ -207,7 +207,7 @@ def test_pareto_ragged_space(ctx, ps):
                           os_.sweep(filt, caps, O.KIND_PARETO, 96, n_threads=4))
 
 
-@pytest.mark.parametrize("k", [64, 7, 128])
+@pytest.mark.parametrize("k", [64, 7, 33])
 def test_topk_c4_sample(ctx, ps, k):
     space = synth.config("C4", n_models=3)
     gs, os_ = both(ctx, space)
