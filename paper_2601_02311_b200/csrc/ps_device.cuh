@@ -110,6 +110,44 @@ __device__ __forceinline__ UnitBase unit_base(const ModelRec& r, const Fact& f, 
   return b;
 }
 
+// Degrees that are all powers of two (every benchmark configuration): the
+// divisions become shifts.  Same values as unit_base / act_base.
+struct Pow2 {
+  u32 sT, sK, sD;
+  bool all;
+};
+__device__ __forceinline__ Pow2 pow2_of(const Fact& f) {
+  Pow2 p;
+  p.all = (((f.T & (f.T - 1)) | (f.K & (f.K - 1)) | (f.D & (f.D - 1))) == 0);
+  p.sT = 31 - __clz(f.T);
+  p.sK = 31 - __clz(f.K);
+  p.sD = 31 - __clz(f.D);
+  return p;
+}
+__device__ __forceinline__ u64 ceil_shift(u64 a, u32 s) { return (a + (((u64)1 << s) - 1)) >> s; }
+
+__device__ __forceinline__ UnitBase unit_base_pow2(const ModelRec& r, const Fact& f, const Pow2& p,
+                                                   u32 tp_max_valid, bool axis_form) {
+  UnitBase b;
+  b.E2 = ceil_shift(ceil_shift(r.P, p.sT), p.sK);
+  b.sh = ceil_shift(b.E2, p.sD);
+  b.x = b.E2 - (b.E2 >> p.sD);
+  b.u = ceil_shift(r.unit, p.sT);
+  b.tp_x = r.Sbh - (r.Sbh >> p.sT);
+  b.sbh_t = ceil_shift(r.Sbh, p.sT);
+  b.lps = (r.L + (f.K - 1)) >> p.sK;
+  const bool k_layers = (r.L & (f.K - 1)) == 0;
+  const bool t_heads = (r.heads & (f.T - 1)) == 0;
+  const bool tp_le = f.T <= tp_max_valid;
+  const bool whole = ((u64)f.T * f.K * f.D == (u64)f.N);
+  u32 cv = (t_heads ? PS_F_T_DIV_HEADS : 0) | (k_layers ? PS_F_K_DIV_LAYERS : 0) |
+           (tp_le ? PS_F_TP_LE_MAX : 0) | (axis_form ? PS_F_AXIS_FORM : 0);
+  if (t_heads && k_layers && tp_le && axis_form && whole) cv |= PS_F_CV;
+  b.cv = cv;
+  b.d1 = (f.D == 1);
+  return b;
+}
+
 // Activations of one replica for variant v (stored / checkpointed) when the
 // tensor axis shards them (tau = 0, sequence parallel) or not (tau = 1); the
 // pipeline axis leaves them whole (Table 2).  Bytes.
@@ -121,6 +159,15 @@ __device__ __forceinline__ ActBase act_base(const ModelRec& r, const Fact& f, u3
   a.EA = tau == 0 ? div_ceil(r.A[v], f.T) : r.A[v];
   a.uA = tau == 0 ? div_ceil(r.UA[v], f.T) : r.UA[v];
   a.shA = div_ceil(a.EA, f.D);
+  return a;
+}
+
+__device__ __forceinline__ ActBase act_base_pow2(const ModelRec& r, const Pow2& p, u32 v, u32 tau) {
+  ActBase a;
+  const u32 s = tau == 0 ? p.sT : 0;
+  a.EA = ceil_shift(r.A[v], s);
+  a.uA = ceil_shift(r.UA[v], s);
+  a.shA = ceil_shift(a.EA, p.sD);
   return a;
 }
 

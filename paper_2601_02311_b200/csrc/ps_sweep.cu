@@ -40,13 +40,14 @@ struct WarpTables {
   ModeEntry theta[2][5];   // [update committed on a shard][mode]
   ModeEntry omega[5];
   ModeEntry grad[2][5];
-  // per activation variant vt = (v, tau) and slot k: k is the activation digit
-  // (top-k) or the rank of the digit by activation bytes, ascending (Pareto)
-  u64 bound[4][5];         // a triple whose own bytes are below this fits the capacity
-  u64 act[4][5];           // activation bytes of the slot
-  u32 digit[4][5];         // activation digit of the slot
+  // per activation variant vt = (v, tau) and activation digit d
+  u64 bound[4][5];         // a triple whose own bytes are below this fits the capacity with digit d
+  u64 act[4][5];           // activation bytes of digit d
   u64 host_bound[4];       // a triple whose own host bytes are below this may offload activations
   u64 c_axis[4];           // tensor + pipeline traffic of the variant (0 if not in the objective)
+  // Pareto: for every set of digits the one with the least activation bytes
+  // (lowest digit on ties), NM for the empty set
+  unsigned char least[4][32];
 };
 
 struct Key {
@@ -68,45 +69,51 @@ struct WarpList {
 };
 
 // Pareto staircase: a = mem ascending, b = comm strictly descending.
-// warp-cooperative insertion; all lanes hold the same (m, c, idx)
+// warp-cooperative insertion; all lanes hold the same (m, c, idx).  Entries are
+// handled 32 at a time, so a short staircase (the usual case) takes one round.
 __device__ __noinline__ void pareto_insert(WarpList& w, u64 m, u64 c, u32 idx, int lane,
-                                              u32* status) {
+                                           u32* status) {
   constexpr int PER = LIST_CAP / 32;
+  const int rounds = (w.n + 31) >> 5;
   u64 ea[PER], eb[PER];
   u32 ei[PER];
   int below = 0, killed = 0;
   bool dominated = false;
 #pragma unroll
   for (int k = 0; k < PER; ++k) {
-    int e = lane + 32 * k;
-    bool valid = e < w.n;
-    ea[k] = valid ? w.a[e] : U64MAX;
-    eb[k] = valid ? w.b[e] : 0;
-    ei[k] = valid ? w.i[e] : 0;
-    if (valid && ea[k] == m && eb[k] == c) {          // same pair: smallest index stays
-      if (idx < ei[k]) w.i[e] = idx;
-      dominated = true;
-    } else if (valid && ea[k] <= m && eb[k] <= c) {
-      dominated = true;
+    if (k < rounds) {
+      const int e = lane + 32 * k;
+      const bool valid = e < w.n;
+      ea[k] = valid ? w.a[e] : U64MAX;
+      eb[k] = valid ? w.b[e] : 0;
+      ei[k] = valid ? w.i[e] : 0;
+      if (valid && ea[k] == m && eb[k] == c) {          // same pair: smallest index stays
+        if (idx < ei[k]) w.i[e] = idx;
+        dominated = true;
+      } else if (valid && ea[k] <= m && eb[k] <= c) {
+        dominated = true;
+      }
+      below += __popc(__ballot_sync(0xffffffffu, valid && ea[k] < m));
+      killed += __popc(__ballot_sync(0xffffffffu, valid && ea[k] >= m && eb[k] >= c));
     }
-    below += __popc(__ballot_sync(0xffffffffu, valid && ea[k] < m));
-    killed += __popc(__ballot_sync(0xffffffffu, valid && ea[k] >= m && eb[k] >= c));
   }
   if (__any_sync(0xffffffffu, dominated)) { __syncwarp(); return; }
-  int n_new = w.n - killed + 1;
+  const int n_new = w.n - killed + 1;
   if (n_new > LIST_CAP) {
     if (lane == 0) atomicOr(status, ST_LIST_OVERFLOW);
     return;
   }
   __syncwarp();
-  int shift = 1 - killed;                              // entries after the killed run move by this
+  const int shift = 1 - killed;                        // entries after the killed run move by this
+  if (shift != 0) {
 #pragma unroll
-  for (int k = 0; k < PER; ++k) {
-    int e = lane + 32 * k;
-    if (e < w.n && e >= below + killed && shift != 0) {
-      w.a[e + shift] = ea[k];
-      w.b[e + shift] = eb[k];
-      w.i[e + shift] = ei[k];
+    for (int k = 0; k < PER; ++k) {
+      const int e = lane + 32 * k;
+      if (k < rounds && e < w.n && e >= below + killed) {
+        w.a[e + shift] = ea[k];
+        w.b[e + shift] = eb[k];
+        w.i[e + shift] = ei[k];
+      }
     }
   }
   if (lane == 0) { w.a[below] = m; w.b[below] = c; w.i[below] = idx; }
@@ -119,7 +126,8 @@ __device__ __noinline__ void pareto_insert(WarpList& w, u64 m, u64 c, u32 idx, i
 // keeps the k smallest and tightens the threshold to the k-th; until the first
 // such compaction the threshold is "everything".  A stale threshold only lets
 // extra candidates in, never keeps a wanted one out.
-__device__ __noinline__ void topk_compact(WarpList& w, int k_keep, int lane, Key& threshold) {
+__device__ __noinline__ void topk_compact(WarpList& w, int k_keep, int lane, Key& threshold,
+                                          unsigned long long* block_comm_limit) {
   for (int p = w.n + lane; p < LIST_CAP; p += 32) { w.a[p] = U64MAX; w.b[p] = U64MAX; w.i[p] = 0xffffffffu; }
   __syncwarp();
   for (int k = 2; k <= LIST_CAP; k <<= 1) {
@@ -142,17 +150,20 @@ __device__ __noinline__ void topk_compact(WarpList& w, int k_keep, int lane, Key
   w.n = min(w.n, k_keep);
   if (w.n == k_keep) {
     threshold.a = w.a[k_keep - 1]; threshold.b = w.b[k_keep - 1]; threshold.i = w.i[k_keep - 1];
+    // k points with at most this much communication exist: tell the other warps
+    if (lane == 0) atomicMin(block_comm_limit, (unsigned long long)threshold.a);
   }
   __syncwarp();
 }
 
 // every lane may bring one candidate
 __device__ __forceinline__ void topk_append(WarpList& w, bool cand, const Key& key, int k_keep,
-                                            int lane, Key& threshold) {
+                                            int lane, Key& threshold,
+                                            unsigned long long* block_comm_limit) {
   u32 votes = __ballot_sync(0xffffffffu, cand);
   if (votes == 0) return;
   if (w.n + __popc(votes) > LIST_CAP) {
-    topk_compact(w, k_keep, lane, threshold);
+    topk_compact(w, k_keep, lane, threshold, block_comm_limit);
     cand = cand && key_less(key, threshold);
     votes = __ballot_sync(0xffffffffu, cand);
   }
@@ -242,6 +253,7 @@ struct SweepShared {
   int warp_n[WARPS];
   u32 warp_survivors[WARPS];
   u32 next_unit;
+  unsigned long long block_comm_limit;   // top-k: no point with more communication can matter
   ModelRec rec;
 };
 
@@ -295,7 +307,7 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
     reinterpret_cast<uint4*>(&sh.rec)[tid] = reinterpret_cast<const uint4*>(&sp.recs[model])[tid];
   const u32 u_begin = (u32)(((u64)blockIdx.x * sp.n_facts) / gridDim.x);
   const u32 u_end = (u32)(((u64)(blockIdx.x + 1) * sp.n_facts) / gridDim.x);
-  if (tid == 0) sh.next_unit = u_begin + WARPS;
+  if (tid == 0) { sh.next_unit = u_begin + WARPS; sh.block_comm_limit = U64MAX; }
   __syncthreads();
   const ModelRec& rec = sh.rec;
 
@@ -349,7 +361,9 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
   // whichever is next when they finish (their work differs with the candidates)
   for (u32 unit = u_begin + warp; unit < u_end;) {
     const Fact f = sp.facts[unit];
-    const UnitBase ub = unit_base(rec, f, sp.tp_max_valid, true);
+    const Pow2 p2 = pow2_of(f);
+    const UnitBase ub = p2.all ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
+                               : unit_base(rec, f, sp.tp_max_valid, true);
     __syncwarp();
     if (lane < 5) {
       const u32 pi = lane;
@@ -380,24 +394,11 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
       const u32 vt = lane / NM, d = lane - vt * NM;
       const bool mine = vt < nvt;
       const u32 v = mine ? vt / sp.nt : 0, tau = mine ? vt - v * sp.nt : 0;
-      const ActBase ab = act_base(rec, f, v, tau);
-      const u32 ac = digit_mode(sp.modemap, d);
-      const u64 am = mu_elems(ac, ab.EA, ab.shA, ab.uA);
-      const u64 bound = am < cap_x ? cap_x - am : 0;
-      u32 slot = d;
-      if (KIND == PS_REDUCE_PARETO) {
-        // rank of this digit among its variant's digits by (bytes, digit)
-        slot = 0;
-#pragma unroll
-        for (int o = 0; o < NM; ++o) {
-          const u64 other = __shfl_sync(0xffffffffu, am, (vt * NM + o) & 31);
-          if (mine && (other < am || (other == am && (u32)o < d))) ++slot;
-        }
-      }
+      const ActBase ab = p2.all ? act_base_pow2(rec, p2, v, tau) : act_base(rec, f, v, tau);
+      const u64 am = mu_elems(digit_mode(sp.modemap, d), ab.EA, ab.shA, ab.uA);
       if (mine) {
-        tb.bound[vt][slot] = bound;
-        tb.act[vt][slot] = am;
-        tb.digit[vt][slot] = d;
+        tb.bound[vt][d] = am < cap_x ? cap_x - am : 0;
+        tb.act[vt][d] = am;
         if (d == 0) {
           const u64 ah = 2 * ab.EA;                            // offload after fwd, reload for bwd
           tb.host_bound[vt] = ah < host_x ? host_x - ah : 0;
@@ -406,6 +407,20 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
       }
     }
     __syncwarp();
+    if (KIND == PS_REDUCE_PARETO) {
+      // lane = a set of activation digits; which of them costs the least bytes
+      for (u32 vt = 0; vt < nvt; ++vt) {
+        u64 least = U64MAX;
+        u32 which = NM;
+#pragma unroll
+        for (int d = NM - 1; d >= 0; --d) {
+          const u64 am = tb.act[vt][d];
+          if (((lane >> d) & 1) && am <= least) { least = am; which = d; }
+        }
+        tb.least[vt][lane] = (unsigned char)which;
+      }
+      __syncwarp();
+    }
 
     // the lane's triples for this unit: own bytes, own communication, allowed digits
     const bool unit_ok = (ub.cv & req_cv) == req_cv;
@@ -426,98 +441,132 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
 
     for (u32 vt = 0; vt < nvt; ++vt) {
       const u64 c_axis = tb.c_axis[vt], host_bound = tb.host_bound[vt];
-      u32 allow_vt[R];
-      u64 comm[R];
+      u64 bound[NM];
+#pragma unroll
+      for (int d = 0; d < NM; ++d) bound[d] = tb.bound[vt][d];
+      // every point of (triple, variant): digit d is a survivor if the triple's
+      // bytes are below the digit's bound and the flags allow the digit
+      u32 pass[R];
 #pragma unroll
       for (int r = 0; r < R; ++r) {
-        comm[r] = comm3[r] + c_axis;
+        u32 fit = 0;
+#pragma unroll
+        for (int d = 0; d < NM; ++d) fit |= (mem3[r] < bound[d]) ? (1u << d) : 0u;
         // offloading activations adds host bytes: drop that digit if they do not fit
-        allow_vt[r] = (host3[r] < host_bound) ? allowed[r] : (allowed[r] & ~is_o);
+        const u32 allow_vt = (host3[r] < host_bound) ? allowed[r] : (allowed[r] & ~is_o);
+        pass[r] = fit & allow_vt;
       }
       const u32 vt_first = unit_first + vt * NC;
 
       if (KIND == PS_REDUCE_PARETO) {
         // For a triple and variant the communication is the same for all NM
-        // activation digits, so only the fitting digit with the least bytes
-        // (lowest digit on ties) can be on the frontier: slots are ordered so.
-        u32 best[R];
-#pragma unroll
-        for (int r = 0; r < R; ++r) best[r] = NM;
-#pragma unroll
-        for (int k = NM - 1; k >= 0; --k) {
-          const u64 bound = tb.bound[vt][k];
-          const u32 dg = tb.digit[vt][k];
-#pragma unroll
-          for (int r = 0; r < R; ++r)
-            if (mem3[r] < bound && ((allow_vt[r] >> dg) & 1u)) best[r] = k;
-        }
+        // activation digits, so of the surviving digits only the one with the
+        // least bytes (lowest digit on ties) can be on the frontier.
         bool some = false;
 #pragma unroll
-        for (int r = 0; r < R; ++r) some = some || best[r] < (u32)NM;
-        if (__any_sync(0xffffffffu, some))
+        for (int r = 0; r < R; ++r) some = some || pass[r] != 0;
+        if (__any_sync(0xffffffffu, some)) {
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-          const bool has = best[r] < (u32)NM;
-          const u32 k = has ? best[r] : 0;
-          const u64 m = mem3[r] + tb.act[vt][k];
-          const u64 c = comm[r];
-          const u32 idx = vt_first + t_local[r] + tb.digit[vt][k] * N3;
-          // cheap test first: strictly dominated by a point already known to survive
-          bool cand = has && !(dom_m <= m && dom_c <= c && (dom_m != m || dom_c != c));
-          if (__any_sync(0xffffffffu, cand)) {
-            if (cand) {
-              int lo = 0, hi = list.n;
-              while (lo < hi) {               // entries with mem <= m
-                const int mid = (lo + hi) >> 1;
-                if (list.a[mid] <= m) lo = mid + 1; else hi = mid;
-              }
-              if (lo > 0) {
-                const u64 em = list.a[lo - 1], ec = list.b[lo - 1];
-                if (ec < c || (ec == c && (em < m || list.i[lo - 1] < idx))) {
-                  cand = false;
-                  dom_m = em; dom_c = ec;
+          for (int r = 0; r < R; ++r) {
+            const bool has = pass[r] != 0;
+            const u32 d = has ? tb.least[vt][pass[r]] : 0;
+            const u64 m = mem3[r] + tb.act[vt][d];
+            const u64 c = comm3[r] + c_axis;
+            const u32 idx = vt_first + t_local[r] + d * N3;
+            // cheap test first: strictly dominated by a point already known to survive
+            bool cand = has && !(dom_m <= m && dom_c <= c && (dom_m != m || dom_c != c));
+            if (__any_sync(0xffffffffu, cand)) {
+              if (cand) {
+                int lo = 0, hi = list.n;
+                while (lo < hi) {               // entries with mem <= m
+                  const int mid = (lo + hi) >> 1;
+                  if (list.a[mid] <= m) lo = mid + 1; else hi = mid;
+                }
+                if (lo > 0) {
+                  const u64 em = list.a[lo - 1], ec = list.b[lo - 1];
+                  if (ec < c || (ec == c && (em < m || list.i[lo - 1] < idx))) {
+                    cand = false;
+                    dom_m = em; dom_c = ec;
+                  }
                 }
               }
-            }
-            u32 pending = __ballot_sync(0xffffffffu, cand);
-            while (pending) {
-              const int src = __ffs(pending) - 1;
-              pending &= pending - 1;
-              const u64 pm = __shfl_sync(0xffffffffu, m, src);
-              const u64 pc = __shfl_sync(0xffffffffu, c, src);
-              const u32 pi = __shfl_sync(0xffffffffu, idx, src);
-              pareto_insert(list, pm, pc, pi, lane, args.status);
+              u32 pending = __ballot_sync(0xffffffffu, cand);
+              while (pending) {
+                const int src = __ffs(pending) - 1;
+                pending &= pending - 1;
+                const u64 pm = __shfl_sync(0xffffffffu, m, src);
+                const u64 pc = __shfl_sync(0xffffffffu, c, src);
+                const u32 pi = __shfl_sync(0xffffffffu, idx, src);
+                pareto_insert(list, pm, pc, pi, lane, args.status);
+              }
             }
           }
         }
       } else {
-        bool above[R];                         // communication already above the k-th smallest
+        // the k-th smallest communication known to this warp or to any warp of the block
+        const u64 comm_limit = min(threshold.a, (u64)sh.block_comm_limit);
+        bool hot = false;
 #pragma unroll
-        for (int r = 0; r < R; ++r) above[r] = comm[r] > threshold.a;
-        u32 hot = 0;                           // digits with a survivor that may enter the list
-#pragma unroll
-        for (int d = 0; d < NM; ++d) {
-          const u64 bound = tb.bound[vt][d];
-          bool any = false;
-#pragma unroll
-          for (int r = 0; r < R; ++r) {
-            const bool pass = mem3[r] < bound && ((allow_vt[r] >> d) & 1u);
-            survivors += pass ? 1u : 0u;
-            any = any || (pass && !above[r]);
-          }
-          if (__any_sync(0xffffffffu, any)) hot |= 1u << d;
+        for (int r = 0; r < R; ++r) {
+          survivors += __popc(pass[r]);
+          hot = hot || (pass[r] != 0 && comm3[r] + c_axis <= comm_limit);
         }
-#pragma unroll 1
-        while (hot) {
-          const u32 d = __ffs(hot) - 1;
-          hot &= hot - 1;
-          const u64 bound = tb.bound[vt][d], am = tb.act[vt][d];
+        if (__any_sync(0xffffffffu, hot)) {
+          // survivors that are below the threshold key, per triple as digit bits
+          u32 cand[R];
+          u32 mine = 0;
 #pragma unroll
           for (int r = 0; r < R; ++r) {
-            const bool pass = mem3[r] < bound && ((allow_vt[r] >> d) & 1u);
-            const Key key{comm[r], mem3[r] + am, vt_first + t_local[r] + d * N3};
-            topk_append(list, pass && key_less(key, threshold), key, k_keep, lane, threshold);
+            const u64 c = comm3[r] + c_axis;
+            cand[r] = (c < threshold.a && c <= comm_limit) ? pass[r] : 0u;
+            if (c == threshold.a && pass[r] != 0) {
+#pragma unroll
+              for (int d = 0; d < NM; ++d) {
+                const Key key{c, mem3[r] + tb.act[vt][d], vt_first + t_local[r] + d * N3};
+                if (((pass[r] >> d) & 1u) && key_less(key, threshold)) cand[r] |= 1u << d;
+              }
+            }
+            mine += __popc(cand[r]);
           }
+          u32 incl = mine;                               // inclusive prefix sum over the lanes
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const u32 up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+          }
+          const u32 total = __shfl_sync(0xffffffffu, incl, 31);
+          if (total != 0 && list.n + total <= (u32)LIST_CAP) {
+            int p = list.n + (int)(incl - mine);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+              u32 bits = cand[r];
+              while (bits) {
+                const u32 d = __ffs(bits) - 1;
+                bits &= bits - 1;
+                list.a[p] = comm3[r] + c_axis;
+                list.b[p] = mem3[r] + tb.act[vt][d];
+                list.i[p] = vt_first + t_local[r] + d * N3;
+                ++p;
+              }
+            }
+            list.n += (int)total;
+            __syncwarp();
+          } else if (total != 0) {
+            // does not fit in one go: one (triple round, digit) at a time, compacting as needed
+#pragma unroll 1
+            for (u32 d = 0; d < (u32)NM; ++d) {
+              const u64 am = tb.act[vt][d];
+#pragma unroll
+              for (int r = 0; r < R; ++r) {
+                const Key key{comm3[r] + c_axis, mem3[r] + am, vt_first + t_local[r] + d * N3};
+                topk_append(list, ((cand[r] >> d) & 1u) && key_less(key, threshold), key, k_keep, lane,
+                            threshold, &sh.block_comm_limit);
+              }
+            }
+          }
+          // the first k candidates give the first threshold
+          if (threshold.i == 0xffffffffu && threshold.a == U64MAX && list.n >= k_keep)
+            topk_compact(list, k_keep, lane, threshold, &sh.block_comm_limit);
         }
       }
     }
