@@ -86,8 +86,9 @@ int enqueue_status_copy(ps_ctx* ctx) {
 }
 
 u32 pick_chunks(const ps_ctx* ctx, const ps_space* sp) {
-  // enough blocks for about eight waves of four resident blocks per SM
-  const u64 target = (u64)ctx->sm_count * 4 * 8;
+  // enough blocks for about six waves of three resident blocks per SM; every
+  // extra block of a model builds its lists from scratch, so no more than that
+  const u64 target = (u64)ctx->sm_count * 3 * 6;
   u64 c = (target + sp->dev.n_models - 1) / sp->dev.n_models;
   if (c < 1) c = 1;
   if (c > SWEEP_MAX_CHUNKS) c = SWEEP_MAX_CHUNKS;

@@ -45,6 +45,7 @@ struct WarpTables {
   u64 act[4][5];           // activation bytes of digit d
   u64 host_bound[4];       // a triple whose own host bytes are below this may offload activations
   u64 c_axis[4];           // tensor + pipeline traffic of the variant (0 if not in the objective)
+  u64 c_axis_least;        // the least of them
   // Pareto: for every set of digits the one with the least activation bytes
   // (lowest digit on ties), NM for the empty set
   unsigned char least[4][32];
@@ -69,10 +70,26 @@ struct WarpList {
 };
 
 // Pareto staircase: a = mem ascending, b = comm strictly descending.
+// A coarse staircase shared by the warps of a block: stair[j] is the least
+// communication of any survivor inserted so far whose bytes fall in bucket j or
+// a lower one (buckets: leading bit and the two bits after it, so a lower bucket
+// means strictly fewer bytes).  A candidate in bucket B with at least
+// stair[B-1] communication is strictly dominated.
+constexpr int STAIR = 256;
+__device__ __forceinline__ int stair_bucket(u64 m) {
+  if (m < 4) return (int)m;
+  const int top = 63 - __clzll((long long)m);
+  return 4 * (top - 1) + (int)((m >> (top - 2)) & 3);
+}
+__device__ __forceinline__ void stair_publish(unsigned long long* stair, u64 m, u64 c, int lane) {
+  for (int j = stair_bucket(m) + lane; j < STAIR; j += 32)
+    if (stair[j] > c) atomicMin(&stair[j], (unsigned long long)c);
+}
+
 // warp-cooperative insertion; all lanes hold the same (m, c, idx).  Entries are
 // handled 32 at a time, so a short staircase (the usual case) takes one round.
 __device__ __noinline__ void pareto_insert(WarpList& w, u64 m, u64 c, u32 idx, int lane,
-                                           u32* status) {
+                                           u32* status, unsigned long long* stair) {
   constexpr int PER = LIST_CAP / 32;
   const int rounds = (w.n + 31) >> 5;
   u64 ea[PER], eb[PER];
@@ -118,6 +135,7 @@ __device__ __noinline__ void pareto_insert(WarpList& w, u64 m, u64 c, u32 idx, i
   }
   if (lane == 0) { w.a[below] = m; w.b[below] = c; w.i[below] = idx; }
   w.n = n_new;
+  stair_publish(stair, m, c, lane);
   __syncwarp();
 }
 
@@ -240,6 +258,7 @@ __device__ __forceinline__ int next_pow2(int n) {
   return p;
 }
 
+static_assert(STAIR == THREADS, "the staircase is cleared one entry per thread");
 struct SweepShared {
   WarpTables tables[WARPS];
   u64 list_a[BLOCK_CAP];
@@ -254,6 +273,7 @@ struct SweepShared {
   u32 warp_survivors[WARPS];
   u32 next_unit;
   unsigned long long block_comm_limit;   // top-k: no point with more communication can matter
+  unsigned long long stair[STAIR];       // Pareto: coarse staircase of the block
   ModelRec rec;
 };
 
@@ -308,6 +328,7 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
   const u32 u_begin = (u32)(((u64)blockIdx.x * sp.n_facts) / gridDim.x);
   const u32 u_end = (u32)(((u64)(blockIdx.x + 1) * sp.n_facts) / gridDim.x);
   if (tid == 0) { sh.next_unit = u_begin + WARPS; sh.block_comm_limit = U64MAX; }
+  if (KIND == PS_REDUCE_PARETO) sh.stair[tid] = U64MAX;   // STAIR == THREADS
   __syncthreads();
   const ModelRec& rec = sh.rec;
 
@@ -326,6 +347,7 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
   // capacities as exclusive bounds (memory and host bytes stay below 2^63)
   const u64 cap_x = min(args.cap_max, (u64)1 << 62) + 1;
   const u64 host_x = min(args.host_cap, (u64)1 << 62) + 1;
+  const bool host_limited = args.host_cap < ((u64)1 << 62);
   constexpr u32 CV_BITS = PS_F_CV | PS_F_T_DIV_HEADS | PS_F_K_DIV_LAYERS | PS_F_TP_LE_MAX | PS_F_AXIS_FORM;
   const u32 req_cv = req & CV_BITS;
 
@@ -396,32 +418,24 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
       const u32 v = mine ? vt / sp.nt : 0, tau = mine ? vt - v * sp.nt : 0;
       const ActBase ab = p2.all ? act_base_pow2(rec, p2, v, tau) : act_base(rec, f, v, tau);
       const u64 am = mu_elems(digit_mode(sp.modemap, d), ab.EA, ab.shA, ab.uA);
+      u64 axis = U64MAX;
       if (mine) {
         tb.bound[vt][d] = am < cap_x ? cap_x - am : 0;
         tb.act[vt][d] = am;
         if (d == 0) {
           const u64 ah = 2 * ab.EA;                            // offload after fwd, reload for bwd
           tb.host_bound[vt] = ah < host_x ? host_x - ah : 0;
-          tb.c_axis[vt] = ext_in_objective ? model_axis_traffic(rec, f, ub, tau, sp.tp_coll) : 0;
+          axis = ext_in_objective ? model_axis_traffic(rec, f, ub, tau, sp.tp_coll) : 0;
+          tb.c_axis[vt] = axis;
         }
       }
+      // least axis traffic over the variants (lanes 0, NM, 2 NM, 3 NM hold them)
+      u64 least_axis = axis;
+#pragma unroll
+      for (int o = 1; o < 4; ++o) least_axis = min(least_axis, __shfl_sync(0xffffffffu, axis, (o * NM) & 31));
+      if (lane == 0) tb.c_axis_least = least_axis;
     }
     __syncwarp();
-    if (KIND == PS_REDUCE_PARETO) {
-      // lane = a set of activation digits; which of them costs the least bytes
-      for (u32 vt = 0; vt < nvt; ++vt) {
-        u64 least = U64MAX;
-        u32 which = NM;
-#pragma unroll
-        for (int d = NM - 1; d >= 0; --d) {
-          const u64 am = tb.act[vt][d];
-          if (((lane >> d) & 1) && am <= least) { least = am; which = d; }
-        }
-        tb.least[vt][lane] = (unsigned char)which;
-      }
-      __syncwarp();
-    }
-
     // the lane's triples for this unit: own bytes, own communication, allowed digits
     const bool unit_ok = (ub.cv & req_cv) == req_cv;
     const u32 a_shift = ub.d1 ? 8 : 0;
@@ -439,6 +453,67 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
     }
     const u32 unit_first = unit * per_unit;      // index of the unit's first point in the model
 
+    // ---- evaluation pass: every point of the unit.  Point (triple r, variant vt,
+    // digit d) is a survivor if the flags allow the digit, the triple's bytes are
+    // below the (variant, digit) bound and, for the offload digit, the host bytes
+    // fit.  Survivors are counted per triple.
+    u32 n_pass[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) n_pass[r] = 0;
+#pragma unroll
+    for (int d = 0; d < NM; ++d) {
+      bool allow[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) allow[r] = (allowed[r] >> d) & 1u;
+      const bool host_check = host_limited && ((is_o >> d) & 1u);
+#pragma unroll
+      for (int vt = 0; vt < 4; ++vt) {
+        if ((u32)vt < nvt) {
+          const u64 bound = tb.bound[vt][d];
+          if (host_check) {
+            const u64 host_bound = tb.host_bound[vt];
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+              n_pass[r] += (allow[r] && mem3[r] < bound && host3[r] < host_bound) ? 1u : 0u;
+          } else {
+#pragma unroll
+            for (int r = 0; r < R; ++r) n_pass[r] += (allow[r] && mem3[r] < bound) ? 1u : 0u;
+          }
+        }
+      }
+    }
+
+    // ---- reduction pass, only if some survivor of this warp can matter
+    bool matters = false;
+    if (KIND == PS_REDUCE_PARETO) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) matters = matters || n_pass[r] != 0;
+    } else {
+      const u64 comm_limit = min(threshold.a, (u64)sh.block_comm_limit);
+      const u64 least_axis = tb.c_axis_least;
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        survivors += n_pass[r];
+        matters = matters || (n_pass[r] != 0 && comm3[r] + least_axis <= comm_limit);
+      }
+    }
+    if (__any_sync(0xffffffffu, matters)) {
+    if (KIND == PS_REDUCE_PARETO) {
+      // lane = a set of activation digits; which of them costs the least bytes
+      for (u32 vt = 0; vt < nvt; ++vt) {
+        u64 least = U64MAX;
+        u32 which = NM;
+#pragma unroll
+        for (int d = NM - 1; d >= 0; --d) {
+          const u64 am = tb.act[vt][d];
+          if (((lane >> d) & 1) && am <= least) { least = am; which = d; }
+        }
+        tb.least[vt][lane] = (unsigned char)which;
+      }
+      __syncwarp();
+    }
+
+#pragma unroll 1
     for (u32 vt = 0; vt < nvt; ++vt) {
       const u64 c_axis = tb.c_axis[vt], host_bound = tb.host_bound[vt];
       u64 bound[NM];
@@ -473,8 +548,12 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
             const u64 m = mem3[r] + tb.act[vt][d];
             const u64 c = comm3[r] + c_axis;
             const u32 idx = vt_first + t_local[r] + d * N3;
-            // cheap test first: strictly dominated by a point already known to survive
+            // cheap tests first: strictly dominated by a point already known to survive
             bool cand = has && !(dom_m <= m && dom_c <= c && (dom_m != m || dom_c != c));
+            if (cand) {
+              const int bucket = stair_bucket(m);
+              if (bucket > 0 && sh.stair[bucket - 1] <= c) cand = false;
+            }
             if (__any_sync(0xffffffffu, cand)) {
               if (cand) {
                 int lo = 0, hi = list.n;
@@ -497,7 +576,7 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
                 const u64 pm = __shfl_sync(0xffffffffu, m, src);
                 const u64 pc = __shfl_sync(0xffffffffu, c, src);
                 const u32 pi = __shfl_sync(0xffffffffu, idx, src);
-                pareto_insert(list, pm, pc, pi, lane, args.status);
+                pareto_insert(list, pm, pc, pi, lane, args.status, sh.stair);
               }
             }
           }
@@ -508,7 +587,6 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
         bool hot = false;
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-          survivors += __popc(pass[r]);
           hot = hot || (pass[r] != 0 && comm3[r] + c_axis <= comm_limit);
         }
         if (__any_sync(0xffffffffu, hot)) {
@@ -569,6 +647,7 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
             topk_compact(list, k_keep, lane, threshold, &sh.block_comm_limit);
         }
       }
+    }
     }
     // next unit
     u32 nxt = 0;
