@@ -176,8 +176,9 @@ __device__ __forceinline__ ActBase act_base_pow2(const ModelRec& r, const Pow2& 
 // devices; one boundary tensor forward and one backward between stages
 __device__ __forceinline__ u64 model_axis_traffic(const ModelRec& r, const Fact& f,
                                                   const UnitBase& b, u32 tau, u32 tp_coll) {
-  u64 tp = (u64)b.lps * tp_coll * 2 * b.tp_x * r.wA;
-  u64 pp = (f.K > 1) ? 2 * (tau == 0 ? b.sbh_t : r.Sbh) * r.wA : 0;
+  const u32 per_elem = 2 * tp_coll * r.wA;                 // <= 2 * 64 * 16
+  const u64 tp = b.tp_x * (u64)(b.lps * per_elem);         // lps <= 2^10
+  const u64 pp = (f.K > 1) ? (tau == 0 ? b.sbh_t : r.Sbh) * (u64)(2 * r.wA) : 0;
   return tp + pp;
 }
 

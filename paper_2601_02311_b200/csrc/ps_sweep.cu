@@ -30,18 +30,14 @@ constexpr int LIST_CAP = SWEEP_LIST_CAP;       // entries per warp list / per pa
 constexpr int BLOCK_CAP = WARPS * LIST_CAP;    // union of the warps' lists
 constexpr u64 U64MAX = ~0ull;
 
-// per-warp tables, rebuilt for every unit.  One entry per (state, mode): what
-// that state contributes to memory, to the objective communication and to the
-// host-link bytes (Theorem 1, Theorem 2 plus unpriced traffic, mode O).
-struct __align__(16) ModeEntry {
-  u64 mem, comm, host, pad;
-};
+// per-warp tables, rebuilt for every unit: what depends on the activation
+// variant and digit.  (What depends on the (Theta, Omega, G) triple needs no
+// table: see the per-lane coefficients in k_sweep.)
 struct WarpTables {
-  ModeEntry theta[2][5];   // [update committed on a shard][mode]
-  ModeEntry omega[5];
-  ModeEntry grad[2][5];
   // per activation variant vt = (v, tau) and activation digit d
-  u64 bound[4][5];         // a triple whose own bytes are below this fits the capacity with digit d
+  // a triple whose own bytes are below bound[d][vt] fits the capacity with digit d
+  // under variant vt (0 for variants the space does not have)
+  __align__(16) u64 bound[5][4];
   u64 act[4][5];           // activation bytes of digit d
   u64 host_bound[4];       // a triple whose own host bytes are below this may offload activations
   u64 c_axis[4];           // tensor + pipeline traffic of the variant (0 if not in the objective)
@@ -278,6 +274,27 @@ struct SweepShared {
 };
 
 // ------------------------------------------------------------------ the sweep
+// a * k + acc for a 64-bit a and a small 32-bit k: two multiply-adds
+__device__ __forceinline__ u64 mad_small(u64 a, u32 k, u64 acc) {
+  u64 r = (u64)(u32)a * (u64)k + acc;
+  r += (u64)((u32)(a >> 32) * k) << 32;
+  return r;
+}
+
+// n += (m >= bound): a 64-bit subtraction whose borrow is folded into the
+// counter by one more subtract-with-borrow (n - (0xffffffff + borrow) = n + 1 - borrow)
+__device__ __forceinline__ void count_not_below(u32& n, u64 m, u64 bound) {
+  u32 scratch;
+  asm("{\n\t"
+      "sub.cc.u32 %1, %2, %4;\n\t"
+      "subc.cc.u32 %1, %3, %5;\n\t"
+      "subc.u32 %0, %0, 0xffffffff;\n\t"
+      "}"
+      : "+r"(n), "=r"(scratch)
+      : "r"((u32)m), "r"((u32)(m >> 32)), "r"((u32)bound), "r"((u32)(bound >> 32)));
+  (void)scratch;
+}
+
 // bits of a triple's static description
 enum : u32 {
   T_THETA_AVAIL = 1u << 0, T_GRAD_COVER = 1u << 1, T_SC = 1u << 2, T_HOST = 1u << 3,
@@ -314,7 +331,7 @@ __device__ __forceinline__ u32 allowed_act_digits(u32 tb, u32 req, u32 all, u32 
 }
 
 template <int KIND, int NM>
-__global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs args) {
+__global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs args) {
   constexpr int N2 = NM * NM, N3 = NM * NM * NM, NC = N3 * NM;
   constexpr int R = (N3 + 31) / 32;                 // triples per lane
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -361,19 +378,52 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
     if (!in_set(SET_M_OR_O, ac)) not_mo |= 1u << d;
   }
 
-  // this lane's triples: modes, table offsets and allowed digits are the same for every unit
+  // This lane's triples.  With E = elements of a state on one (t, k) position,
+  // s = its largest data-axis shard, u = the reconstruction unit and x = the ring
+  // volume in elements (all four the same for Theta, Omega and G), a triple's
+  //   bytes          = ka * E + kb * s + kc * u     (Theorem 1, widths of Remark 1)
+  //   communication  = kx * x                       (Theorem 2 [+ unpriced traffic])
+  //   host bytes     = kh * s                       (mode O)
+  // with small integer coefficients that depend only on the triple's modes and
+  // the model's byte widths -- fixed for the whole kernel.
   u32 t_local[R];      // triple number (0 if the lane has none in this round)
-  u32 t_modes[R];      // th | om << 3 | gr << 6 | on_shard << 9
   u32 t_allowed[R];    // allowed activation digits: bits 0..4 for D > 1, bits 8..12 for D = 1
+  u32 ka[R], kb[R], kc[R], kx[R], kh[R];
 #pragma unroll
   for (int r = 0; r < R; ++r) {
     const u32 t = lane + 32 * r;
     const bool live = t < (u32)N3;
     const u32 tt = live ? t : 0;
-    const u32 th = digit_mode(sp.modemap, tt % NM), om = digit_mode(sp.modemap, (tt / NM) % NM),
-              gr = digit_mode(sp.modemap, tt / N2);
+    const u32 modes[3] = {digit_mode(sp.modemap, tt % NM), digit_mode(sp.modemap, (tt / NM) % NM),
+                          digit_mode(sp.modemap, tt / N2)};
+    const u32 width[3] = {rec.wT, rec.wO, rec.wG};
+    const u32 th = modes[0], om = modes[1], gr = modes[2];
+    const bool on_shard = in_set(SET_UPDATE_ON_SHARD, om);
+    u32 a = 0, b = 0, c = 0, h = 0;
+#pragma unroll
+    for (int st = 0; st < 3; ++st) {
+      if (modes[st] == PS_MODE_R) a += width[st];
+      if (in_set(SET_SHARDLIKE, modes[st])) b += width[st];
+      if (in_set(SET_TRANSIENT, modes[st])) c += width[st];
+    }
+    // Theorem 2: all-reduce of replicated gradients, reduce-scatter of sharded
+    // ones, two all-gathers of gathered parameters
+    u32 ct = (th == PS_MODE_SG) ? 2 : 0, co = 0;
+    u32 cg = (gr == PS_MODE_R) ? 2 : (gr == PS_MODE_S ? 1 : 0);
+    if (ext_in_objective) {                  // traffic the theorem does not price
+      if (th == PS_MODE_O) ct += 2;
+      if (th == PS_MODE_R && on_shard) ct += 1;
+      if (om == PS_MODE_SG) co = 1;
+      if (gr == PS_MODE_SG) cg += 2;
+      if (gr == PS_MODE_M) cg += on_shard ? 1 : 2;
+      if (gr == PS_MODE_O) cg += 1;
+    }
+    if (th == PS_MODE_O) h += 3 * rec.wT;
+    if (om == PS_MODE_O) h += 2 * rec.wO;
+    if (gr == PS_MODE_O) h += 2 * rec.wG;
     t_local[r] = tt;
-    t_modes[r] = th | (om << 3) | (gr << 6) | (in_set(SET_UPDATE_ON_SHARD, om) ? 1u << 9 : 0);
+    ka[r] = a; kb[r] = b; kc[r] = c; kh[r] = h;
+    kx[r] = ct * rec.wT + co * rec.wO + cg * rec.wG;
     const u32 a_many = allowed_act_digits(triple_bits(th, om, gr, false), req, all, own, is_o, not_mo);
     const u32 a_one = allowed_act_digits(triple_bits(th, om, gr, true), req, all, all, is_o, not_mo);
     t_allowed[r] = live ? (a_many | (a_one << 8)) : 0;
@@ -387,29 +437,6 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
     const UnitBase ub = p2.all ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
                                : unit_base(rec, f, sp.tp_max_valid, true);
     __syncwarp();
-    if (lane < 5) {
-      const u32 pi = lane;
-      const u64 pe = mu_elems(pi, ub.E2, ub.sh, ub.u);
-      const u64 xT = ub.x * rec.wT, xO = ub.x * rec.wO, xG = ub.x * rec.wG;
-      // Theorem 2's terms, plus (if asked for) the traffic it does not price
-      u64 ct0 = (pi == PS_MODE_SG) ? 2 * xT : 0, ct1 = ct0, co = 0;
-      u64 cg0 = (pi == PS_MODE_R) ? 2 * xG : (pi == PS_MODE_S ? xG : 0), cg1 = cg0;
-      if (ext_in_objective) {
-        if (pi == PS_MODE_O) { ct0 += 2 * xT; ct1 += 2 * xT; }
-        if (pi == PS_MODE_R) ct1 += xT;                       // re-replicate updated shards
-        if (pi == PS_MODE_SG) { cg0 += 2 * xG; cg1 += 2 * xG; co = xO; }
-        if (pi == PS_MODE_M) { cg0 += 2 * xG; cg1 += xG; }
-        if (pi == PS_MODE_O) { cg0 += xG; cg1 += xG; }
-      }
-      const bool off = (pi == PS_MODE_O);
-      const u64 hT = off ? 3 * ub.sh * rec.wT : 0, hO = off ? 2 * ub.sh * rec.wO : 0,
-                hG = off ? 2 * ub.sh * rec.wG : 0;
-      tb.theta[0][pi] = ModeEntry{rec.wT * pe, ct0, hT, 0};
-      tb.theta[1][pi] = ModeEntry{rec.wT * pe, ct1, hT, 0};
-      tb.omega[pi] = ModeEntry{rec.wO * pe, co, hO, 0};
-      tb.grad[0][pi] = ModeEntry{rec.wG * pe, cg0, hG, 0};
-      tb.grad[1][pi] = ModeEntry{rec.wG * pe, cg1, hG, 0};
-    }
     {
       // lane (vt, d): activation bytes of digit d under variant vt, and the bound
       // a triple's own bytes must stay below for the sum to fit the capacity
@@ -419,8 +446,9 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
       const ActBase ab = p2.all ? act_base_pow2(rec, p2, v, tau) : act_base(rec, f, v, tau);
       const u64 am = mu_elems(digit_mode(sp.modemap, d), ab.EA, ab.shA, ab.uA);
       u64 axis = U64MAX;
+      if (!mine && vt < 4) { tb.bound[d][vt] = 0; if (d == 0) tb.host_bound[vt] = 0; }
       if (mine) {
-        tb.bound[vt][d] = am < cap_x ? cap_x - am : 0;
+        tb.bound[d][vt] = am < cap_x ? cap_x - am : 0;
         tb.act[vt][d] = am;
         if (d == 0) {
           const u64 ah = 2 * ab.EA;                            // offload after fwd, reload for bwd
@@ -443,12 +471,9 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
     u32 allowed[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      const u32 tm = t_modes[r];
-      const u32 th = tm & 7u, om = (tm >> 3) & 7u, gr = (tm >> 6) & 7u, rho = (tm >> 9) & 1u;
-      const ModeEntry et = tb.theta[rho][th], eo = tb.omega[om], eg = tb.grad[rho][gr];
-      mem3[r] = et.mem + eo.mem + eg.mem;
-      comm3[r] = et.comm + eo.comm + eg.comm;
-      host3[r] = et.host + eo.host + eg.host;
+      mem3[r] = mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0)));
+      comm3[r] = mad_small(ub.x, kx[r], 0);
+      host3[r] = host_limited ? mad_small(ub.sh, kh[r], 0) : 0;
       allowed[r] = (unit_ok && host3[r] < host_x) ? ((t_allowed[r] >> a_shift) & all) : 0;
     }
     const u32 unit_first = unit * per_unit;      // index of the unit's first point in the model
@@ -462,23 +487,29 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
     for (int r = 0; r < R; ++r) n_pass[r] = 0;
 #pragma unroll
     for (int d = 0; d < NM; ++d) {
-      bool allow[R];
+      u64 bound[4];
+      {
+        const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(&tb.bound[d][0]);
+        const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(&tb.bound[d][2]);
+        bound[0] = b01.x; bound[1] = b01.y; bound[2] = b23.x; bound[3] = b23.y;
+      }
+      if (host_limited && ((is_o >> d) & 1u)) {
+        // offloading activations also has to fit the host budget of the variant
 #pragma unroll
-      for (int r = 0; r < R; ++r) allow[r] = (allowed[r] >> d) & 1u;
-      const bool host_check = host_limited && ((is_o >> d) & 1u);
+        for (int r = 0; r < R; ++r) {
+          u32 c = 0;
 #pragma unroll
-      for (int vt = 0; vt < 4; ++vt) {
-        if ((u32)vt < nvt) {
-          const u64 bound = tb.bound[vt][d];
-          if (host_check) {
-            const u64 host_bound = tb.host_bound[vt];
+          for (int vt = 0; vt < 4; ++vt)
+            c += (mem3[r] < bound[vt] && host3[r] < tb.host_bound[vt]) ? 1u : 0u;
+          n_pass[r] += ((allowed[r] >> d) & 1u) ? c : 0u;
+        }
+      } else {
 #pragma unroll
-            for (int r = 0; r < R; ++r)
-              n_pass[r] += (allow[r] && mem3[r] < bound && host3[r] < host_bound) ? 1u : 0u;
-          } else {
+        for (int r = 0; r < R; ++r) {
+          u32 not_below = 0;               // variants whose bound the triple's bytes reach
 #pragma unroll
-            for (int r = 0; r < R; ++r) n_pass[r] += (allow[r] && mem3[r] < bound) ? 1u : 0u;
-          }
+          for (int vt = 0; vt < 4; ++vt) count_not_below(not_below, mem3[r], bound[vt]);
+          n_pass[r] += ((allowed[r] >> d) & 1u) ? 4u - not_below : 0u;
         }
       }
     }
@@ -518,7 +549,7 @@ __global__ void __launch_bounds__(THREADS, 3) k_sweep(SpaceDev sp, SweepArgs arg
       const u64 c_axis = tb.c_axis[vt], host_bound = tb.host_bound[vt];
       u64 bound[NM];
 #pragma unroll
-      for (int d = 0; d < NM; ++d) bound[d] = tb.bound[vt][d];
+      for (int d = 0; d < NM; ++d) bound[d] = tb.bound[d][vt];
       // every point of (triple, variant): digit d is a survivor if the triple's
       // bytes are below the digit's bound and the flags allow the digit
       u32 pass[R];
