@@ -41,7 +41,6 @@ struct WarpTables {
   u64 act[4][5];           // activation bytes of digit d
   u64 host_bound[4];       // a triple whose own host bytes are below this may offload activations
   u64 c_axis[4];           // tensor + pipeline traffic of the variant (0 if not in the objective)
-  u64 c_axis_least;        // the least of them
   // Pareto: for every set of digits the one with the least activation bytes
   // (lowest digit on ties), NM for the empty set
   unsigned char least[4][32];
@@ -427,7 +426,17 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
     const u32 a_many = allowed_act_digits(triple_bits(th, om, gr, false), req, all, own, is_o, not_mo);
     const u32 a_one = allowed_act_digits(triple_bits(th, om, gr, true), req, all, all, is_o, not_mo);
     t_allowed[r] = live ? (a_many | (a_one << 8)) : 0;
+    // keep the coefficients in registers instead of recomputing them for every unit
+    asm volatile("" : "+r"(ka[r]), "+r"(kb[r]), "+r"(kc[r]), "+r"(kx[r]), "+r"(kh[r]), "+r"(t_allowed[r]));
   }
+
+  // this lane's table entry (variant, digit), also fixed for the whole kernel
+  const u32 tl_vt = lane / NM, tl_d = lane - tl_vt * NM;
+  const bool tl_mine = tl_vt < nvt;
+  const u32 tl_v = tl_mine ? tl_vt / sp.nt : 0;
+  const u32 tl_tau = tl_mine ? tl_vt - tl_v * sp.nt : 0;
+  const u32 tl_mode = digit_mode(sp.modemap, tl_d);
+  const u64 tl_A = rec.A[tl_v], tl_UA = rec.UA[tl_v];
 
   // warps take the block's units in turn: the first one by warp number, then
   // whichever is next when they finish (their work differs with the candidates)
@@ -440,28 +449,30 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
     {
       // lane (vt, d): activation bytes of digit d under variant vt, and the bound
       // a triple's own bytes must stay below for the sum to fit the capacity
-      const u32 vt = lane / NM, d = lane - vt * NM;
-      const bool mine = vt < nvt;
-      const u32 v = mine ? vt / sp.nt : 0, tau = mine ? vt - v * sp.nt : 0;
-      const ActBase ab = p2.all ? act_base_pow2(rec, p2, v, tau) : act_base(rec, f, v, tau);
-      const u64 am = mu_elems(digit_mode(sp.modemap, d), ab.EA, ab.shA, ab.uA);
-      u64 axis = U64MAX;
-      if (!mine && vt < 4) { tb.bound[d][vt] = 0; if (d == 0) tb.host_bound[vt] = 0; }
-      if (mine) {
-        tb.bound[d][vt] = am < cap_x ? cap_x - am : 0;
-        tb.act[vt][d] = am;
-        if (d == 0) {
-          const u64 ah = 2 * ab.EA;                            // offload after fwd, reload for bwd
-          tb.host_bound[vt] = ah < host_x ? host_x - ah : 0;
-          axis = ext_in_objective ? model_axis_traffic(rec, f, ub, tau, sp.tp_coll) : 0;
-          tb.c_axis[vt] = axis;
-        }
+      ActBase ab;
+      if (p2.all) {
+        const u32 s = tl_tau == 0 ? p2.sT : 0;
+        ab.EA = ceil_shift(tl_A, s);
+        ab.uA = ceil_shift(tl_UA, s);
+        ab.shA = ceil_shift(ab.EA, p2.sD);
+      } else {
+        ab.EA = tl_tau == 0 ? div_ceil(tl_A, f.T) : tl_A;
+        ab.uA = tl_tau == 0 ? div_ceil(tl_UA, f.T) : tl_UA;
+        ab.shA = div_ceil(ab.EA, f.D);
       }
-      // least axis traffic over the variants (lanes 0, NM, 2 NM, 3 NM hold them)
-      u64 least_axis = axis;
-#pragma unroll
-      for (int o = 1; o < 4; ++o) least_axis = min(least_axis, __shfl_sync(0xffffffffu, axis, (o * NM) & 31));
-      if (lane == 0) tb.c_axis_least = least_axis;
+      const u64 am = mu_elems(tl_mode, ab.EA, ab.shA, ab.uA);
+      if (tl_mine) {
+        tb.bound[tl_d][tl_vt] = am < cap_x ? cap_x - am : 0;
+        tb.act[tl_vt][tl_d] = am;
+        if (tl_d == 0) {
+          const u64 ah = 2 * ab.EA;                            // offload after fwd, reload for bwd
+          tb.host_bound[tl_vt] = ah < host_x ? host_x - ah : 0;
+          tb.c_axis[tl_vt] = ext_in_objective ? model_axis_traffic(rec, f, ub, tl_tau, sp.tp_coll) : 0;
+        }
+      } else if (tl_vt < 4) {
+        tb.bound[tl_d][tl_vt] = 0;
+        if (tl_d == 0) tb.host_bound[tl_vt] = 0;
+      }
     }
     __syncwarp();
     // the lane's triples for this unit: own bytes, own communication, allowed digits
@@ -521,7 +532,7 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
       for (int r = 0; r < R; ++r) matters = matters || n_pass[r] != 0;
     } else {
       const u64 comm_limit = min(threshold.a, (u64)sh.block_comm_limit);
-      const u64 least_axis = tb.c_axis_least;
+      const u64 least_axis = tb.c_axis[0];   // tau = 0 sends the smaller boundary tensor; v does not matter
 #pragma unroll
       for (int r = 0; r < R; ++r) {
         survivors += n_pass[r];
