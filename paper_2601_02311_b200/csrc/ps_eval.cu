@@ -2,17 +2,21 @@
 // filter and compact the survivors in index order.
 //
 // A "group" is the n_codes consecutive points that share (model, factorisation,
-// activation variant, tensor-axis variant).  One warp owns one group: it
-// computes the group's shard quantities once, builds two pair tables in its
-// shared-memory slice -- (Theta, Omega) digits and (G, A) digits, each entry
-// holding the pair's mem / comm_paper / comm_ext / host contributions and flag
-// bits -- and then every point is two table reads, a few adds and the flag
-// logic.  Lanes take consecutive codes, so all output stores are coalesced.
+// activation variant, tensor-axis variant).  A warp owns a contiguous run of the
+// window's groups.  Within a group a lane owns up to four (Theta, Omega, G)
+// triples.  A triple's bytes, priced communication, unpriced communication and
+// host bytes are small-integer multiples of four per-group scalars (elements per
+// position E, largest shard s, reconstruction unit u, ring volume x), and the
+// integer coefficients depend only on the triple's modes and the model's byte
+// widths -- so they are computed once per model and a group costs a few
+// multiply-adds per triple.  The activation digit then adds one of NM
+// per-group values.  Codes of a group run digit-major, triple-minor, so for a
+// fixed digit the lanes write consecutive elements: all stores are coalesced.
 //
 // Compaction is count -> scan -> write: the count pass stores the survivors of
-// each warp's group, a single-block scan turns them into offsets, the write
-// pass evaluates again and places survivors with ballot/popc prefix sums.
-// Output order is the index order, so the result is unique.
+// each group, a single-block scan turns them into offsets, the write pass
+// evaluates again and places survivors with ballot/popc prefix sums.  Output
+// order is the index order, so the result is unique.
 #include "ps_device.cuh"
 #include "ps_internal.h"
 
@@ -21,247 +25,274 @@ namespace {
 constexpr int THREADS = EVAL_THREADS;
 constexpr int WARPS = THREADS / 32;
 
-// internal flag bits of the pair tables (above the public 13 bits)
+// internal bits of a triple's static description (above the public flag bits)
 enum : u32 {
-  X_ON_SHARD = 1u << 16,   // update committed on a shard (Omega in S, S*, O)
-  X_M_OR_O = 1u << 17,     // some state materialised or offloaded
-  X_G_FULL = 1u << 18,     // gradients delivered in full (G in R, S*, M)
-  X_G_IS_M = 1u << 19,
-  X_D1 = 1u << 20,
-  X_PUBLIC = 0x1FFFu
+  X_HOST3 = 1u << 16,     // one of Theta, Omega, G is offloaded
+  X_MO3 = 1u << 17,       // one of them is materialised or offloaded
+  X_EXT0 = 1u << 18       // the data axis moves nothing beyond Theorem 2's terms
 };
 
-struct __align__(16) PairEntry {
-  u64 mem, comm_paper, comm_ext, host;
-};
-
-struct WarpGroupTables {
-  PairEntry p1[25];   // index dth + nm*dom
-  PairEntry p2[25];   // index dgr + nm*dac
-  u32 f1[25];
-  u32 f2[25];
-};
-
-struct GroupConst {
-  u64 xG;        // ring bytes of G: added once more when G is materialised and the update is on the full range
-  u64 c_axis;    // tensor + pipeline traffic
-  u32 fbase;     // composition bits, X_D1
-  u64 lo, hi;    // window of this group's points, as offsets into the space
-  u64 group_first;
-};
-
-// build the tables of global group `g`; returns false if the group lies outside the window
-__device__ __forceinline__ bool build_group(const SpaceDev& sp, const EvalArgs& a, u64 g, int lane,
-                                            WarpGroupTables& tb, GroupConst& gc) {
-  const u64 gfirst = g * sp.n_codes;
-  gc.group_first = gfirst;
-  gc.lo = max(gfirst, a.first);
-  gc.hi = min(gfirst + sp.n_codes, a.first + a.count);
-  if (gc.lo >= gc.hi) return false;
-  const u64 groups_per_model = (u64)sp.n_facts * sp.nvt;
-  const u32 model = (u32)(g / groups_per_model);
-  const u32 gl = (u32)(g - (u64)model * groups_per_model);
-  const u32 unit = gl / sp.nvt, vt = gl - unit * sp.nvt;
-  const u32 v = vt / sp.nt, tau = vt - v * sp.nt;
-  // the model record: 96 bytes as six 16-byte loads through the read-only path
-  ModelRec rec;
-  {
-    const uint4* src = reinterpret_cast<const uint4*>(&sp.recs[model]);
-    uint4* dst = reinterpret_cast<uint4*>(&rec);
-#pragma unroll
-    for (int k = 0; k < 6; ++k) dst[k] = __ldg(src + k);
-  }
-  const Fact f = sp.facts[unit];
-  const UnitBase ub = unit_base(rec, f, sp.tp_max_valid, true);
-  const ActBase ab = act_base(rec, f, v, tau);
-  const u64 xT = ub.x * rec.wT, xO = ub.x * rec.wO, xG = ub.x * rec.wG;
-  gc.xG = xG;
-  gc.c_axis = model_axis_traffic(rec, f, ub, tau, sp.tp_coll);
-  gc.fbase = ub.cv | (ub.d1 ? X_D1 : 0);
-  const u32 nm2 = sp.nm * sp.nm;
-  __syncwarp();
-  if (lane < (int)nm2) {
-    const u32 d0 = lane % sp.nm, d1 = lane / sp.nm;
-    {  // (Theta, Omega)
-      const u32 th = digit_mode(sp.modemap, d0), om = digit_mode(sp.modemap, d1);
-      const bool on_shard = in_set(SET_UPDATE_ON_SHARD, om);
-      PairEntry e;
-      e.mem = rec.wT * mu_elems(th, ub.E2, ub.sh, ub.u) + rec.wO * mu_elems(om, ub.E2, ub.sh, ub.u);
-      e.comm_paper = (th == PS_MODE_SG) ? 2 * xT : 0;
-      e.comm_ext = (th == PS_MODE_O ? 2 * xT : 0) + ((th == PS_MODE_R && on_shard) ? xT : 0) +
-                   (om == PS_MODE_SG ? xO : 0);
-      e.host = (th == PS_MODE_O ? 3 * ub.sh * rec.wT : 0) + (om == PS_MODE_O ? 2 * ub.sh * rec.wO : 0);
-      const bool omega_full = (om == PS_MODE_R) || (ub.d1 && in_set(SET_SHARDLIKE, om));
-      const bool theta_avail = in_set(SET_THETA_ALWAYS, th) || (th == PS_MODE_S && ub.d1) ||
-                               (th == PS_MODE_M && omega_full);
-      u32 fl = (theta_avail ? PS_F_THETA_AVAIL : 0) | (om != PS_MODE_M ? PS_F_SC : 0) |
-               (on_shard ? X_ON_SHARD : 0);
-      if (th == PS_MODE_O || om == PS_MODE_O) fl |= PS_F_USES_HOST;
-      if (in_set(SET_M_OR_O, th) || in_set(SET_M_OR_O, om)) fl |= X_M_OR_O;
-      tb.p1[lane] = e;
-      tb.f1[lane] = fl;
-    }
-    {  // (G, A); comm_ext as if the update is committed on a shard
-      const u32 gr = digit_mode(sp.modemap, d0), ac = digit_mode(sp.modemap, d1);
-      PairEntry e;
-      e.mem = rec.wG * mu_elems(gr, ub.E2, ub.sh, ub.u) + mu_elems(ac, ab.EA, ab.shA, ab.uA);
-      e.comm_paper = (gr == PS_MODE_R) ? 2 * xG : (gr == PS_MODE_S ? xG : 0);
-      e.comm_ext = (gr == PS_MODE_SG ? 2 * xG : 0) + ((gr == PS_MODE_M || gr == PS_MODE_O) ? xG : 0);
-      e.host = (gr == PS_MODE_O ? 2 * ub.sh * rec.wG : 0) + (ac == PS_MODE_O ? 2 * ab.EA : 0);
-      u32 fl = (in_set(SET_GRAD_FULL, gr) ? X_G_FULL : 0) | (gr == PS_MODE_M ? X_G_IS_M : 0) |
-               ((ub.d1 || in_set(SET_ACT_OWN, ac)) ? PS_F_ACT_AVAIL : 0);
-      if (gr == PS_MODE_O || ac == PS_MODE_O) fl |= PS_F_USES_HOST;
-      if (in_set(SET_M_OR_O, gr) || in_set(SET_M_OR_O, ac)) fl |= X_M_OR_O;
-      tb.p2[lane] = e;
-      tb.f2[lane] = fl;
-    }
-  }
-  __syncwarp();
-  return true;
+__device__ __forceinline__ u64 mad_small(u64 a, u32 k, u64 acc) {
+  u64 r = (u64)(u32)a * (u64)k + acc;
+  r += (u64)((u32)(a >> 32) * k) << 32;
+  return r;
 }
 
-struct PointVals {
-  u64 mem, comm_paper, comm_ext, host;
-  u32 flags;
-};
-
-__device__ __forceinline__ PointVals eval_from_tables(const WarpGroupTables& tb, const GroupConst& gc,
-                                                      u32 i1, u32 i2) {
-  const PairEntry a = tb.p1[i1], b = tb.p2[i2];
-  const u32 x = tb.f1[i1] | tb.f2[i2] | gc.fbase;
-  PointVals o;
-  o.mem = a.mem + b.mem;
-  o.comm_paper = a.comm_paper + b.comm_paper;
-  o.host = a.host + b.host;
-  u64 ext = a.comm_ext + b.comm_ext;
-  if ((x & (X_G_IS_M | X_ON_SHARD)) == X_G_IS_M) ext += gc.xG;   // reduced per unit by all-reduce
-  u32 fl = x & X_PUBLIC;
-  if (x & (X_ON_SHARD | X_G_FULL | X_D1)) fl |= PS_F_GRAD_COVER;
-  constexpr u32 gi_needs = PS_F_THETA_AVAIL | PS_F_ACT_AVAIL | PS_F_GRAD_COVER;
-  if ((fl & gi_needs) == gi_needs) fl |= PS_F_GI;
-  if (ext == 0 && !(x & X_M_OR_O)) fl |= PS_F_PAPER_PRICED;
-  o.comm_ext = ext + gc.c_axis;
-  o.flags = fl;
-  return o;
+// static description of a triple for D > 1 (d1 = false) or D = 1
+__device__ __forceinline__ u32 triple_static(u32 th, u32 om, u32 gr, bool d1) {
+  const bool on_shard = in_set(SET_UPDATE_ON_SHARD, om);
+  const bool omega_full = (om == PS_MODE_R) || (d1 && in_set(SET_SHARDLIKE, om));
+  const bool theta_avail = in_set(SET_THETA_ALWAYS, th) || (th == PS_MODE_S && d1) ||
+                           (th == PS_MODE_M && omega_full);
+  const bool grad_cover = d1 || on_shard || in_set(SET_GRAD_FULL, gr);
+  const u32 seen = (1u << th) | (1u << om) | (1u << gr);
+  // with one replica nothing moves; otherwise the unpriced data-axis terms are
+  // non-zero exactly when their mode conditions hold (ring volume >= 1 element)
+  const bool ext0 = d1 || !((th == PS_MODE_O) || (th == PS_MODE_R && on_shard) ||
+                            in_set((1u << PS_MODE_SG) | SET_M_OR_O, gr) || om == PS_MODE_SG);
+  return (theta_avail ? PS_F_THETA_AVAIL : 0) | (grad_cover ? PS_F_GRAD_COVER : 0) |
+         (om != PS_MODE_M ? PS_F_SC : 0) | (((seen >> PS_MODE_O) & 1u) ? X_HOST3 : 0) |
+         ((seen & SET_M_OR_O) ? X_MO3 : 0) | (ext0 ? X_EXT0 : 0);
 }
-
-// walks the codes lane, lane+32, ... of a group's window, keeping the two
-// table indices incrementally
-struct CodeWalk {
-  u32 i1, i2, step_q, step_r, nm2;
-  __device__ __forceinline__ void init(u32 code, u32 nm2_) {
-    nm2 = nm2_;
-    i2 = code / nm2;
-    i1 = code - i2 * nm2;
-    step_q = 32 / nm2;
-    step_r = 32 - step_q * nm2;
-  }
-  __device__ __forceinline__ void next() {
-    i1 += step_r;
-    i2 += step_q;
-    if (i1 >= nm2) { i1 -= nm2; ++i2; }
-  }
-};
 
 enum { MODE_MATERIALISE = 0, MODE_COUNT = 1, MODE_WRITE = 2 };
 
-template <int MODE>
-__global__ void __launch_bounds__(THREADS) k_eval(SpaceDev sp, EvalArgs a) {
-  __shared__ WarpGroupTables tables[WARPS];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const u64 seg = (u64)blockIdx.x * WARPS + warp;      // which group of the window
-  const u64 g = a.first_group + seg;
-  WarpGroupTables& tb = tables[warp];
-  GroupConst gc;
-  const bool any = build_group(sp, a, g, lane, tb, gc);
-  if (!any) {
-    if (MODE == MODE_COUNT && lane == 0 && seg < a.n_tiles) a.tile_count[seg] = 0;
-    return;
+template <int MODE, int NM>
+__global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
+  constexpr int N2 = NM * NM, N3 = NM * NM * NM, NC = N3 * NM;
+  constexpr int R = (N3 + 31) / 32;
+  const int lane = threadIdx.x & 31;
+  const u32 warp_global = blockIdx.x * WARPS + (threadIdx.x >> 5);
+  const u32 n_warps = gridDim.x * WARPS;
+  const u32 per_warp = (a.n_tiles + n_warps - 1) / n_warps;
+  const u32 seg_begin = min(warp_global * per_warp, a.n_tiles);
+  const u32 seg_end = min(seg_begin + per_warp, a.n_tiles);
+  const u32 groups_per_model = sp.n_facts * sp.nvt;
+
+  // the lane's triples: modes never change
+  u32 th[R], om[R], gr[R];
+  bool live[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const u32 t = lane + 32 * r;
+    live[r] = t < (u32)N3;
+    const u32 tt = live[r] ? t : 0;
+    th[r] = digit_mode(sp.modemap, tt % NM);
+    om[r] = digit_mode(sp.modemap, (tt / NM) % NM);
+    gr[r] = digit_mode(sp.modemap, tt / N2);
   }
-  const u32 n_pts = (u32)(gc.hi - gc.lo);
-  const u32 code0 = (u32)(gc.lo - gc.group_first);
-  CodeWalk walk;
-  walk.init(code0 + lane, sp.nm * sp.nm);
-  const u64 out_base = gc.lo - a.first;                // output position of the group's first point
+  // classes of the activation digit (Theorem 3: a replica needs its own activations)
+  u32 own = 0, is_o = 0, not_mo = 0;
+#pragma unroll
+  for (int d = 0; d < NM; ++d) {
+    const u32 ac = digit_mode(sp.modemap, d);
+    if (in_set(SET_ACT_OWN, ac)) own |= 1u << d;
+    if (ac == PS_MODE_O) is_o |= 1u << d;
+    if (!in_set(SET_M_OR_O, ac)) not_mo |= 1u << d;
+  }
 
-  u32 n_kept = 0;                                      // survivors so far (warp-uniform)
-  u64 write_base = 0;
-  if (MODE == MODE_WRITE) write_base = a.tile_offset[seg];
+  // per model: widths and the coefficients that follow from them
+  u32 model_cur = 0xffffffffu;
+  ModelRec rec;
+  u32 ka[R], kb[R], kc[R], kp[R], ke[R], kh[R];   // bytes (E, s, u), priced / unpriced comm (x), host (s)
+  u32 st_many[R], st_one[R];                      // static description for D > 1 and D = 1
 
-  for (u32 k = 0; k < n_pts; k += 32, walk.next()) {
-    const bool live = k + lane < n_pts;
-    PointVals p;
-    if (live) p = eval_from_tables(tb, gc, walk.i1, walk.i2);
-    if (MODE == MODE_MATERIALISE) {
-      if (live) {
-        const u64 o = out_base + k + lane;
-        if (a.out.mem) a.out.mem[o] = p.mem;
-        if (a.out.comm_paper) a.out.comm_paper[o] = p.comm_paper;
-        if (a.out.comm_ext) a.out.comm_ext[o] = p.comm_ext;
-        if (a.out.host) a.out.host[o] = p.host;
-        if (a.out.flags) a.out.flags[o] = p.flags;
+  for (u32 seg = seg_begin; seg < seg_end; ++seg) {
+    const u64 g = a.first_group + seg;
+    const u32 model = (u32)(g / groups_per_model);
+    const u32 gl = (u32)(g - (u64)model * groups_per_model);
+    const u32 unit = gl / sp.nvt, vt = gl - unit * sp.nvt;
+    const u32 v = vt / sp.nt, tau = vt - v * sp.nt;
+    if (model != model_cur) {
+      model_cur = model;
+      const uint4* src = reinterpret_cast<const uint4*>(&sp.recs[model]);
+      uint4* dst = reinterpret_cast<uint4*>(&rec);
+#pragma unroll
+      for (int k = 0; k < 6; ++k) dst[k] = __ldg(src + k);   // the 96-byte record, 16 bytes at a time
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const u32 modes[3] = {th[r], om[r], gr[r]};
+        const u32 width[3] = {rec.wT, rec.wO, rec.wG};
+        const bool on_shard = in_set(SET_UPDATE_ON_SHARD, om[r]);
+        u32 ca = 0, cb = 0, cc = 0;
+#pragma unroll
+        for (int s = 0; s < 3; ++s) {        // Theorem 1: R holds E, S and S* a shard, S* and M a unit
+          if (modes[s] == PS_MODE_R) ca += width[s];
+          if (in_set(SET_SHARDLIKE, modes[s])) cb += width[s];
+          if (in_set(SET_TRANSIENT, modes[s])) cc += width[s];
+        }
+        ka[r] = ca; kb[r] = cb; kc[r] = cc;
+        // Theorem 2: all-reduce (2x) or reduce-scatter (1x) of G, two all-gathers of gathered Theta
+        kp[r] = (th[r] == PS_MODE_SG ? 2 * rec.wT : 0) +
+                (gr[r] == PS_MODE_R ? 2 * rec.wG : (gr[r] == PS_MODE_S ? rec.wG : 0));
+        // what the execution model moves beyond that
+        u32 e = 0;
+        if (th[r] == PS_MODE_O) e += 2 * rec.wT;
+        if (th[r] == PS_MODE_R && on_shard) e += rec.wT;
+        if (om[r] == PS_MODE_SG) e += rec.wO;
+        if (gr[r] == PS_MODE_SG) e += 2 * rec.wG;
+        if (gr[r] == PS_MODE_M) e += (on_shard ? 1 : 2) * rec.wG;
+        if (gr[r] == PS_MODE_O) e += rec.wG;
+        ke[r] = e;
+        kh[r] = (th[r] == PS_MODE_O ? 3 * rec.wT : 0) + (om[r] == PS_MODE_O ? 2 * rec.wO : 0) +
+                (gr[r] == PS_MODE_O ? 2 * rec.wG : 0);
+        st_many[r] = triple_static(th[r], om[r], gr[r], false);
+        st_one[r] = triple_static(th[r], om[r], gr[r], true);
       }
-    } else {
-      const bool pass = live && p.mem <= a.cap_bytes && p.host <= a.host_cap &&
-                        (p.flags & a.require_flags) == a.require_flags;
-      const u32 votes = __ballot_sync(0xffffffffu, pass);
-      if (MODE == MODE_WRITE && pass) {
-        const u64 o = write_base + n_kept + __popc(votes & ((1u << lane) - 1u));
-        if (a.idx_out) a.idx_out[o] = gc.lo + k + lane;
-        if (a.out.mem) a.out.mem[o] = p.mem;
-        if (a.out.comm_paper) a.out.comm_paper[o] = p.comm_paper;
-        if (a.out.comm_ext) a.out.comm_ext[o] = p.comm_ext;
-        if (a.out.host) a.out.host[o] = p.host;
-        if (a.out.flags) a.out.flags[o] = p.flags | PS_F_FEASIBLE;
-      }
-      n_kept += __popc(votes);
     }
+
+    // ---- per group: shard quantities (all divisions), activation bytes per digit
+    const Fact f = sp.facts[unit];
+    const Pow2 p2 = pow2_of(f);
+    const UnitBase ub = p2.all ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
+                               : unit_base(rec, f, sp.tp_max_valid, true);
+    const ActBase ab = p2.all ? act_base_pow2(rec, p2, v, tau) : act_base(rec, f, v, tau);
+    const u64 c_axis = model_axis_traffic(rec, f, ub, tau, sp.tp_coll);
+    u64 act[NM];
+#pragma unroll
+    for (int d = 0; d < NM; ++d) act[d] = mu_elems(digit_mode(sp.modemap, d), ab.EA, ab.shA, ab.uA);
+    const u64 act_host = 2 * ab.EA;
+    const u32 avail = ub.d1 ? ((1u << NM) - 1u) : own;     // digits with PS_F_ACT_AVAIL
+
+    u64 mem3[R], paper3[R], ext3[R], host3[R];
+    u32 st[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      mem3[r] = mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0)));
+      paper3[r] = mad_small(ub.x, kp[r], 0);
+      ext3[r] = mad_small(ub.x, ke[r], 0);
+      host3[r] = mad_small(ub.sh, kh[r], 0);
+      st[r] = ub.d1 ? st_one[r] : st_many[r];
+    }
+
+    // ---- the group's points inside the window
+    const u64 group_first = g * NC;
+    const u32 code_lo = a.first > group_first ? (u32)(a.first - group_first) : 0u;
+    const u64 window_end = a.first + a.count;
+    const u32 code_hi = window_end < group_first + NC ? (u32)(window_end - group_first) : (u32)NC;
+    const u64 out_base = group_first - a.first;          // (wraps when the group starts before the window; only used with code >= code_lo)
+
+    u32 n_kept = 0;
+    u64 write_base = 0;
+    if (MODE == MODE_WRITE) write_base = a.tile_offset[seg];
+
+#pragma unroll
+    for (int d = 0; d < NM; ++d) {
+      const bool d_avail = (avail >> d) & 1u, d_off = (is_o >> d) & 1u, d_notmo = (not_mo >> d) & 1u;
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const u32 code = lane + 32 * r + d * N3;
+        const bool inside = live[r] && code >= code_lo && code < code_hi;
+        const u64 mem = mem3[r] + act[d];
+        const u64 host = host3[r] + (d_off ? act_host : 0);
+        u32 fl = ub.cv | (st[r] & (PS_F_THETA_AVAIL | PS_F_GRAD_COVER | PS_F_SC));
+        constexpr u32 both = PS_F_THETA_AVAIL | PS_F_GRAD_COVER;
+        if (d_avail) fl |= PS_F_ACT_AVAIL | (((st[r] & both) == both) ? PS_F_GI : 0);
+        if (d_off || (st[r] & X_HOST3)) fl |= PS_F_USES_HOST;
+        if (d_notmo && (st[r] & (X_EXT0 | X_MO3)) == X_EXT0) fl |= PS_F_PAPER_PRICED;
+        if (MODE == MODE_MATERIALISE) {
+          if (inside) {
+            const u64 o = out_base + code;
+            if (a.out.mem) a.out.mem[o] = mem;
+            if (a.out.comm_paper) a.out.comm_paper[o] = paper3[r];
+            if (a.out.comm_ext) a.out.comm_ext[o] = ext3[r] + c_axis;
+            if (a.out.host) a.out.host[o] = host;
+            if (a.out.flags) a.out.flags[o] = fl;
+          }
+        } else {
+          const bool pass = inside && mem <= a.cap_bytes && host <= a.host_cap &&
+                            (fl & a.require_flags) == a.require_flags;
+          const u32 votes = __ballot_sync(0xffffffffu, pass);
+          if (MODE == MODE_WRITE && pass) {
+            const u64 o = write_base + n_kept + __popc(votes & ((1u << lane) - 1u));
+            if (a.idx_out) a.idx_out[o] = group_first + code;
+            if (a.out.mem) a.out.mem[o] = mem;
+            if (a.out.comm_paper) a.out.comm_paper[o] = paper3[r];
+            if (a.out.comm_ext) a.out.comm_ext[o] = ext3[r] + c_axis;
+            if (a.out.host) a.out.host[o] = host;
+            if (a.out.flags) a.out.flags[o] = fl | PS_F_FEASIBLE;
+          }
+          n_kept += __popc(votes);
+        }
+      }
+    }
+    if (MODE == MODE_COUNT && lane == 0) a.tile_count[seg] = n_kept;
   }
-  if (MODE == MODE_COUNT && lane == 0) a.tile_count[seg] = n_kept;
 }
 
-// exclusive prefix sum of the per-group survivor counts; one block
+// exclusive prefix sum of the per-group survivor counts; one block that walks
+// the counts in tiles of 4096 with coalesced loads, a shuffle scan per warp and
+// one shared-memory pass per tile
 __global__ void __launch_bounds__(1024) k_tile_scan(EvalArgs a) {
-  __shared__ u64 part[1024];
-  const int tid = threadIdx.x;
+  __shared__ u64 warp_sum[32];
+  __shared__ u64 carry;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const u32 n = a.n_tiles;
-  const u32 per = (n + 1023) / 1024;
-  const u32 lo = min((u32)tid * per, n), hi = min(lo + per, n);
-  u64 s = 0;
-  for (u32 i = lo; i < hi; ++i) s += a.tile_count[i];
-  part[tid] = s;
+  if (tid == 0) carry = 0;
   __syncthreads();
-  for (int off = 1; off < 1024; off <<= 1) {     // inclusive scan of the partial sums
-    u64 add = (tid >= off) ? part[tid - off] : 0;
+  for (u32 tile = 0; tile < n; tile += 4096) {
+    const u32 i0 = tile + 4 * tid;
+    u32 c[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) c[k] = (i0 + k < n) ? a.tile_count[i0 + k] : 0u;
+    const u64 mine = (u64)c[0] + c[1] + c[2] + c[3];
+    u64 incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const u64 up = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += up;
+    }
+    if (lane == 31) warp_sum[warp] = incl;
     __syncthreads();
-    part[tid] += add;
+    u64 before = carry;                          // everything before this warp
+    for (int w = 0; w < warp; ++w) before += warp_sum[w];
+    u64 run = before + incl - mine;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (i0 + k < n) a.tile_offset[i0 + k] = run;
+      run += c[k];
+    }
+    __syncthreads();
+    if (tid == 1023) carry = before + incl;
     __syncthreads();
   }
-  u64 run = part[tid] - s;
-  for (u32 i = lo; i < hi; ++i) {
-    a.tile_offset[i] = run;
-    run += a.tile_count[i];
+  if (tid == 0) *a.n_out = carry;
+}
+
+template <int MODE, int NM>
+cudaError_t launch_eval_t(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream) {
+  // one warp per run of groups; enough blocks to fill the GPU, no more than groups
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const unsigned needed = (a.n_tiles + WARPS - 1) / WARPS;
+  const unsigned blocks = needed < (unsigned)(sms * 16) ? needed : (unsigned)(sms * 16);
+  k_eval<MODE, NM><<<blocks, THREADS, 0, stream>>>(sp, a);
+  return cudaGetLastError();
+}
+
+template <int MODE>
+cudaError_t launch_eval_m(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream) {
+  switch (sp.nm) {
+    case 1: return launch_eval_t<MODE, 1>(sp, a, stream);
+    case 2: return launch_eval_t<MODE, 2>(sp, a, stream);
+    case 3: return launch_eval_t<MODE, 3>(sp, a, stream);
+    case 4: return launch_eval_t<MODE, 4>(sp, a, stream);
+    default: return launch_eval_t<MODE, 5>(sp, a, stream);
   }
-  if (tid == 1023) *a.n_out = part[1023];
 }
 
 }  // namespace
 
-static unsigned eval_blocks(const EvalArgs& a) { return (a.n_tiles + WARPS - 1) / WARPS; }
-
 cudaError_t launch_eval_materialise(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream) {
-  k_eval<MODE_MATERIALISE><<<eval_blocks(a), THREADS, 0, stream>>>(sp, a);
-  return cudaGetLastError();
+  return launch_eval_m<MODE_MATERIALISE>(sp, a, stream);
 }
 cudaError_t launch_eval_count(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream) {
-  k_eval<MODE_COUNT><<<eval_blocks(a), THREADS, 0, stream>>>(sp, a);
-  return cudaGetLastError();
+  return launch_eval_m<MODE_COUNT>(sp, a, stream);
 }
 cudaError_t launch_tile_scan(const EvalArgs& a, cudaStream_t stream) {
   k_tile_scan<<<1, 1024, 0, stream>>>(a);
   return cudaGetLastError();
 }
 cudaError_t launch_eval_write(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream) {
-  k_eval<MODE_WRITE><<<eval_blocks(a), THREADS, 0, stream>>>(sp, a);
-  return cudaGetLastError();
+  return launch_eval_m<MODE_WRITE>(sp, a, stream);
 }

@@ -283,15 +283,14 @@ __device__ __forceinline__ u64 mad_small(u64 a, u32 k, u64 acc) {
 // n += (m >= bound): a 64-bit subtraction whose borrow is folded into the
 // counter by one more subtract-with-borrow (n - (0xffffffff + borrow) = n + 1 - borrow)
 __device__ __forceinline__ void count_not_below(u32& n, u64 m, u64 bound) {
-  u32 scratch;
   asm("{\n\t"
-      "sub.cc.u32 %1, %2, %4;\n\t"
-      "subc.cc.u32 %1, %3, %5;\n\t"
+      ".reg .u32 diff;\n\t"
+      "sub.cc.u32 diff, %1, %3;\n\t"
+      "subc.cc.u32 diff, %2, %4;\n\t"
       "subc.u32 %0, %0, 0xffffffff;\n\t"
       "}"
-      : "+r"(n), "=r"(scratch)
+      : "+r"(n)
       : "r"((u32)m), "r"((u32)(m >> 32)), "r"((u32)bound), "r"((u32)(bound >> 32)));
-  (void)scratch;
 }
 
 // bits of a triple's static description
