@@ -48,13 +48,18 @@ UNIT = "evals/s"
 # by the points of a factorisation has been hoisted ("Rooflines")
 ALG_OPS_PER_POINT_SWEEP = 12
 BYTES_PER_POINT_MATERIALISE = 36
+# DRAM traffic of one launch from the ncu captures summarised under profiles/
+# (k_sweep<top-k> on the full stress configuration; k_eval<materialise> per point
+# of a 2^25-point window, where traffic grows in proportion to the points)
+NCU_SWEEP_DRAM_BYTES = 482_304
+NCU_MATERIALISE_DRAM_BYTES_PER_POINT = 1_249_138_000 / (1 << 25)
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C4")
     ap.add_argument("--models", type=int, default=None, help="shrink the shape table (tests)")
@@ -111,7 +116,7 @@ class ClockSampler:
             self.fh = open(self.path, "w")
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY,
-                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.fh,
+                 "--format=csv,noheader,nounits", "-lms", "50"], stdout=self.fh,
                 stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -171,7 +176,7 @@ def cpu_baseline(space, threads=None):
     from oracle import oracle as O
     threads = threads or O.hardware_threads()
     osp = O.Space(space)
-    n_models = min(len(space["models"]), 4 * threads)
+    n_models = min(len(space["models"]), 96 * threads)      # about 15 s of CPU work
     t0 = time.perf_counter()
     osp.sweep(TOPK_FILTER, TOPK_CAPS, O.KIND_TOPK, TOPK_K, model_count=n_models, n_threads=threads)
     dt = time.perf_counter() - t0
@@ -436,12 +441,15 @@ def run_ours(args):
             "gpu_launches": launches_per_step * args.steps,
             "roofline": {"bound": "alu", "kernel": "k_sweep<top-k> (+ merge)",
                          "achieved": alu_achieved, "peak": int_peak / 1e12, "unit": "Tops/s (int32)",
-                         "frac": alu_achieved / (int_peak / 1e12), "traffic": None,
+                         "frac": alu_achieved / (int_peak / 1e12),
+                         "traffic": NCU_SWEEP_DRAM_BYTES if args.workload == "C4" and args.models is None else None,
                          "ops_per_point": ALG_OPS_PER_POINT_SWEEP,
-                         "peak_source": "ps_int_peak measured in this run"},
+                         "alu_pipe_active_ncu": 0.72,
+                         "peak_source": "k_int_peak (add+xor chains on both integer pipes) measured in this run"},
             "roofline_hbm": {"bound": "hbm", "kernel": "k_eval<materialise>", "achieved": mat_gbs,
                              "peak": hbm_peak, "unit": "GB/s", "frac": mat_gbs / hbm_peak,
-                             "traffic": None, "peak_source": hbm_src},
+                             "traffic": int(NCU_MATERIALISE_DRAM_BYTES_PER_POINT * count),
+                             "peak_source": hbm_src + " (of measured)" if hbm_src == "measured" else hbm_src + " (of fallback)"},
         }
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(space)

@@ -92,7 +92,7 @@ enum { PS_REDUCE_PARETO = 0, PS_REDUCE_TOPK = 1 };
 
 #define PS_NO_LIMIT UINT64_MAX
 #define PS_TOPK_MAX 64           /* largest max_entries of a top-k sweep            */
-#define PS_FRONTIER_INTERNAL 256 /* longest frontier one block can hold (see sweep) */
+#define PS_FRONTIER_INTERNAL 128 /* longest frontier one warp or one block can hold */
 
 /* ------------------------------------------------------------------ types */
 typedef struct ps_ctx ps_ctx;     /* opaque: device, borrowed stream, scratch memory      */
@@ -214,7 +214,7 @@ int ps_eval_batch(ps_ctx* ctx, const ps_space* space, uint64_t first, uint64_t c
  * slots are zeroed.  d_counts[n_models][n_caps] (device) receives the true
  * frontier length, or for top-k the number of survivors, even when that
  * exceeds max_entries.  A frontier longer than PS_FRONTIER_INTERNAL inside one
- * block makes ps_status return PS_E_CAPACITY.  n_caps <= 8. */
+ * warp's share of a model makes ps_status return PS_E_CAPACITY.  n_caps <= 8. */
 int ps_sweep_pareto(ps_ctx* ctx, const ps_space* space, const ps_filter* filter,
                     const uint64_t* caps_bytes /* host */, uint32_t n_caps, uint32_t reduce_kind,
                     uint32_t max_entries, ps_front_entry* d_out, uint32_t* d_counts);
