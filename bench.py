@@ -220,6 +220,20 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------- ours
+def aggregate_over_ranks(dist, device, total_ms, e2e_ms, world, points_per_step, steps, e2e_steps):
+    """Whole-job figures: every rank processed `points_per_step` points per step
+    (weak scaling, no data-path collective); the job's time is the slowest rank's.
+    Returns (value, e2e_value, total_ms_max, e2e_ms_max)."""
+    import torch
+    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms_max, e2e_ms_max = float(t[0]), float(t[1])
+    value = points_per_step * steps * world / (total_ms_max * 1e-3)
+    e2e_value = points_per_step * e2e_steps * world / (e2e_ms_max * 1e-3)
+    return value, e2e_value, total_ms_max, e2e_ms_max
+
+
 def parity_gate(ps, gs, space, first):
     """Sampled outputs against the oracle, bit for bit."""
     from oracle import oracle as O
@@ -398,13 +412,8 @@ def run_ours(args):
     int_peak = ops / (e0.elapsed_time(e1) * 1e-3)
 
     # ---- aggregate over ranks: max time, summed points
-    t_total = torch.tensor([total_ms, e2e_s * 1e3], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t_total, op=dist.ReduceOp.MAX)
-    total_ms_max, e2e_ms_max = float(t_total[0]), float(t_total[1])
-    all_points = points_per_step * args.steps * world
-    value = all_points / (total_ms_max * 1e-3)
-    e2e_value = points_per_step * e2e_steps * world / (e2e_ms_max * 1e-3)
+    value, e2e_value, total_ms_max, e2e_ms_max = aggregate_over_ranks(
+        dist, dev, total_ms, e2e_s * 1e3, world, points_per_step, args.steps, e2e_steps)
 
     if rank == 0:
         peaks = {}
