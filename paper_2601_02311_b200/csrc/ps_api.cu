@@ -86,9 +86,10 @@ int enqueue_status_copy(ps_ctx* ctx) {
 }
 
 u32 pick_chunks(const ps_ctx* ctx, const ps_space* sp) {
-  // enough blocks for about six waves of three resident blocks per SM; every
-  // extra block of a model builds its lists from scratch, so no more than that
-  const u64 target = (u64)ctx->sm_count * 3 * 6;
+  // enough blocks for about three waves of two resident blocks per SM; every
+  // extra block of a model builds its lists from scratch and ends with a merge,
+  // so no more than that
+  const u64 target = (u64)ctx->sm_count * 2 * 3;
   u64 c = (target + sp->dev.n_models - 1) / sp->dev.n_models;
   if (c < 1) c = 1;
   if (c > SWEEP_MAX_CHUNKS) c = SWEEP_MAX_CHUNKS;

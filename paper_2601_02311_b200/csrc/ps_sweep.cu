@@ -698,31 +698,59 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
 
   // ---- block-level merge of the warps' lists
   for (int o = 16; o > 0; o >>= 1) survivors += __shfl_xor_sync(0xffffffffu, survivors, o);
-  if (lane == 0) { sh.warp_n[warp] = list.n; sh.warp_survivors[warp] = survivors; }
-  __syncthreads();
-  int total = 0, my_off = 0;
-  for (int w = 0; w < WARPS; ++w) {
-    if (w < warp) my_off += sh.warp_n[w];
-    total += sh.warp_n[w];
-  }
-  const int n_pad = next_pow2(max(total, 1));
-  for (int p = lane; p < list.n; p += 32) {
-    sh.merge_a[my_off + p] = list.a[p]; sh.merge_b[my_off + p] = list.b[p]; sh.merge_i[my_off + p] = list.i[p];
-  }
-  for (int p = total + tid; p < n_pad; p += THREADS) {
-    sh.merge_a[p] = U64MAX; sh.merge_b[p] = U64MAX; sh.merge_i[p] = 0xffffffffu;
-  }
-  __syncthreads();
-  block_sort(sh.merge_a, sh.merge_b, sh.merge_i, n_pad, tid, THREADS);
   int n_out;
-  if (KIND == PS_REDUCE_PARETO) {
+  if (KIND == PS_REDUCE_TOPK) {
+    // every warp sorts its own list and keeps its k smallest; an entry's place in
+    // the block's list is then its place at home plus, for every other warp, the
+    // number of that warp's entries below it (keys are distinct: binary searches,
+    // no block-wide sort)
+    if (list.n > 0) topk_compact(list, k_keep, lane, threshold, &sh.block_comm_limit);
+    if (lane == 0) { sh.warp_n[warp] = list.n; sh.warp_survivors[warp] = survivors; }
+    __syncthreads();
+    int total = 0;
+    for (int w = 0; w < WARPS; ++w) total += sh.warp_n[w];
+    for (int e = lane; e < list.n; e += 32) {
+      const Key key{list.a[e], list.b[e], list.i[e]};
+      int rank = e;
+      for (int w = 0; w < WARPS; ++w) {
+        if (w == warp) continue;
+        const u64* oa = sh.list_a + w * LIST_CAP;
+        const u64* ob = sh.list_b + w * LIST_CAP;
+        const u32* oi = sh.list_i + w * LIST_CAP;
+        int lo = 0, hi = sh.warp_n[w];
+        while (lo < hi) {
+          const int mid = (lo + hi) >> 1;
+          const Key other{oa[mid], ob[mid], oi[mid]};
+          if (key_less(other, key)) lo = mid + 1; else hi = mid;
+        }
+        rank += lo;
+      }
+      if (rank < k_keep) { sh.merge_a[rank] = key.a; sh.merge_b[rank] = key.b; sh.merge_i[rank] = key.i; }
+    }
+    __syncthreads();
+    n_out = min(total, k_keep);
+  } else {
+    if (lane == 0) { sh.warp_n[warp] = list.n; sh.warp_survivors[warp] = survivors; }
+    __syncthreads();
+    int total = 0, my_off = 0;
+    for (int w = 0; w < WARPS; ++w) {
+      if (w < warp) my_off += sh.warp_n[w];
+      total += sh.warp_n[w];
+    }
+    const int n_pad = next_pow2(max(total, 1));
+    for (int p = lane; p < list.n; p += 32) {
+      sh.merge_a[my_off + p] = list.a[p]; sh.merge_b[my_off + p] = list.b[p]; sh.merge_i[my_off + p] = list.i[p];
+    }
+    for (int p = total + tid; p < n_pad; p += THREADS) {
+      sh.merge_a[p] = U64MAX; sh.merge_b[p] = U64MAX; sh.merge_i[p] = 0xffffffffu;
+    }
+    __syncthreads();
+    block_sort(sh.merge_a, sh.merge_b, sh.merge_i, n_pad, tid, THREADS);
     n_out = block_pareto_prune(sh.merge_a, sh.merge_b, sh.merge_i, total, tid, THREADS, sh.smin, sh.scount);
     if (n_out > LIST_CAP) {
       if (tid == 0) atomicOr(args.status, ST_LIST_OVERFLOW);
       n_out = LIST_CAP;
     }
-  } else {
-    n_out = min(total, k_keep);
   }
   const u64 slot = (u64)model * n_chunks + chunk;
   PartialEntry* dst = args.partial + slot * LIST_CAP;
