@@ -411,6 +411,27 @@ def run_ours(args):
     torch.cuda.synchronize()
     int_peak = ops / (e0.elapsed_time(e1) * 1e-3)
 
+    # ---- Algorithm 1 batched (ps_select), measured beside the step, not inside it
+    n_sel = 1 << 24
+    sel_q = synth.select_queries(4096, 17)                                  # (4096, 8) u64 on the host
+    rec = np.zeros(4096, dtype=ps.SELECT_QUERY_DTYPE)                       # 32-byte records
+    rec["param_elems"], rec["layer_elems"], rec["device_bytes"] = sel_q[:, 0], sel_q[:, 1], sel_q[:, 2]
+    rec["n_devices"] = sel_q[:, 3]
+    rec["w_param"], rec["w_grad"], rec["w_opt"] = sel_q[:, 4], sel_q[:, 5], sel_q[:, 6]
+    rec["fast_interconnect"] = sel_q[:, 7]
+    d_sel_q = torch.from_numpy(rec.view(np.uint8).reshape(4096, 32).copy()).to(dev).repeat(n_sel // 4096, 1).contiguous()
+    d_sel_o = torch.empty(n_sel * 4, dtype=torch.int64, device=dev)
+    for _ in range(3):
+        ctx.select_into(d_sel_q, n_sel, d_sel_o)
+    torch.cuda.synchronize()
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0.record(stream)
+    for _ in range(10):
+        ctx.select_into(d_sel_q, n_sel, d_sel_o)
+    s1.record(stream)
+    torch.cuda.synchronize()
+    select_ms = s0.elapsed_time(s1) / 10
+
     # ---- aggregate over ranks: max time, summed points
     value, e2e_value, total_ms_max, e2e_ms_max = aggregate_over_ranks(
         dist, dev, total_ms, e2e_s * 1e3, world, points_per_step, args.steps, e2e_steps)
@@ -460,6 +481,9 @@ def run_ours(args):
                              "traffic": int(NCU_MATERIALISE_DRAM_BYTES_PER_POINT * count),
                              "peak_source": hbm_src + " (of measured)" if hbm_src == "measured" else hbm_src + " (of fallback)"},
         }
+        line["select"] = {"queries": n_sel, "ms": select_ms, "queries_per_s": n_sel / (select_ms * 1e-3),
+                          "GB/s": 64 * n_sel / (select_ms * 1e-3) / 1e9,
+                          "frac_of_hbm_peak": 64 * n_sel / (select_ms * 1e-3) / 1e9 / hbm_peak}
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(space)
         print(json.dumps(line), flush=True)

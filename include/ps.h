@@ -232,6 +232,43 @@ int ps_check_composition(ps_ctx* ctx, const ps_model_shape* shape /* host */, ui
                          uint32_t tp_max_valid, uint32_t tp_coll_per_layer, uint32_t comm_kind,
                          ps_front_entry* h_out);
 
+/* ------------------------------------------------------------------ Algorithm 1 */
+/* Batched form of the paper's illustrative strategy selection (Algorithm 1).
+ * For every query, with M_model = (w_param + w_grad + w_opt) * P bytes (line 1:
+ * "16P") and headroom = headroom_num / headroom_den (the paper's 0.7):
+ *   branch 0  M_model < headroom * M_d            -> (R,R,R,R), data parallel
+ *   branch 1  M_model / N < headroom * M_d        -> (S*,S,S,R), ZeRO-3 / FSDP
+ *   branch 2  otherwise, if one layer's model state (w sum * layer_elems) exceeds
+ *             layer_num / layer_den (0.3) of M_d and the interconnect is fast
+ *                                                  -> ZeRO-3 composed with tensor
+ *             parallelism of degree T = the largest divisor of N not above tp_degree
+ *   branch 3  otherwise                            -> ZeRO-3 alone (nothing of the
+ *             algorithm fits; the caller must look further)
+ * All comparisons are exact (integers, no rounding of the thresholds).  The
+ * result also carries Theorem 1's bytes and Theorem 2's volume of the chosen
+ * specification (activations excluded, as in the algorithm) and PS_F_FEASIBLE
+ * if those bytes fit M_d.  d_queries and d_out are device pointers (16-byte
+ * aligned), n may be 0.  Ranges as commented in the query; values outside give
+ * unspecified numbers but no fault. */
+typedef struct {
+  uint64_t param_elems;     /* P, 1 .. 2^46                                   */
+  uint64_t layer_elems;     /* elements of one layer (12 H^2, Def. 3), may be 0 */
+  uint64_t device_bytes;    /* M_d, <= 2^50                                    */
+  uint32_t n_devices;       /* N, 1 .. 2^24                                    */
+  uint8_t w_param, w_grad, w_opt; /* bytes per element, 1..16 (Remark 1: 2, 2, 12) */
+  uint8_t fast_interconnect;
+} ps_select_query;          /* 32 bytes */
+typedef struct {
+  uint64_t mem, comm;       /* Theorem 1, Theorem 2 for the chosen specification */
+  uint32_t branch;          /* 0..3 as above                                    */
+  uint32_t T;               /* tensor-parallel degree (1 unless branch 2)       */
+  uint32_t code_dp;         /* data-axis code: 0 (DP) or 32 (ZeRO-3)            */
+  uint32_t flags;           /* PS_F_FEASIBLE or 0                               */
+} ps_select_result;         /* 32 bytes */
+int ps_select(ps_ctx* ctx, const ps_select_query* d_queries, uint64_t n, uint32_t headroom_num,
+              uint32_t headroom_den, uint32_t layer_num, uint32_t layer_den, uint32_t tp_degree,
+              ps_select_result* d_out);
+
 /* The filter-and-compact form of ps_eval_batch for callers that cannot
  * allocate device memory.  (The paper has no counterpart: this is a property of
  * the library, not of the method.)

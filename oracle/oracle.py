@@ -190,5 +190,15 @@ def eval_record(rec: dict, N, T, K, D, v, tau, code, tp_max_valid=8, tp_coll_per
                 flags=int(out[4]))
 
 
+def select(queries: np.ndarray, headroom=(7, 10), layer=(3, 10), tp_degree=8) -> np.ndarray:
+    """Algorithm 1 on an (n, 8) uint64 array of queries (P, layer elements, device bytes, N,
+    w_param, w_grad, w_opt, fast); returns (n, 6): mem, comm, branch, T, code, flags."""
+    q = np.ascontiguousarray(queries, dtype=np.uint64)
+    out = np.zeros((len(q), 6), dtype=np.uint64)
+    lib().orc_select(_ptr(q), C.c_uint64(len(q)), headroom[0], headroom[1], layer[0], layer[1], tp_degree,
+                     _ptr(out))
+    return out
+
+
 def hardware_threads() -> int:
     return lib().orc_hardware_threads()

@@ -510,6 +510,42 @@ void orc_model_record(const OShape* shape, u64* rec) {
   rec[9] = m.w_theta; rec[10] = m.w_omega; rec[11] = m.w_grad; rec[12] = m.w_act;
 }
 
+// Algorithm 1 of the paper, one query at a time.  query: P, layer elements,
+// device bytes, N, w_param, w_grad, w_opt, fast (8 u64).  out: mem, comm,
+// branch, T, code, flags (6 u64).  Thresholds are the rationals hn/hd (0.7) and
+// ln/ld (0.3); comparisons are exact.
+void orc_select(const u64* query, u64 n, u32 hn, u32 hd, u32 ln, u32 ld, u32 tp_degree, u64* out) {
+  typedef unsigned __int128 u128;
+  for (u64 i = 0; i < n; ++i) {
+    const u64* q = query + 8 * i;
+    u64 P = q[0], layer = q[1], Md = q[2], N = q[3];
+    u64 wsum = q[4] + q[5] + q[6];
+    bool fast = q[7] != 0;
+    u128 m_model = (u128)wsum * P;                    // line 1: params + optimizer + gradients
+    u32 branch, T = 1, code;
+    if (m_model * hd < (u128)hn * Md) {               // fits one device with headroom: data parallel
+      branch = 0; code = 0;
+    } else if (m_model * hd < (u128)hn * Md * N) {    // fits when sharded N ways: ZeRO-3 / FSDP
+      branch = 1; code = 32;
+    } else if (fast && (u128)wsum * layer * ld > (u128)ln * Md) {   // a layer is too big: add TP
+      branch = 2; code = 32;
+      for (u64 t = std::min<u64>(tp_degree, N); t >= 1; --t)
+        if (N % t == 0) { T = (u32)t; break; }
+    } else {
+      branch = 3; code = 32;
+    }
+    ORecord m;
+    m.P = P; m.unit = layer; m.A[0] = m.A[1] = m.UA[0] = m.UA[1] = 0; m.Sbh = 1; m.L = 1; m.heads = T;
+    m.w_theta = (u32)q[4]; m.w_grad = (u32)q[5]; m.w_omega = (u32)q[6]; m.w_act = 1;
+    int pi[4]; u32 c = code;
+    for (int s = 0; s < 4; ++s) { pi[s] = c % 5; c /= 5; }
+    OResult r = eval_point(m, N, T, 1, N / T, 0, 0, pi[0], pi[1], pi[2], pi[3], 0xffffffffu, 0, true);
+    u64* o = out + 6 * i;
+    o[0] = r.mem; o[1] = r.comm_paper; o[2] = branch; o[3] = T; o[4] = code;
+    o[5] = r.mem <= Md ? F_FEASIBLE : 0;
+  }
+}
+
 u32 orc_hardware_threads() { return std::thread::hardware_concurrency(); }
 
 }  // extern "C"

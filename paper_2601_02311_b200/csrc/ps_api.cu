@@ -474,6 +474,24 @@ int ps_check_composition(ps_ctx* ctx, const ps_model_shape* shape, uint32_t N, u
   return PS_OK;
 }
 
+// ------------------------------------------------------------------ Algorithm 1
+int ps_select(ps_ctx* ctx, const ps_select_query* d_queries, uint64_t n, uint32_t headroom_num,
+              uint32_t headroom_den, uint32_t layer_num, uint32_t layer_den, uint32_t tp_degree,
+              ps_select_result* d_out) {
+  if (!ctx || (n && (!d_queries || !d_out))) return PS_E_NULLPTR;
+  if (!aligned(d_queries, 16) || !aligned(d_out, 16)) return PS_E_ALIGN;
+  if (headroom_den < 1 || layer_den < 1 || tp_degree < 1 || headroom_num > (1u << 16) ||
+      headroom_den > (1u << 16) || layer_num > (1u << 16) || layer_den > (1u << 16) ||
+      n > ((u64)1 << 38))
+    return PS_E_RANGE;
+  if (n == 0) return PS_OK;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return PS_E_CUDA;
+  CUDA_OK(launch_select(d_queries, n, headroom_num, headroom_den, layer_num, layer_den, tp_degree, d_out,
+                        ctx->stream));
+  return PS_OK;
+}
+
 // ------------------------------------------------------------------ measurement
 int ps_int_peak(ps_ctx* ctx, uint32_t blocks, uint32_t iters, uint32_t* d_sink, uint64_t* thread_ops) {
   if (!ctx || !d_sink || !thread_ops) return PS_E_NULLPTR;

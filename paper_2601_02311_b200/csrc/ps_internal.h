@@ -107,4 +107,6 @@ cudaError_t launch_model_derive(const ps_model_shape* d_shapes, ModelRec* d_recs
 cudaError_t launch_check_point(const ModelRec* d_rec, Fact f, u32 v, u32 tau, u32 code_dp,
                                u32 tp_max_valid, u32 tp_coll, u32 axis_form, u32 comm_kind,
                                u64 cap_bytes, ps_front_entry* d_out, cudaStream_t stream);
+cudaError_t launch_select(const ps_select_query* d_q, u64 n, u32 head_num, u32 head_den, u32 layer_num,
+                          u32 layer_den, u32 tp_degree, ps_select_result* d_out, cudaStream_t stream);
 cudaError_t launch_int_peak(u32 blocks, u32 iters, u32* d_sink, cudaStream_t stream);

@@ -77,6 +77,54 @@ __global__ void k_check_point(const ModelRec* rec, Fact f, u32 v, u32 tau, u32 c
   *out = e;
 }
 
+// Algorithm 1, one query per thread.  Thresholds are rationals; the comparisons
+// are carried out exactly in 128-bit integers.
+__global__ void __launch_bounds__(256) k_select(const ps_select_query* __restrict__ q, u64 n,
+                                                u32 head_num, u32 head_den, u32 layer_num,
+                                                u32 layer_den, u32 tp_degree,
+                                                ps_select_result* __restrict__ out) {
+  const u64 i = (u64)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  ps_select_query s;
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(q + i);
+    uint4* dst = reinterpret_cast<uint4*>(&s);
+    dst[0] = __ldg(src); dst[1] = __ldg(src + 1);
+  }
+  typedef unsigned __int128 u128;
+  const u32 wsum = (u32)s.w_param + s.w_grad + s.w_opt;
+  const u128 m_model = (u128)wsum * s.param_elems;
+  const u128 budget = (u128)head_num * s.device_bytes;        // headroom * M_d, times head_den
+  u32 branch, T = 1, code = 32;                                // ZeRO-3 unless data parallel fits
+  if (m_model * head_den < budget) {
+    branch = 0; code = 0;
+  } else if (m_model * head_den < budget * s.n_devices) {
+    branch = 1;
+  } else {
+    const u128 layer = (u128)wsum * s.layer_elems;
+    if (s.fast_interconnect && layer * layer_den > (u128)layer_num * s.device_bytes) {
+      branch = 2;
+      for (u32 t = min(tp_degree, s.n_devices); t >= 1; --t)
+        if (s.n_devices % t == 0) { T = t; break; }
+    } else {
+      branch = 3;
+    }
+  }
+  ModelRec r;
+  r.P = s.param_elems; r.unit = s.layer_elems; r.A[0] = r.A[1] = r.UA[0] = r.UA[1] = 0;
+  r.Sbh = 1; r.L = 1; r.heads = T;
+  r.wT = s.w_param; r.wO = s.w_opt; r.wG = s.w_grad; r.wA = 1; r.ok = 1;
+  const Fact f{s.n_devices, T, 1, s.n_devices / T};
+  const PointOut p = eval_point(r, f, 0, 0, code % 5, (code / 5) % 5, (code / 25) % 5, (code / 125) % 5,
+                                0xffffffffu, 0, true);
+  ps_select_result o;
+  o.mem = p.mem; o.comm = p.comm_paper; o.branch = branch; o.T = T; o.code_dp = code;
+  o.flags = p.mem <= s.device_bytes ? PS_F_FEASIBLE : 0;
+  uint4* dst = reinterpret_cast<uint4*>(out + i);
+  const uint4* src = reinterpret_cast<const uint4*>(&o);
+  dst[0] = src[0]; dst[1] = src[1];
+}
+
 // 8 independent chains per thread; each round applies to every chain an add
 // and an xor with loop-carried values the compiler cannot fold, so a round is
 // 16 independent-across-chains 32-bit operations and a chain's operations are
@@ -112,6 +160,13 @@ cudaError_t launch_check_point(const ModelRec* d_rec, Fact f, u32 v, u32 tau, u3
                                u64 cap_bytes, ps_front_entry* d_out, cudaStream_t stream) {
   k_check_point<<<1, 32, 0, stream>>>(d_rec, f, v, tau, code_dp, tp_max_valid, tp_coll, axis_form,
                                       comm_kind, cap_bytes, d_out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_select(const ps_select_query* d_q, u64 n, u32 head_num, u32 head_den, u32 layer_num,
+                          u32 layer_den, u32 tp_degree, ps_select_result* d_out, cudaStream_t stream) {
+  k_select<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(d_q, n, head_num, head_den, layer_num, layer_den,
+                                                             tp_degree, d_out);
   return cudaGetLastError();
 }
 

@@ -35,13 +35,18 @@ REDUCE_PARETO, REDUCE_TOPK = 0, 1
 NO_LIMIT = (1 << 64) - 1
 TOPK_MAX = 64
 
+SELECT_QUERY_DTYPE = np.dtype([("param_elems", "<u8"), ("layer_elems", "<u8"), ("device_bytes", "<u8"),
+                               ("n_devices", "<u4"), ("w_param", "u1"), ("w_grad", "u1"), ("w_opt", "u1"),
+                               ("fast_interconnect", "u1")])
+SELECT_RESULT_DTYPE = np.dtype([("mem", "<u8"), ("comm", "<u8"), ("branch", "<u4"), ("T", "<u4"),
+                                ("code_dp", "<u4"), ("flags", "<u4")])
 ENTRY_DTYPE = np.dtype([("mem", "<u8"), ("comm", "<u8"), ("host", "<u8"), ("idx", "<u8"),
                         ("flags", "<u4"), ("pad", "<u4")])
 
 EXPORTS = ("ps_create", "ps_destroy", "ps_status", "ps_strerror", "ps_space_create",
            "ps_space_destroy", "ps_space_set_models", "ps_space_rederive", "ps_space_size",
            "ps_space_points_per_model", "ps_space_decode", "ps_eval_batch", "ps_sweep_pareto",
-           "ps_check_composition", "ps_int_peak", "ps_eval_compact_noalloc")
+           "ps_check_composition", "ps_int_peak", "ps_eval_compact_noalloc", "ps_select")
 
 
 class _SpaceDesc(C.Structure):
@@ -94,6 +99,8 @@ _lib.ps_sweep_pareto.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(_Filter), C.c
 _lib.ps_check_composition.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32,
                                       C.c_uint32, C.c_uint16, C.c_uint16, C.c_uint16, C.c_uint32,
                                       C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p]
+_lib.ps_select.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32,
+                           C.c_uint32, C.c_uint32, C.c_void_p]
 _lib.ps_int_peak.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_void_p,
                              C.POINTER(C.c_uint64)]
 
@@ -162,6 +169,22 @@ class Context:
                                          tp_coll_per_layer, comm_kind, out.ctypes.data),
                "ps_check_composition")
         return {k: int(out[0][k]) for k in ("mem", "comm", "host", "flags")}
+
+    def select_into(self, d_queries: torch.Tensor, n: int, d_out: torch.Tensor, headroom=(7, 10),
+                    layer=(3, 10), tp_degree=8):
+        """ps_select on device buffers (uint8 tensors of 32-byte records)."""
+        _check(_lib.ps_select(self._h, _dptr(d_queries), n, headroom[0], headroom[1], layer[0], layer[1],
+                              tp_degree, _dptr(d_out)), "ps_select")
+
+    def select(self, queries: np.ndarray, headroom=(7, 10), layer=(3, 10), tp_degree=8) -> np.ndarray:
+        """Algorithm 1 for a structured array of SELECT_QUERY_DTYPE; returns SELECT_RESULT_DTYPE."""
+        q = np.ascontiguousarray(queries)
+        assert q.dtype.itemsize == 32
+        d_q = torch.from_numpy(q.view(np.uint8).reshape(-1).copy()).to(self.torch_device)
+        d_o = torch.empty(max(len(q), 1) * 32, dtype=torch.uint8, device=self.torch_device)
+        self.select_into(d_q, len(q), d_o, headroom, layer, tp_degree)
+        self.check_status()
+        return d_o.cpu().numpy()[:len(q) * 32].view(SELECT_RESULT_DTYPE)
 
     def int_peak(self, blocks: int, iters: int, sink: torch.Tensor) -> int:
         ops = C.c_uint64()

@@ -286,3 +286,25 @@ def test_argument_errors(ctx, ps):
         gs.sweep(dict(), [1], ps.REDUCE_TOPK, ps.TOPK_MAX + 1)
     assert e.value.code == ps.E_RANGE
     assert ctx.status() == ps.OK
+
+
+# ------------------------------------------------------------------ Algorithm 1
+def to_query_records(ps, q):
+    rec = np.zeros(len(q), dtype=ps.SELECT_QUERY_DTYPE)
+    rec["param_elems"], rec["layer_elems"], rec["device_bytes"] = q[:, 0], q[:, 1], q[:, 2]
+    rec["n_devices"] = q[:, 3]
+    rec["w_param"], rec["w_grad"], rec["w_opt"], rec["fast_interconnect"] = q[:, 4], q[:, 5], q[:, 6], q[:, 7]
+    return rec
+
+
+@pytest.mark.parametrize("n,tp_degree,headroom", [(100_003, 8, (7, 10)), (1, 4, (1, 2)), (0, 8, (7, 10)),
+                                                   (4097, 6, (9, 10))])
+def test_select_matches_oracle(ctx, ps, n, tp_degree, headroom):
+    q = synth.select_queries(n, seed=n + tp_degree)
+    got = ctx.select(to_query_records(ps, q), headroom=headroom, tp_degree=tp_degree)
+    want = O.select(q, headroom=headroom, tp_degree=tp_degree)
+    assert len(got) == n
+    for j, name in enumerate(("mem", "comm", "branch", "T", "code_dp", "flags")):
+        assert np.array_equal(got[name].astype(np.uint64), want[:, j]), name
+    if n > 1000:
+        assert set(np.unique(want[:, 2]).tolist()) == {0, 1, 2, 3}     # every branch is exercised

@@ -414,3 +414,44 @@ def test_generator_is_deterministic_and_in_range():
     assert (a["hidden"] % 128 == 0).all() and a["hidden"].max() <= 32768
     assert (a["heads"] * 128 == a["hidden"]).all()
     assert synth.table_checksum(a) != synth.table_checksum(synth.zoo(64, 3))
+
+
+# ------------------------------------------------------------ Algorithm 1
+def _q(P, layer, Md, N, fast=1):
+    return [P, layer, Md, N, 2, 2, 12, fast]
+
+
+def test_algorithm1_on_the_papers_example():
+    """Section 1 / Example 3: a 70B model needs 1120 GB, far more than an 80 GB GPU;
+    ZeRO-3 needs 16P/N.  With the 0.7 headroom of Algorithm 1: not data parallel;
+    ZeRO-3 once 1120/N < 56 GB, i.e. from N = 32 (35 GB); below that the last branch."""
+    P, Md = 70_000_000_000, 80 * synth.GB
+    layer = 12 * 8192 * 8192
+    r = O.select(np.array([_q(P, layer, Md, N) for N in (1, 8, 16, 32, 64)], dtype=np.uint64))
+    assert r[:, 2].tolist() == [3, 3, 3, 1, 1]          # layer state 12.9 GB < 0.3 * 80 GB: no TP
+    assert r[3, 0] == 16 * P // 32 + layer * 2            # Theorem 1: 16P/N plus the gathered unit
+    assert r[4, 4] == 32 and r[4, 3] == 1
+    # a 1B model fits one device with headroom: data parallel, 16 P bytes, all-reduce of 2P
+    r = O.select(np.array([_q(10 ** 9, 0, Md, 8)], dtype=np.uint64))
+    assert r[0].tolist()[:5] == [16 * 10 ** 9, 2 * (10 ** 9 - 10 ** 9 // 8) * 2, 0, 1, 0]
+    assert r[0, 5] == O.F_FEASIBLE
+
+
+def test_algorithm1_thresholds_are_strict_and_exact():
+    Md = 10 ** 10
+    # M_model = 16 P; boundary 16 P = 0.7 M_d  <=>  P = 437 500 000
+    r = O.select(np.array([_q(437_499_999, 0, Md, 4), _q(437_500_000, 0, Md, 4)], dtype=np.uint64))
+    assert r[:, 2].tolist() == [0, 1]
+    # ZeRO-3 boundary 16 P / N = 0.7 M_d at N = 4  <=>  P = 1 750 000 000
+    r = O.select(np.array([_q(1_749_999_999, 0, Md, 4), _q(1_750_000_000, 0, Md, 4)], dtype=np.uint64))
+    assert r[:, 2].tolist() == [1, 3]
+    # layer boundary 16 * layer > 0.3 M_d  <=>  layer > 187 500 000; needs a fast interconnect
+    big = 10 ** 12
+    r = O.select(np.array([_q(big, 187_500_000, Md, 8), _q(big, 187_500_001, Md, 8),
+                           _q(big, 187_500_001, Md, 8, fast=0), _q(big, 187_500_001, Md, 12)],
+                          dtype=np.uint64))
+    assert r[:, 2].tolist() == [3, 2, 3, 2]
+    assert r[1, 3] == 8 and r[3, 3] == 6                  # largest divisor of N not above 8
+    # tensor parallelism divides the state before the data axis shards it (Remark 4)
+    E2 = -(-big // 8)
+    assert r[1, 0] == 16 * E2 + 2 * (-(-187_500_001 // 8))
