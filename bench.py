@@ -45,7 +45,11 @@ VALID = 1 | 2 | 4
 METRIC = "placement evaluations/sec (bit-exact vs oracle)"
 UNIT = "evals/s"
 # integer operations the method needs per point once everything that is shared
-# by the points of a factorisation has been hoisted ("Rooflines")
+# by the points of a factorisation has been hoisted: a 64-bit compare against a
+# shifted bound or the equivalent add (2), the capacity compare (2), the
+# required-flags bit (1), the host-budget check of the offload digit (~1), the
+# reduction test (3), the survivor count (1) and the amortised per-triple set-up
+# (~1.5), rounded up
 ALG_OPS_PER_POINT_SWEEP = 12
 BYTES_PER_POINT_MATERIALISE = 36
 # DRAM traffic of one launch from the ncu captures summarised under profiles/

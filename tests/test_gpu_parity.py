@@ -308,3 +308,50 @@ def test_select_matches_oracle(ctx, ps, n, tp_degree, headroom):
         assert np.array_equal(got[name].astype(np.uint64), want[:, j]), name
     if n > 1000:
         assert set(np.unique(want[:, 2]).tolist()) == {0, 1, 2, 3}     # every branch is exercised
+
+
+# ------------------------------------------------------------------ extremes
+def extreme_space():
+    """Shapes at the edges of the supported ranges (2^46 parameters, 16-byte
+    widths, the largest boundary tensor, the largest stored activations) and
+    device counts up to 2^24 with non-trivial T and K."""
+    m = synth.zoo(4, 99)
+    m["param_elems_override"][0] = 1 << 46
+    m["w_param"][0], m["w_grad"][0], m["w_opt"][0], m["w_act"][0] = 16, 16, 16, 16
+    m["layers"][1], m["hidden"][1], m["heads"][1] = 1024, 1 << 16, 1 << 16
+    m["param_elems_override"][1] = (1 << 46) - 12345
+    m["seq"][1], m["micro_batch"][1], m["vocab"][1] = 1 << 10, 1 << 4, 1 << 24      # S b H = 2^30
+    m["seq"][2], m["micro_batch"][2], m["hidden"][2], m["heads"][2] = 1 << 17, 8, 1 << 16, 1 << 13
+    m["layers"][2] = 32                                     # stored activations 2^57.3 bytes, S b H = 2^36
+    m["layers"][3], m["hidden"][3], m["heads"][3], m["vocab"][3] = 1, 1, 1, 1
+    m["seq"][3], m["micro_batch"][3] = 1, 1
+    return dict(models=m, n_values=np.asarray([1, 1 << 24, 3 * (1 << 20), 16777213], dtype=np.uint32),
+                t_enum_max=64, k_enum_max=1 << 24, tp_max_valid=8, n_act_variants=2, n_tpa_variants=2,
+                mode_mask=0x1F, tp_coll_per_layer=64)
+
+
+def test_extreme_shapes_and_device_counts(ctx, ps):
+    space = extreme_space()
+    gs, os_ = both(ctx, space)
+    n = gs.size
+    assert n == os_.size and n < 6_000_000
+    got, want = gs.eval_batch(0, n), os_.eval_range(0, n)
+    assert_same_arrays(got, want, "extreme")
+    assert int(want["mem"].max()) < 1 << 62 and int((want["comm_paper"] + want["comm_ext"]).max()) < 1 << 63
+    filt = dict(require_flags=O.F_GI | O.F_SC, host_cap=1 << 40)
+    caps = [1 << 30, 1 << 45]
+    assert_same_sweep(gs.sweep(filt, caps, ps.REDUCE_PARETO, 128), os_.sweep(filt, caps, O.KIND_PARETO, 128, n_threads=4))
+    assert_same_sweep(gs.sweep(filt, caps, ps.REDUCE_TOPK, 64), os_.sweep(filt, caps, O.KIND_TOPK, 64, n_threads=4))
+
+
+def test_smallest_possible_space(ctx, ps):
+    """One model, one device, one mode, no variants: a single point."""
+    m = synth.zoo(1, 1)
+    space = dict(models=m, n_values=np.asarray([1], dtype=np.uint32), t_enum_max=1, k_enum_max=1,
+                 tp_max_valid=8, n_act_variants=1, n_tpa_variants=1, mode_mask=0b00001, tp_coll_per_layer=4)
+    gs, os_ = both(ctx, space)
+    assert gs.size == os_.size == 1
+    assert_same_arrays(gs.eval_batch(0, 1), os_.eval_range(0, 1))
+    filt = dict(require_flags=VALID)
+    for kind_g, kind_o in ((ps.REDUCE_PARETO, O.KIND_PARETO), (ps.REDUCE_TOPK, O.KIND_TOPK)):
+        assert_same_sweep(gs.sweep(filt, [O.NO_LIMIT], kind_g, 4), os_.sweep(filt, [O.NO_LIMIT], kind_o, 4))
