@@ -38,6 +38,8 @@ struct WarpTables {
   // a triple whose own bytes are below bound[d][vt] fits the capacity with digit d
   // under variant vt (0 for variants the space does not have)
   __align__(16) u64 bound[5][4];
+  // the same bounds as doubles, exact while they are below 2^53 (see the evaluation pass)
+  __align__(16) double bound_f64[5][4];
   u64 act[4][5];           // activation bytes of digit d
   u64 host_bound[4];       // a triple whose own host bytes are below this may offload activations
   u64 c_axis[4];           // tensor + pipeline traffic of the variant (0 if not in the objective)
@@ -293,6 +295,10 @@ __device__ __forceinline__ void count_not_below(u32& n, u64 m, u64 bound) {
       : "r"((u32)m), "r"((u32)(m >> 32)), "r"((u32)bound), "r"((u32)(bound >> 32)));
 }
 
+// digits whose capacity compares run on the fp64 pipe when the unit's numbers are
+// exact there; the other digits use the carry chain, so both pipes work
+constexpr u32 F64_DIGITS = 0x1f;
+
 // bits of a triple's static description
 enum : u32 {
   T_THETA_AVAIL = 1u << 0, T_GRAD_COVER = 1u << 1, T_SC = 1u << 2, T_HOST = 1u << 3,
@@ -461,7 +467,9 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
       }
       const u64 am = mu_elems(tl_mode, ab.EA, ab.shA, ab.uA);
       if (tl_mine) {
-        tb.bound[tl_d][tl_vt] = am < cap_x ? cap_x - am : 0;
+        const u64 bound = am < cap_x ? cap_x - am : 0;
+        tb.bound[tl_d][tl_vt] = bound;
+        tb.bound_f64[tl_d][tl_vt] = (double)bound;
         tb.act[tl_vt][tl_d] = am;
         if (tl_d == 0) {
           const u64 ah = 2 * ab.EA;                            // offload after fwd, reload for bwd
@@ -470,6 +478,7 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
         }
       } else if (tl_vt < 4) {
         tb.bound[tl_d][tl_vt] = 0;
+        tb.bound_f64[tl_d][tl_vt] = 0.0;
         if (tl_d == 0) tb.host_bound[tl_vt] = 0;
       }
     }
@@ -495,6 +504,56 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
     u32 n_pass[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) n_pass[r] = 0;
+    // Integers below 2^53 are exact in fp64, so when every quantity of the unit is
+    // that small (uniform test) the compares run on the fp64 pipe, which is idle
+    // otherwise, and only the counting stays on the integer pipe.
+    const bool small = cap_x < ((u64)1 << 53) &&
+                       (u64)(rec.wT + rec.wO + rec.wG) * (ub.E2 + ub.u) < ((u64)1 << 53);
+    if (small) {
+      double mem_f64[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) mem_f64[r] = (double)mem3[r];
+#pragma unroll
+      for (int d = 0; d < NM; ++d) {
+        const bool host_check = host_limited && ((is_o >> d) & 1u);
+        if (((F64_DIGITS >> d) & 1u) || host_check) {
+          double bound[4];
+          {
+            const double2 b01 = *reinterpret_cast<const double2*>(&tb.bound_f64[d][0]);
+            const double2 b23 = *reinterpret_cast<const double2*>(&tb.bound_f64[d][2]);
+            bound[0] = b01.x; bound[1] = b01.y; bound[2] = b23.x; bound[3] = b23.y;
+          }
+#pragma unroll
+          for (int r = 0; r < R; ++r) {
+            u32 c = 0;
+            if (host_check) {
+              // offloading activations also has to fit the host budget of the variant
+#pragma unroll
+              for (int vt = 0; vt < 4; ++vt)
+                c += (mem_f64[r] < bound[vt] && host3[r] < tb.host_bound[vt]) ? 1u : 0u;
+            } else {
+#pragma unroll
+              for (int vt = 0; vt < 4; ++vt) c += (mem_f64[r] < bound[vt]) ? 1u : 0u;
+            }
+            n_pass[r] += ((allowed[r] >> d) & 1u) ? c : 0u;
+          }
+        } else {
+          u64 bound[4];
+          {
+            const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(&tb.bound[d][0]);
+            const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(&tb.bound[d][2]);
+            bound[0] = b01.x; bound[1] = b01.y; bound[2] = b23.x; bound[3] = b23.y;
+          }
+#pragma unroll
+          for (int r = 0; r < R; ++r) {
+            u32 not_below = 0;
+#pragma unroll
+            for (int vt = 0; vt < 4; ++vt) count_not_below(not_below, mem3[r], bound[vt]);
+            n_pass[r] += ((allowed[r] >> d) & 1u) ? 4u - not_below : 0u;
+          }
+        }
+      }
+    } else {
 #pragma unroll
     for (int d = 0; d < NM; ++d) {
       u64 bound[4];
@@ -524,6 +583,7 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
       }
     }
 
+    }
     // ---- reduction pass, only if some survivor of this warp can matter
     bool matters = false;
     if (KIND == PS_REDUCE_PARETO) {
