@@ -176,28 +176,49 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
     u64 write_base = 0;
     if (MODE == MODE_WRITE) write_base = a.tile_offset[seg];
 
+    // flags of a point = what the triple fixes | what the digit fixes | what needs both:
+    //   gradient integrity needs the triple's two availability bits and the digit's,
+    //   "paper priced" needs a triple without M/O and unpriced traffic and a digit without M/O
+    u32 fl_base[R], fl_gi[R], fl_priced[R];
+    constexpr u32 both = PS_F_THETA_AVAIL | PS_F_GRAD_COVER;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      fl_base[r] = ub.cv | (st[r] & (both | PS_F_SC)) | ((st[r] & X_HOST3) ? PS_F_USES_HOST : 0);
+      fl_gi[r] = ((st[r] & both) == both) ? PS_F_GI : 0;
+      fl_priced[r] = ((st[r] & (X_EXT0 | X_MO3)) == X_EXT0) ? PS_F_PAPER_PRICED : 0;
+    }
+    const bool whole = code_lo == 0 && code_hi == (u32)NC;      // the window covers the group
+    const bool all_out = a.out.mem && a.out.comm_paper && a.out.comm_ext && a.out.host && a.out.flags;
+
 #pragma unroll
     for (int d = 0; d < NM; ++d) {
       const bool d_avail = (avail >> d) & 1u, d_off = (is_o >> d) & 1u, d_notmo = (not_mo >> d) & 1u;
+      const u32 fl_digit = (d_avail ? PS_F_ACT_AVAIL : 0) | (d_off ? PS_F_USES_HOST : 0);
+      const u32 gi_mask = d_avail ? ~0u : 0u, priced_mask = d_notmo ? ~0u : 0u;
+      const u64 host_add = d_off ? act_host : 0;
 #pragma unroll
       for (int r = 0; r < R; ++r) {
         const u32 code = lane + 32 * r + d * N3;
-        const bool inside = live[r] && code >= code_lo && code < code_hi;
+        const bool inside = live[r] && (whole || (code >= code_lo && code < code_hi));
         const u64 mem = mem3[r] + act[d];
-        const u64 host = host3[r] + (d_off ? act_host : 0);
-        u32 fl = ub.cv | (st[r] & (PS_F_THETA_AVAIL | PS_F_GRAD_COVER | PS_F_SC));
-        constexpr u32 both = PS_F_THETA_AVAIL | PS_F_GRAD_COVER;
-        if (d_avail) fl |= PS_F_ACT_AVAIL | (((st[r] & both) == both) ? PS_F_GI : 0);
-        if (d_off || (st[r] & X_HOST3)) fl |= PS_F_USES_HOST;
-        if (d_notmo && (st[r] & (X_EXT0 | X_MO3)) == X_EXT0) fl |= PS_F_PAPER_PRICED;
+        const u64 host = host3[r] + host_add;
+        const u32 fl = fl_base[r] | fl_digit | (fl_gi[r] & gi_mask) | (fl_priced[r] & priced_mask);
         if (MODE == MODE_MATERIALISE) {
           if (inside) {
             const u64 o = out_base + code;
-            if (a.out.mem) a.out.mem[o] = mem;
-            if (a.out.comm_paper) a.out.comm_paper[o] = paper3[r];
-            if (a.out.comm_ext) a.out.comm_ext[o] = ext3[r] + c_axis;
-            if (a.out.host) a.out.host[o] = host;
-            if (a.out.flags) a.out.flags[o] = fl;
+            if (all_out) {
+              a.out.mem[o] = mem;
+              a.out.comm_paper[o] = paper3[r];
+              a.out.comm_ext[o] = ext3[r] + c_axis;
+              a.out.host[o] = host;
+              a.out.flags[o] = fl;
+            } else {
+              if (a.out.mem) a.out.mem[o] = mem;
+              if (a.out.comm_paper) a.out.comm_paper[o] = paper3[r];
+              if (a.out.comm_ext) a.out.comm_ext[o] = ext3[r] + c_axis;
+              if (a.out.host) a.out.host[o] = host;
+              if (a.out.flags) a.out.flags[o] = fl;
+            }
           }
         } else {
           const bool pass = inside && mem <= a.cap_bytes && host <= a.host_cap &&
