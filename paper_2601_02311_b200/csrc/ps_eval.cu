@@ -57,10 +57,39 @@ __device__ __forceinline__ u32 triple_static(u32 th, u32 om, u32 gr, bool d1) {
 
 enum { MODE_MATERIALISE = 0, MODE_COUNT = 1, MODE_WRITE = 2 };
 
+// Copy n staged elements of a warp to global memory: scalar stores up to the
+// next 128-byte line, then 16-byte stores (one warp instruction = 512
+// contiguous, line-aligned bytes), then the remainder.  Fewer and fuller
+// requests to the memory system than 8-byte stores at arbitrary offsets.
+template <typename T>
+__device__ __forceinline__ void warp_copy_out(T* __restrict__ dst, const T* buf, int n, int lane) {
+  constexpr int PER16 = 16 / (int)sizeof(T);
+  const uintptr_t addr = reinterpret_cast<uintptr_t>(dst);
+  int head = (int)(((128 - (addr & 127)) & 127) / sizeof(T));
+  head = min(head, n);
+  for (int i = lane; i < head; i += 32) dst[i] = buf[i];
+  const int body = (n - head) / PER16;
+  for (int k = lane; k < body; k += 32) {
+    const T* src = buf + head + k * PER16;
+    uint4 v;
+    if (sizeof(T) == 8) {
+      const u64 x = (u64)src[0], y = (u64)src[1];
+      v = make_uint4((u32)x, (u32)(x >> 32), (u32)y, (u32)(y >> 32));
+    } else {
+      v = make_uint4((u32)src[0], (u32)src[1], (u32)src[2], (u32)src[3]);
+    }
+    *reinterpret_cast<uint4*>(dst + head + k * PER16) = v;
+  }
+  for (int i = head + body * PER16 + lane; i < n; i += 32) dst[i] = buf[i];
+}
+
 template <int MODE, int NM>
 __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
   constexpr int N2 = NM * NM, N3 = NM * NM * NM, NC = N3 * NM;
   constexpr int R = (N3 + 31) / 32;
+  // materialise: one group's values of one output array, staged per warp
+  __shared__ __align__(16) u64 stage_all[MODE == MODE_MATERIALISE ? WARPS * NC : 1];
+  u64* stage = stage_all + (MODE == MODE_MATERIALISE ? (threadIdx.x >> 5) * NC : 0);
   const int lane = threadIdx.x & 31;
   const u32 warp_global = blockIdx.x * WARPS + (threadIdx.x >> 5);
   const u32 n_warps = gridDim.x * WARPS;
@@ -189,6 +218,40 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
     }
     const bool whole = code_lo == 0 && code_hi == (u32)NC;      // the window covers the group
     const bool all_out = a.out.mem && a.out.comm_paper && a.out.comm_ext && a.out.host && a.out.flags;
+
+    if (MODE == MODE_MATERIALISE && whole && all_out) {
+      // one output array at a time: stage the group's NC values, copy them out
+      // with line-aligned 16-byte stores
+#pragma unroll
+      for (int which = 0; which < 5; ++which) {
+        u32* stage32 = reinterpret_cast<u32*>(stage);
+#pragma unroll
+        for (int d = 0; d < NM; ++d) {
+          const bool d_avail = (avail >> d) & 1u, d_off = (is_o >> d) & 1u, d_notmo = (not_mo >> d) & 1u;
+          const u32 fl_digit = (d_avail ? PS_F_ACT_AVAIL : 0) | (d_off ? PS_F_USES_HOST : 0);
+          const u32 gi_mask = d_avail ? ~0u : 0u, priced_mask = d_notmo ? ~0u : 0u;
+          const u64 host_add = d_off ? act_host : 0;
+#pragma unroll
+          for (int r = 0; r < R; ++r) {
+            if (!live[r]) continue;
+            const u32 code = lane + 32 * r + d * N3;
+            if (which == 0) stage[code] = mem3[r] + act[d];
+            else if (which == 1) stage[code] = paper3[r];
+            else if (which == 2) stage[code] = ext3[r] + c_axis;
+            else if (which == 3) stage[code] = host3[r] + host_add;
+            else stage32[code] = fl_base[r] | fl_digit | (fl_gi[r] & gi_mask) | (fl_priced[r] & priced_mask);
+          }
+        }
+        __syncwarp();
+        if (which == 0) warp_copy_out(a.out.mem + out_base, stage, NC, lane);
+        else if (which == 1) warp_copy_out(a.out.comm_paper + out_base, stage, NC, lane);
+        else if (which == 2) warp_copy_out(a.out.comm_ext + out_base, stage, NC, lane);
+        else if (which == 3) warp_copy_out(a.out.host + out_base, stage, NC, lane);
+        else warp_copy_out(a.out.flags + out_base, stage32, NC, lane);
+        __syncwarp();
+      }
+      continue;
+    }
 
 #pragma unroll
     for (int d = 0; d < NM; ++d) {
