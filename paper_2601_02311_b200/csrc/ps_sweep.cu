@@ -511,8 +511,9 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
                        (u64)(rec.wT + rec.wO + rec.wG) * (ub.E2 + ub.u) < ((u64)1 << 53);
     if (small) {
       double mem_f64[R];
+      float pass_f32[R];
 #pragma unroll
-      for (int r = 0; r < R; ++r) mem_f64[r] = (double)mem3[r];
+      for (int r = 0; r < R; ++r) { mem_f64[r] = (double)mem3[r]; pass_f32[r] = 0.0f; }
 #pragma unroll
       for (int d = 0; d < NM; ++d) {
         const bool host_check = host_limited && ((is_o >> d) & 1u);
@@ -525,17 +526,20 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
           }
 #pragma unroll
           for (int r = 0; r < R; ++r) {
-            u32 c = 0;
+            // compare on the fp64 pipe, count with predicated fp32 adds (small
+            // integers are exact): nothing here uses the integer ALU pipe
+            float c = 0.0f;
             if (host_check) {
               // offloading activations also has to fit the host budget of the variant
 #pragma unroll
               for (int vt = 0; vt < 4; ++vt)
-                c += (mem_f64[r] < bound[vt] && host3[r] < tb.host_bound[vt]) ? 1u : 0u;
+                if (mem_f64[r] < bound[vt] && host3[r] < tb.host_bound[vt]) c += 1.0f;
             } else {
 #pragma unroll
-              for (int vt = 0; vt < 4; ++vt) c += (mem_f64[r] < bound[vt]) ? 1u : 0u;
+              for (int vt = 0; vt < 4; ++vt)
+                if (mem_f64[r] < bound[vt]) c += 1.0f;
             }
-            n_pass[r] += ((allowed[r] >> d) & 1u) ? c : 0u;
+            if ((allowed[r] >> d) & 1u) pass_f32[r] += c;
           }
         } else {
           u64 bound[4];
@@ -553,6 +557,8 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
           }
         }
       }
+#pragma unroll
+      for (int r = 0; r < R; ++r) n_pass[r] += (u32)pass_f32[r];
     } else {
 #pragma unroll
     for (int d = 0; d < NM; ++d) {
