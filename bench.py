@@ -56,7 +56,7 @@ BYTES_PER_POINT_MATERIALISE = 36
 # (k_sweep<top-k> on the full stress configuration; k_eval<materialise> per point
 # of a 2^25-point window, where traffic grows in proportion to the points)
 NCU_SWEEP_DRAM_BYTES = 499_968
-NCU_MATERIALISE_DRAM_BYTES_PER_POINT = 1_249_138_000 / (1 << 25)
+NCU_MATERIALISE_DRAM_BYTES_PER_POINT = 1_268_337_000 / (1 << 25)
 
 
 def parse_args():
