@@ -1,6 +1,9 @@
 """Compile the CUDA library for sm_100a into ``paper_2601_02311_b200/libps_b200.so``.
 
 ``python -m paper_2601_02311_b200.build [--verbose]``
+
+Extra compiler flags (for instance ``-DEVAL_GRID_PER_SM=4`` to try another launch
+shape) can be given in the environment variable ``PS_NVCC_FLAGS``.
 """
 from __future__ import annotations
 
@@ -36,6 +39,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc] + NVCC_FLAGS + ["-I", os.path.join(ROOT, "include"), "-I", CSRC]
+    cmd += os.environ.get("PS_NVCC_FLAGS", "").split()
     if verbose:
         cmd += ["-Xptxas", "-v"]
     tmp = LIB + ".tmp.%d" % os.getpid()

@@ -11,7 +11,10 @@
 // widths -- so they are computed once per model and a group costs a few
 // multiply-adds per triple.  The activation digit then adds one of NM
 // per-group values.  Codes of a group run digit-major, triple-minor, so for a
-// fixed digit the lanes write consecutive elements: all stores are coalesced.
+// fixed digit the lanes write consecutive elements.  Materialise stages one
+// output array of a group in shared memory and stores it with one bulk copy
+// (shared -> global, asynchronous), so the warp computes the next array while
+// the previous one drains.
 //
 // Compaction is count -> scan -> write: the count pass stores the survivors of
 // each group, a single-block scan turns them into offsets, the write pass
@@ -22,6 +25,18 @@
 
 namespace {
 
+// Launch shapes (blocks per SM; two are resident at a time).  Materialise is
+// fastest with about one group per warp: short-lived blocks keep the warps of an
+// SM at different stages (set-up, staging, draining stores) and the running
+// warps write neighbouring stretches of every output array.  Count and write
+// are arithmetic-bound and prefer long runs of groups per warp (the per-model
+// coefficients are then computed once).
+#ifndef EVAL_GRID_PER_SM_MATERIALISE
+#define EVAL_GRID_PER_SM_MATERIALISE 64
+#endif
+#ifndef EVAL_GRID_PER_SM_COMPACT
+#define EVAL_GRID_PER_SM_COMPACT 2
+#endif
 constexpr int THREADS = EVAL_THREADS;
 constexpr int WARPS = THREADS / 32;
 
@@ -57,39 +72,61 @@ __device__ __forceinline__ u32 triple_static(u32 th, u32 om, u32 gr, bool d1) {
 
 enum { MODE_MATERIALISE = 0, MODE_COUNT = 1, MODE_WRITE = 2 };
 
-// Copy n staged elements of a warp to global memory: scalar stores up to the
-// next 128-byte line, then 16-byte stores (one warp instruction = 512
-// contiguous, line-aligned bytes), then the remainder.  Fewer and fuller
-// requests to the memory system than 8-byte stores at arbitrary offsets.
+// Staging for the materialise path.  A warp builds one output array of one
+// group (NC elements) in shared memory and hands it to the copy engine as a
+// single bulk store (cp.async.bulk, shared -> global), then goes on computing the
+// next array while the store drains; two staging buffers per warp alternate.
+// A bulk store needs both addresses 16-byte aligned and a size that is a
+// multiple of 16 bytes, while an output array is only aligned to its element and
+// a group starts anywhere in it.  So element c of the group is staged at slot
+// c + skew, where skew = (destination address / element size) mod (16 / element
+// size): the shared and global addresses of every element then agree modulo 16,
+// the elements before the first 16-byte boundary and after the last one (at
+// most 16 / element size - 1 each) are written with plain stores, and everything
+// between goes out as one bulk store.
+template <int NC>
+struct Stage {
+  static constexpr int SLOTS = NC + 4;                                   // u64 slots, room for the skew
+  static constexpr int BYTES = ((SLOTS * 8 + 127) / 128) * 128;          // one buffer
+};
+
+__device__ __forceinline__ u32 smem_addr(const void* p) { return (u32)__cvta_generic_to_shared(p); }
+
+// lane 0 owns the warp's bulk stores: wait until at most `pending` of them still read shared memory
+template <int PENDING>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(PENDING) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// All lanes have written `n` elements of type T to buf[skew ...]; store them to dst[0 .. n).
 template <typename T>
-__device__ __forceinline__ void warp_copy_out(T* __restrict__ dst, const T* buf, int n, int lane) {
+__device__ __forceinline__ void warp_bulk_store(T* __restrict__ dst, const T* buf, int skew, int n, int lane) {
   constexpr int PER16 = 16 / (int)sizeof(T);
-  const uintptr_t addr = reinterpret_cast<uintptr_t>(dst);
-  int head = (int)(((128 - (addr & 127)) & 127) / sizeof(T));
-  head = min(head, n);
-  for (int i = lane; i < head; i += 32) dst[i] = buf[i];
-  const int body = (n - head) / PER16;
-  for (int k = lane; k < body; k += 32) {
-    const T* src = buf + head + k * PER16;
-    uint4 v;
-    if (sizeof(T) == 8) {
-      const u64 x = (u64)src[0], y = (u64)src[1];
-      v = make_uint4((u32)x, (u32)(x >> 32), (u32)y, (u32)(y >> 32));
-    } else {
-      v = make_uint4((u32)src[0], (u32)src[1], (u32)src[2], (u32)src[3]);
-    }
-    *reinterpret_cast<uint4*>(dst + head + k * PER16) = v;
+  // make the lanes' shared-memory writes visible to the copy engine
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncwarp();
+  const int head = min((PER16 - skew) & (PER16 - 1), n);                 // elements before the first boundary
+  const int body = ((n - head) / PER16) * PER16;
+  if (lane < head) dst[lane] = buf[skew + lane];
+  const int tail = n - head - body;
+  if (lane < tail) dst[head + body + lane] = buf[skew + head + body + lane];
+  if (lane == 0 && body > 0) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(dst + head), "r"(smem_addr(buf + skew + head)), "r"(body * (int)sizeof(T))
+                 : "memory");
   }
-  for (int i = head + body * PER16 + lane; i < n; i += 32) dst[i] = buf[i];
+  if (lane == 0) asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 
 template <int MODE, int NM>
 __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
   constexpr int N2 = NM * NM, N3 = NM * NM * NM, NC = N3 * NM;
   constexpr int R = (N3 + 31) / 32;
-  // materialise: one group's values of one output array, staged per warp
-  __shared__ __align__(16) u64 stage_all[MODE == MODE_MATERIALISE ? WARPS * NC : 1];
-  u64* stage = stage_all + (MODE == MODE_MATERIALISE ? (threadIdx.x >> 5) * NC : 0);
+  // materialise: two staging buffers per warp (dynamic shared memory, none in the other modes)
+  extern __shared__ __align__(128) unsigned char stage_all[];
+  unsigned char* const stage_warp = stage_all + (threadIdx.x >> 5) * 2 * Stage<NC>::BYTES;
+  u32 stage_turn = 0;                                                     // which buffer is next
   const int lane = threadIdx.x & 31;
   const u32 warp_global = blockIdx.x * WARPS + (threadIdx.x >> 5);
   const u32 n_warps = gridDim.x * WARPS;
@@ -220,11 +257,20 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
     const bool all_out = a.out.mem && a.out.comm_paper && a.out.comm_ext && a.out.host && a.out.flags;
 
     if (MODE == MODE_MATERIALISE && whole && all_out) {
-      // one output array at a time: stage the group's NC values, copy them out
-      // with line-aligned 16-byte stores
+      // one output array at a time: stage the group's NC values, hand them to the copy engine
 #pragma unroll
       for (int which = 0; which < 5; ++which) {
-        u32* stage32 = reinterpret_cast<u32*>(stage);
+        u64* const stage = reinterpret_cast<u64*>(stage_warp + (stage_turn & 1u) * Stage<NC>::BYTES);
+        u32* const stage32 = reinterpret_cast<u32*>(stage);
+        ++stage_turn;
+        u64* const dst64 = (which == 0 ? a.out.mem : which == 1 ? a.out.comm_paper
+                            : which == 2 ? a.out.comm_ext : a.out.host) + out_base;
+        u32* const dst32 = a.out.flags + out_base;
+        const int skew = which < 4 ? (int)((reinterpret_cast<uintptr_t>(dst64) >> 3) & 1)
+                                   : (int)((reinterpret_cast<uintptr_t>(dst32) >> 2) & 3);
+        // the store that used this buffer two arrays ago must have read it completely
+        if (lane == 0) bulk_wait_read<1>();
+        __syncwarp();
 #pragma unroll
         for (int d = 0; d < NM; ++d) {
           const bool d_avail = (avail >> d) & 1u, d_off = (is_o >> d) & 1u, d_notmo = (not_mo >> d) & 1u;
@@ -234,21 +280,16 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
 #pragma unroll
           for (int r = 0; r < R; ++r) {
             if (!live[r]) continue;
-            const u32 code = lane + 32 * r + d * N3;
-            if (which == 0) stage[code] = mem3[r] + act[d];
-            else if (which == 1) stage[code] = paper3[r];
-            else if (which == 2) stage[code] = ext3[r] + c_axis;
-            else if (which == 3) stage[code] = host3[r] + host_add;
-            else stage32[code] = fl_base[r] | fl_digit | (fl_gi[r] & gi_mask) | (fl_priced[r] & priced_mask);
+            const u32 slot = lane + 32 * r + d * N3 + skew;
+            if (which == 0) stage[slot] = mem3[r] + act[d];
+            else if (which == 1) stage[slot] = paper3[r];
+            else if (which == 2) stage[slot] = ext3[r] + c_axis;
+            else if (which == 3) stage[slot] = host3[r] + host_add;
+            else stage32[slot] = fl_base[r] | fl_digit | (fl_gi[r] & gi_mask) | (fl_priced[r] & priced_mask);
           }
         }
-        __syncwarp();
-        if (which == 0) warp_copy_out(a.out.mem + out_base, stage, NC, lane);
-        else if (which == 1) warp_copy_out(a.out.comm_paper + out_base, stage, NC, lane);
-        else if (which == 2) warp_copy_out(a.out.comm_ext + out_base, stage, NC, lane);
-        else if (which == 3) warp_copy_out(a.out.host + out_base, stage, NC, lane);
-        else warp_copy_out(a.out.flags + out_base, stage32, NC, lane);
-        __syncwarp();
+        if (which < 4) warp_bulk_store(dst64, stage, skew, NC, lane);
+        else warp_bulk_store(dst32, stage32, skew, NC, lane);
       }
       continue;
     }
@@ -302,6 +343,8 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
     }
     if (MODE == MODE_COUNT && lane == 0) a.tile_count[seg] = n_kept;
   }
+  // the staging buffers must outlive the bulk stores that read them
+  if (MODE == MODE_MATERIALISE && lane == 0) bulk_wait_all();
 }
 
 // exclusive prefix sum of the per-group survivor counts; one block that walks
@@ -349,8 +392,15 @@ cudaError_t launch_eval_t(const SpaceDev& sp, const EvalArgs& a, cudaStream_t st
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const unsigned needed = (a.n_tiles + WARPS - 1) / WARPS;
-  const unsigned blocks = needed < (unsigned)(sms * 16) ? needed : (unsigned)(sms * 16);
-  k_eval<MODE, NM><<<blocks, THREADS, 0, stream>>>(sp, a);
+  const unsigned most = (unsigned)sms * (MODE == MODE_MATERIALISE ? EVAL_GRID_PER_SM_MATERIALISE : EVAL_GRID_PER_SM_COMPACT);
+  const unsigned blocks = needed < most ? needed : most;
+  constexpr int NC = NM * NM * NM * NM;
+  const size_t smem = MODE == MODE_MATERIALISE ? (size_t)WARPS * 2 * Stage<NC>::BYTES : 0;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(k_eval<MODE, NM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  k_eval<MODE, NM><<<blocks, THREADS, smem, stream>>>(sp, a);
   return cudaGetLastError();
 }
 
