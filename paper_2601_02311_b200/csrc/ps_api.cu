@@ -85,15 +85,15 @@ int enqueue_status_copy(ps_ctx* ctx) {
   return PS_OK;
 }
 
-u32 pick_chunks(const ps_ctx* ctx, const ps_space* sp) {
-  // enough blocks for about three waves of two resident blocks per SM; every
+u32 pick_chunks(const ps_ctx* ctx, const ps_space* sp, int kind) {
+  // enough blocks for about three waves of the resident blocks of every SM; every
   // extra block of a model builds its lists from scratch and ends with a merge,
   // so no more than that
-  const u64 target = (u64)ctx->sm_count * 2 * 3;
+  const u64 target = (u64)ctx->sm_count * sweep_blocks_per_sm(kind) * 3;
   u64 c = (target + sp->dev.n_models - 1) / sp->dev.n_models;
   if (c < 1) c = 1;
   if (c > SWEEP_MAX_CHUNKS) c = SWEEP_MAX_CHUNKS;
-  const u64 by_units = (sp->dev.n_facts + SWEEP_WARPS - 1) / SWEEP_WARPS;   // a unit per warp at least
+  const u64 by_units = (sp->dev.n_facts + sweep_warps(kind) - 1) / sweep_warps(kind);   // a unit per warp at least
   if (c > by_units) c = by_units;
   if (c < 1) c = 1;
   return (u32)c;
@@ -391,8 +391,8 @@ int ps_sweep_pareto(ps_ctx* ctx, const ps_space* sp, const ps_filter* filter,
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return PS_E_CUDA;
 
-  const u32 n_chunks = pick_chunks(ctx, sp);
-  const size_t slots = (size_t)sp->dev.n_models * n_chunks;
+  const u32 n_chunks = pick_chunks(ctx, sp, (int)reduce_kind);
+  const size_t slots = (size_t)sp->dev.n_models * n_chunks * sweep_warps((int)reduce_kind);   // one list per warp
   const size_t partial_bytes = slots * SWEEP_LIST_CAP * sizeof(PartialEntry);
   rc = ensure_scratch(ctx, partial_bytes + slots * sizeof(uint2));
   if (rc != PS_OK) return rc;
@@ -409,7 +409,7 @@ int ps_sweep_pareto(ps_ctx* ctx, const ps_space* sp, const ps_filter* filter,
   memset(&m, 0, sizeof(m));
   m.partial = s.partial;
   m.partial_n = s.partial_n;
-  m.n_chunks = n_chunks;
+  m.n_lists = n_chunks * sweep_warps((int)reduce_kind);
   m.n_caps_total = n_caps;
   m.max_entries = max_entries;
   m.k_keep = s.k_keep;

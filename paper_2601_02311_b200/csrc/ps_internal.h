@@ -31,11 +31,28 @@ struct ps_space {
 };
 
 // ---- sweep
-#define SWEEP_WARPS 8
+// Block shapes of the sweep: warps per block and the resident blocks per SM the
+// kernel is compiled for (which caps its registers).  The top-k sweep gains from
+// more resident warps (five blocks of four warps: 96 registers); the Pareto
+// sweep is fastest with two blocks of eight warps (128 registers).
+#ifndef SWEEP_WARPS_TOPK
+#define SWEEP_WARPS_TOPK 4
+#endif
+#ifndef SWEEP_BLOCKS_TOPK
+#define SWEEP_BLOCKS_TOPK 5
+#endif
+#ifndef SWEEP_WARPS_PARETO
+#define SWEEP_WARPS_PARETO 8
+#endif
+#ifndef SWEEP_BLOCKS_PARETO
+#define SWEEP_BLOCKS_PARETO 2
+#endif
+static inline int sweep_warps(int kind) { return kind == PS_REDUCE_PARETO ? SWEEP_WARPS_PARETO : SWEEP_WARPS_TOPK; }
+static inline int sweep_blocks_per_sm(int kind) { return kind == PS_REDUCE_PARETO ? SWEEP_BLOCKS_PARETO : SWEEP_BLOCKS_TOPK; }
 #define SWEEP_LIST_CAP 128        /* entries of a warp's list and of a block's partial list */
 #define SWEEP_MAX_CHUNKS 16       /* blocks per model                                        */
-#define MERGE_CAP (SWEEP_MAX_CHUNKS * SWEEP_LIST_CAP)
-#define SWEEP_MAX_PER_THREAD 8    /* MERGE_CAP / threads per block                           */
+#define MERGE_CAP (9 * SWEEP_LIST_CAP)    /* entries the merge kernel combines at a time: what it
+                                     has kept plus the lists of one block of the sweep       */
 #define PS_MAX_CAPS 8
 
 struct PartialEntry {
@@ -50,8 +67,8 @@ struct SweepArgs {
   u32 require_flags;    // without PS_F_FEASIBLE
   u32 comm_kind;
   u32 k_keep;           // top-k: entries kept
-  PartialEntry* partial;   // [n_models * n_chunks][SWEEP_LIST_CAP]
-  uint2* partial_n;        // [n_models * n_chunks]: (entries, survivors)
+  PartialEntry* partial;   // [n_models * n_chunks * warps][SWEEP_LIST_CAP]: one list per warp
+  uint2* partial_n;        // [n_models * n_chunks * warps]: (entries, survivors)
   u32* status;
 };
 
@@ -59,7 +76,7 @@ struct MergeArgs {
   const PartialEntry* partial;
   const uint2* partial_n;
   u64 caps[PS_MAX_CAPS];
-  u32 n_chunks;
+  u32 n_lists;          // partial lists per model: blocks per model x warps per block
   u32 n_caps;           // capacities this launch emits
   u32 n_caps_total;     // capacities of the output layout
   u32 cap_index;        // top-k: which capacity this launch is for

@@ -14,20 +14,17 @@
 //
 // Reductions.  Every warp keeps a private sorted list in shared memory
 // (Pareto staircase or top-k), tests its candidates against it lane-parallel
-// and inserts the few that pass warp-cooperatively.  At the end the block sorts
-// the union of its warps' lists, prunes it and writes one partial list per
-// block to global scratch; k_sweep_merge combines the partial lists of a model
-// and emits entries, re-evaluating each emitted point from its index as a
-// self-check.
+// and inserts the few that pass warp-cooperatively.  A warp that has run out of
+// units writes its list to global scratch and is done -- the warps of a block
+// never wait for one another; k_sweep_merge combines the partial lists of a
+// model (one block per model: sort, prune) and emits entries, re-evaluating
+// each emitted point from its index as a self-check.
 #include "ps_device.cuh"
 #include "ps_internal.h"
 
 namespace {
 
-constexpr int WARPS = SWEEP_WARPS;
-constexpr int THREADS = WARPS * 32;
 constexpr int LIST_CAP = SWEEP_LIST_CAP;       // entries per warp list / per partial list
-constexpr int BLOCK_CAP = WARPS * LIST_CAP;    // union of the warps' lists
 constexpr u64 U64MAX = ~0ull;
 
 // per-warp tables, rebuilt for every unit: what depends on the activation
@@ -141,28 +138,69 @@ __device__ __noinline__ void pareto_insert(WarpList& w, u64 m, u64 c, u32 idx, i
 // keeps the k smallest and tightens the threshold to the k-th; until the first
 // such compaction the threshold is "everything".  A stale threshold only lets
 // extra candidates in, never keeps a wanted one out.
+//
+// The sort runs in registers: lane l holds entries 4l .. 4l+3, a bitonic network
+// exchanges within a lane for distances below four and by shuffles above.
+__device__ __forceinline__ Key key_shfl_xor(const Key& x, int lanes) {
+  Key o;
+  o.a = __shfl_xor_sync(0xffffffffu, x.a, lanes);
+  o.b = __shfl_xor_sync(0xffffffffu, x.b, lanes);
+  o.i = __shfl_xor_sync(0xffffffffu, x.i, lanes);
+  return o;
+}
+
 __device__ __noinline__ void topk_compact(WarpList& w, int k_keep, int lane, Key& threshold,
                                           unsigned long long* block_comm_limit) {
-  for (int p = w.n + lane; p < LIST_CAP; p += 32) { w.a[p] = U64MAX; w.b[p] = U64MAX; w.i[p] = 0xffffffffu; }
-  __syncwarp();
-  for (int k = 2; k <= LIST_CAP; k <<= 1) {
-    for (int j = k >> 1; j > 0; j >>= 1) {
+  constexpr int PER = LIST_CAP / 32;
+  Key e[PER];
 #pragma unroll
-      for (int e = 0; e < LIST_CAP / 64; ++e) {
-        const int t = lane + 32 * e;                       // pair number
-        const int p = ((t & ~(j - 1)) << 1) | (t & (j - 1));
-        const int q = p | j;
-        const Key x{w.a[p], w.b[p], w.i[p]}, y{w.a[q], w.b[q], w.i[q]};
-        const bool up = (p & k) == 0;
-        if (key_less(y, x) == up) {
-          w.a[p] = y.a; w.b[p] = y.b; w.i[p] = y.i;
-          w.a[q] = x.a; w.b[q] = x.b; w.i[q] = x.i;
+  for (int r = 0; r < PER; ++r) {
+    const int p = PER * lane + r;
+    if (p < w.n) { e[r].a = w.a[p]; e[r].b = w.b[p]; e[r].i = w.i[p]; }
+    else { e[r].a = U64MAX; e[r].b = U64MAX; e[r].i = 0xffffffffu; }
+  }
+  // the network's steps as rolled loops: this code runs rarely, so it is kept
+  // small (a long unrolled sequence that is not in the instruction cache costs
+  // more to fetch than to execute)
+  static_assert(PER == 4, "the exchanges inside a lane are written out for four entries");
+#pragma unroll 1
+  for (int k = 2; k <= LIST_CAP; k <<= 1) {
+#pragma unroll 1
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      if (j >= PER) {
+        const int lanes = j / PER;
+        const bool lower = (lane & lanes) == 0;            // this lane holds the lower index of each pair
+#pragma unroll
+        for (int r = 0; r < PER; ++r) {
+          const Key o = key_shfl_xor(e[r], lanes);
+          const bool up = ((PER * lane + r) & k) == 0;     // ascending run
+          const bool o_less = key_less(o, e[r]);
+          if ((lower == up) ? o_less : !o_less) e[r] = o;   // keep the smaller / the larger of the pair
+        }
+      } else if (j == 2) {
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          const bool up = ((PER * lane + r) & k) == 0;
+          if (key_less(e[r + 2], e[r]) == up) { const Key t = e[r]; e[r] = e[r + 2]; e[r + 2] = t; }
+        }
+      } else {
+#pragma unroll
+        for (int r = 0; r < PER; r += 2) {
+          const bool up = ((PER * lane + r) & k) == 0;
+          if (key_less(e[r + 1], e[r]) == up) { const Key t = e[r]; e[r] = e[r + 1]; e[r + 1] = t; }
         }
       }
-      __syncwarp();
     }
   }
-  w.n = min(w.n, k_keep);
+  const int n_new = min(w.n, k_keep);
+  __syncwarp();
+#pragma unroll
+  for (int r = 0; r < PER; ++r) {
+    const int p = PER * lane + r;
+    if (p < n_new) { w.a[p] = e[r].a; w.b[p] = e[r].b; w.i[p] = e[r].i; }
+  }
+  w.n = n_new;
+  __syncwarp();
   if (w.n == k_keep) {
     threshold.a = w.a[k_keep - 1]; threshold.b = w.b[k_keep - 1]; threshold.i = w.i[k_keep - 1];
     // k points with at most this much communication exist: tell the other warps
@@ -190,84 +228,12 @@ __device__ __forceinline__ void topk_append(WarpList& w, bool cand, const Key& k
   __syncwarp();
 }
 
-// ------------------------------------------------------------------ block sort / prune
-// Bitonic sort of n_pad (power of two) keys in shared memory by key_less.
-__device__ void block_sort(u64* a, u64* b, u32* i, int n_pad, int tid, int n_threads) {
-  for (int k = 2; k <= n_pad; k <<= 1) {
-    for (int j = k >> 1; j > 0; j >>= 1) {
-      for (int p = tid; p < n_pad; p += n_threads) {
-        int q = p ^ j;
-        if (q > p) {
-          Key x{a[p], b[p], i[p]}, y{a[q], b[q], i[q]};
-          bool up = (p & k) == 0;
-          if (key_less(y, x) == up) {
-            a[p] = y.a; b[p] = y.b; i[p] = y.i;
-            a[q] = x.a; b[q] = x.b; i[q] = x.i;
-          }
-        }
-      }
-      __syncthreads();
-    }
-  }
-}
-
-// After sorting by (mem, comm, idx): an entry is on the frontier iff its comm
-// is below the comm of every earlier entry.  Keeps the frontier at the front,
-// returns its length.  `scratch` holds >= n_threads u64 and n_threads int.
-__device__ int block_pareto_prune(u64* a, u64* b, u32* i, int n, int tid, int n_threads,
-                                  u64* smin, int* scount) {
-  int per = (n + n_threads - 1) / n_threads;
-  int lo = min(tid * per, n), hi = min(lo + per, n);
-  u64 local = U64MAX;
-  for (int p = lo; p < hi; ++p) local = min(local, b[p]);
-  smin[tid] = local;
-  __syncthreads();
-  u64 before = U64MAX;                               // min comm of all entries before lo
-  for (int t = 0; t < tid; ++t) before = min(before, smin[t]);
-  int kept = 0;
-  u64 run = before;
-  for (int p = lo; p < hi; ++p) {
-    if (b[p] < run) { ++kept; run = b[p]; }
-  }
-  scount[tid] = kept;
-  __syncthreads();
-  int offset = 0, total = 0;
-  for (int t = 0; t < n_threads; ++t) {
-    if (t < tid) offset += scount[t];
-    total += scount[t];
-  }
-  // gather survivors into registers (at most `per`), then write after a barrier
-  Key keep[SWEEP_MAX_PER_THREAD];
-  int nk = 0;
-  run = before;
-  for (int p = lo; p < hi; ++p) {
-    if (b[p] < run) { run = b[p]; keep[nk].a = a[p]; keep[nk].b = b[p]; keep[nk].i = i[p]; ++nk; }
-  }
-  __syncthreads();
-  for (int k = 0; k < nk; ++k) { a[offset + k] = keep[k].a; b[offset + k] = keep[k].b; i[offset + k] = keep[k].i; }
-  __syncthreads();
-  return total;
-}
-
-__device__ __forceinline__ int next_pow2(int n) {
-  int p = 1;
-  while (p < n) p <<= 1;
-  return p;
-}
-
-static_assert(STAIR == THREADS, "the staircase is cleared one entry per thread");
+template <int WARPS>
 struct SweepShared {
   WarpTables tables[WARPS];
-  u64 list_a[BLOCK_CAP];
-  u64 list_b[BLOCK_CAP];
-  u32 list_i[BLOCK_CAP];
-  u64 merge_a[BLOCK_CAP];
-  u64 merge_b[BLOCK_CAP];
-  u32 merge_i[BLOCK_CAP];
-  u64 smin[THREADS];
-  int scount[THREADS];
-  int warp_n[WARPS];
-  u32 warp_survivors[WARPS];
+  u64 list_a[WARPS * LIST_CAP];
+  u64 list_b[WARPS * LIST_CAP];
+  u32 list_i[WARPS * LIST_CAP];
   u32 next_unit;
   unsigned long long block_comm_limit;   // top-k: no point with more communication can matter
   unsigned long long stair[STAIR];       // Pareto: coarse staircase of the block
@@ -334,12 +300,15 @@ __device__ __forceinline__ u32 allowed_act_digits(u32 tb, u32 req, u32 all, u32 
   return ok;
 }
 
-template <int KIND, int NM>
-__global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs args) {
+// KIND: the reduction; NM: allowed modes; WARPS x 32 threads per block, compiled
+// for MIN_BLOCKS resident blocks per SM
+template <int KIND, int NM, int WARPS, int MIN_BLOCKS>
+__global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, SweepArgs args) {
+  constexpr int THREADS = WARPS * 32;
   constexpr int N2 = NM * NM, N3 = NM * NM * NM, NC = N3 * NM;
   constexpr int R = (N3 + 31) / 32;                 // triples per lane
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  SweepShared& sh = *reinterpret_cast<SweepShared*>(smem_raw);
+  SweepShared<WARPS>& sh = *reinterpret_cast<SweepShared<WARPS>*>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const u32 model = blockIdx.y, chunk = blockIdx.x, n_chunks = gridDim.x;
 
@@ -349,7 +318,8 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
   const u32 u_begin = (u32)(((u64)blockIdx.x * sp.n_facts) / gridDim.x);
   const u32 u_end = (u32)(((u64)(blockIdx.x + 1) * sp.n_facts) / gridDim.x);
   if (tid == 0) { sh.next_unit = u_begin + WARPS; sh.block_comm_limit = U64MAX; }
-  if (KIND == PS_REDUCE_PARETO) sh.stair[tid] = U64MAX;   // STAIR == THREADS
+  if (KIND == PS_REDUCE_PARETO)
+    for (int j = tid; j < STAIR; j += THREADS) sh.stair[j] = U64MAX;
   __syncthreads();
   const ModelRec& rec = sh.rec;
 
@@ -593,8 +563,19 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
     // ---- reduction pass, only if some survivor of this warp can matter
     bool matters = false;
     if (KIND == PS_REDUCE_PARETO) {
+      // a triple's survivors hold at least the triple's own bytes and send at least
+      // its own volume plus the cheapest variant's axis traffic: if a point the
+      // block has already kept beats that bound strictly in bytes (a lower bucket
+      // of the coarse staircase) with no more communication, none of them can be
+      // on the frontier
+      const u64 least_axis = tb.c_axis[0];   // tau = 0 sends the smaller boundary tensor; v does not matter
 #pragma unroll
-      for (int r = 0; r < R; ++r) matters = matters || n_pass[r] != 0;
+      for (int r = 0; r < R; ++r) {
+        if (n_pass[r] != 0) {
+          const int bucket = stair_bucket(mem3[r]);
+          if (bucket == 0 || sh.stair[bucket - 1] > comm3[r] + least_axis) matters = true;
+        }
+      }
     } else {
       const u64 comm_limit = min(threshold.a, (u64)sh.block_comm_limit);
       const u64 least_axis = tb.c_axis[0];   // tau = 0 sends the smaller boundary tensor; v does not matter
@@ -605,56 +586,64 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
       }
     }
     if (__any_sync(0xffffffffu, matters)) {
-    if (KIND == PS_REDUCE_PARETO) {
-      // lane = a set of activation digits; which of them costs the least bytes
-      for (u32 vt = 0; vt < nvt; ++vt) {
-        u64 least = U64MAX;
-        u32 which = NM;
-#pragma unroll
-        for (int d = NM - 1; d >= 0; --d) {
-          const u64 am = tb.act[vt][d];
-          if (((lane >> d) & 1) && am <= least) { least = am; which = d; }
-        }
-        tb.least[vt][lane] = (unsigned char)which;
-      }
-      __syncwarp();
-    }
-
-#pragma unroll 1
-    for (u32 vt = 0; vt < nvt; ++vt) {
-      const u64 c_axis = tb.c_axis[vt], host_bound = tb.host_bound[vt];
-      u64 bound[NM];
-#pragma unroll
-      for (int d = 0; d < NM; ++d) bound[d] = tb.bound[d][vt];
-      // every point of (triple, variant): digit d is a survivor if the triple's
-      // bytes are below the digit's bound and the flags allow the digit
-      u32 pass[R];
+      // This part runs for a few units in a hundred, so it is written as rolled
+      // loops over the lane's triples, whose values it first copies to arrays that
+      // can be indexed at run time: code that is rarely executed is not in the
+      // instruction cache, and fetching a long unrolled sequence costs far more
+      // than executing it.
+      u64 l_mem[R], l_comm[R], l_host[R];
+      u32 l_allowed[R], l_triple[R], l_pass[R];
 #pragma unroll
       for (int r = 0; r < R; ++r) {
-        u32 fit = 0;
-#pragma unroll
-        for (int d = 0; d < NM; ++d) fit |= (mem3[r] < bound[d]) ? (1u << d) : 0u;
-        // offloading activations adds host bytes: drop that digit if they do not fit
-        const u32 allow_vt = (host3[r] < host_bound) ? allowed[r] : (allowed[r] & ~is_o);
-        pass[r] = fit & allow_vt;
+        l_mem[r] = mem3[r]; l_comm[r] = comm3[r]; l_host[r] = host3[r];
+        l_allowed[r] = allowed[r]; l_triple[r] = t_local[r];
       }
-      const u32 vt_first = unit_first + vt * NC;
-
       if (KIND == PS_REDUCE_PARETO) {
-        // For a triple and variant the communication is the same for all NM
-        // activation digits, so of the surviving digits only the one with the
-        // least bytes (lowest digit on ties) can be on the frontier.
+        // lane = a set of activation digits; which of them costs the least bytes
+        for (u32 vt = 0; vt < nvt; ++vt) {
+          u64 least = U64MAX;
+          u32 which = NM;
+#pragma unroll 1
+          for (int d = NM - 1; d >= 0; --d) {
+            const u64 am = tb.act[vt][d];
+            if (((lane >> d) & 1) && am <= least) { least = am; which = d; }
+          }
+          tb.least[vt][lane] = (unsigned char)which;
+        }
+        __syncwarp();
+      }
+
+#pragma unroll 1
+      for (u32 vt = 0; vt < nvt; ++vt) {
+        const u64 c_axis = tb.c_axis[vt], host_bound = tb.host_bound[vt];
+        const u32 vt_first = unit_first + vt * NC;
+        // every point of (triple, variant): digit d is a survivor if the triple's
+        // bytes are below the digit's bound and the flags allow the digit
         bool some = false;
-#pragma unroll
-        for (int r = 0; r < R; ++r) some = some || pass[r] != 0;
-        if (__any_sync(0xffffffffu, some)) {
-#pragma unroll
+#pragma unroll 1
+        for (int r = 0; r < R; ++r) {
+          u32 fit = 0;
+#pragma unroll 1
+          for (int d = 0; d < NM; ++d) fit |= (l_mem[r] < tb.bound[d][vt]) ? (1u << d) : 0u;
+          // offloading activations adds host bytes: drop that digit if they do not fit
+          const u32 allow_vt = (l_host[r] < host_bound) ? l_allowed[r] : (l_allowed[r] & ~is_o);
+          l_pass[r] = fit & allow_vt;
+          some = some || l_pass[r] != 0;
+        }
+        if (!__any_sync(0xffffffffu, some)) continue;
+
+        if (KIND == PS_REDUCE_PARETO) {
+          // For a triple and variant the communication is the same for all NM
+          // activation digits, so of the surviving digits only the one with the
+          // least bytes (lowest digit on ties) can be on the frontier.
+#pragma unroll 1
           for (int r = 0; r < R; ++r) {
-            const bool has = pass[r] != 0;
-            const u32 d = has ? tb.least[vt][pass[r]] : 0;
-            const u64 m = mem3[r] + tb.act[vt][d];
-            const u64 c = comm3[r] + c_axis;
-            const u32 idx = vt_first + t_local[r] + d * N3;
+            const u32 pass = l_pass[r];
+            const bool has = pass != 0;
+            const u32 d = has ? tb.least[vt][pass] : 0;
+            const u64 m = l_mem[r] + tb.act[vt][d];
+            const u64 c = l_comm[r] + c_axis;
+            const u32 idx = vt_first + l_triple[r] + d * N3;
             // cheap tests first: strictly dominated by a point already known to survive
             bool cand = has && !(dom_m <= m && dom_c <= c && (dom_m != m || dom_c != c));
             if (cand) {
@@ -687,31 +676,25 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
               }
             }
           }
-        }
-      } else {
-        // the k-th smallest communication known to this warp or to any warp of the block
-        const u64 comm_limit = min(threshold.a, (u64)sh.block_comm_limit);
-        bool hot = false;
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-          hot = hot || (pass[r] != 0 && comm3[r] + c_axis <= comm_limit);
-        }
-        if (__any_sync(0xffffffffu, hot)) {
+        } else {
+          // the k-th smallest communication known to this warp or to any warp of the block
+          const u64 comm_limit = min(threshold.a, (u64)sh.block_comm_limit);
           // survivors that are below the threshold key, per triple as digit bits
-          u32 cand[R];
           u32 mine = 0;
-#pragma unroll
+#pragma unroll 1
           for (int r = 0; r < R; ++r) {
-            const u64 c = comm3[r] + c_axis;
-            cand[r] = (c < threshold.a && c <= comm_limit) ? pass[r] : 0u;
-            if (c == threshold.a && pass[r] != 0) {
-#pragma unroll
+            const u64 c = l_comm[r] + c_axis;
+            const u32 pass = l_pass[r];
+            u32 cand = (c < threshold.a && c <= comm_limit) ? pass : 0u;
+            if (c == threshold.a && pass != 0) {
+#pragma unroll 1
               for (int d = 0; d < NM; ++d) {
-                const Key key{c, mem3[r] + tb.act[vt][d], vt_first + t_local[r] + d * N3};
-                if (((pass[r] >> d) & 1u) && key_less(key, threshold)) cand[r] |= 1u << d;
+                const Key key{c, l_mem[r] + tb.act[vt][d], vt_first + l_triple[r] + d * N3};
+                if (((pass >> d) & 1u) && key_less(key, threshold)) cand |= 1u << d;
               }
             }
-            mine += __popc(cand[r]);
+            l_pass[r] = cand;
+            mine += __popc(cand);
           }
           u32 incl = mine;                               // inclusive prefix sum over the lanes
 #pragma unroll
@@ -720,31 +703,32 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
             if (lane >= o) incl += up;
           }
           const u32 total = __shfl_sync(0xffffffffu, incl, 31);
-          if (total != 0 && list.n + total <= (u32)LIST_CAP) {
+          if (total == 0) continue;
+          if (list.n + total <= (u32)LIST_CAP) {
             int p = list.n + (int)(incl - mine);
-#pragma unroll
+#pragma unroll 1
             for (int r = 0; r < R; ++r) {
-              u32 bits = cand[r];
+              u32 bits = l_pass[r];
               while (bits) {
                 const u32 d = __ffs(bits) - 1;
                 bits &= bits - 1;
-                list.a[p] = comm3[r] + c_axis;
-                list.b[p] = mem3[r] + tb.act[vt][d];
-                list.i[p] = vt_first + t_local[r] + d * N3;
+                list.a[p] = l_comm[r] + c_axis;
+                list.b[p] = l_mem[r] + tb.act[vt][d];
+                list.i[p] = vt_first + l_triple[r] + d * N3;
                 ++p;
               }
             }
             list.n += (int)total;
             __syncwarp();
-          } else if (total != 0) {
+          } else {
             // does not fit in one go: one (triple round, digit) at a time, compacting as needed
 #pragma unroll 1
             for (u32 d = 0; d < (u32)NM; ++d) {
               const u64 am = tb.act[vt][d];
-#pragma unroll
+#pragma unroll 1
               for (int r = 0; r < R; ++r) {
-                const Key key{comm3[r] + c_axis, mem3[r] + am, vt_first + t_local[r] + d * N3};
-                topk_append(list, ((cand[r] >> d) & 1u) && key_less(key, threshold), key, k_keep, lane,
+                const Key key{l_comm[r] + c_axis, l_mem[r] + am, vt_first + l_triple[r] + d * N3};
+                topk_append(list, ((l_pass[r] >> d) & 1u) && key_less(key, threshold), key, k_keep, lane,
                             threshold, &sh.block_comm_limit);
               }
             }
@@ -755,133 +739,179 @@ __global__ void __launch_bounds__(THREADS, 2) k_sweep(SpaceDev sp, SweepArgs arg
         }
       }
     }
-    }
     // next unit
     u32 nxt = 0;
     if (lane == 0) nxt = atomicAdd(&sh.next_unit, 1u);
     unit = __shfl_sync(0xffffffffu, nxt, 0);
   }
 
-  // ---- block-level merge of the warps' lists
+  // ---- the warp's list goes to global scratch, sorted (top-k: its k smallest
+  // by key; Pareto: the staircase, ascending bytes); nothing waits for the other warps
   for (int o = 16; o > 0; o >>= 1) survivors += __shfl_xor_sync(0xffffffffu, survivors, o);
-  int n_out;
-  if (KIND == PS_REDUCE_TOPK) {
-    // every warp sorts its own list and keeps its k smallest; an entry's place in
-    // the block's list is then its place at home plus, for every other warp, the
-    // number of that warp's entries below it (keys are distinct: binary searches,
-    // no block-wide sort)
-    if (list.n > 0) topk_compact(list, k_keep, lane, threshold, &sh.block_comm_limit);
-    if (lane == 0) { sh.warp_n[warp] = list.n; sh.warp_survivors[warp] = survivors; }
-    __syncthreads();
-    int total = 0;
-    for (int w = 0; w < WARPS; ++w) total += sh.warp_n[w];
-    for (int e = lane; e < list.n; e += 32) {
-      const Key key{list.a[e], list.b[e], list.i[e]};
-      int rank = e;
-      for (int w = 0; w < WARPS; ++w) {
-        if (w == warp) continue;
-        const u64* oa = sh.list_a + w * LIST_CAP;
-        const u64* ob = sh.list_b + w * LIST_CAP;
-        const u32* oi = sh.list_i + w * LIST_CAP;
-        int lo = 0, hi = sh.warp_n[w];
-        while (lo < hi) {
-          const int mid = (lo + hi) >> 1;
-          const Key other{oa[mid], ob[mid], oi[mid]};
-          if (key_less(other, key)) lo = mid + 1; else hi = mid;
-        }
-        rank += lo;
-      }
-      if (rank < k_keep) { sh.merge_a[rank] = key.a; sh.merge_b[rank] = key.b; sh.merge_i[rank] = key.i; }
-    }
-    __syncthreads();
-    n_out = min(total, k_keep);
-  } else {
-    if (lane == 0) { sh.warp_n[warp] = list.n; sh.warp_survivors[warp] = survivors; }
-    __syncthreads();
-    int total = 0, my_off = 0;
-    for (int w = 0; w < WARPS; ++w) {
-      if (w < warp) my_off += sh.warp_n[w];
-      total += sh.warp_n[w];
-    }
-    const int n_pad = next_pow2(max(total, 1));
-    for (int p = lane; p < list.n; p += 32) {
-      sh.merge_a[my_off + p] = list.a[p]; sh.merge_b[my_off + p] = list.b[p]; sh.merge_i[my_off + p] = list.i[p];
-    }
-    for (int p = total + tid; p < n_pad; p += THREADS) {
-      sh.merge_a[p] = U64MAX; sh.merge_b[p] = U64MAX; sh.merge_i[p] = 0xffffffffu;
-    }
-    __syncthreads();
-    block_sort(sh.merge_a, sh.merge_b, sh.merge_i, n_pad, tid, THREADS);
-    n_out = block_pareto_prune(sh.merge_a, sh.merge_b, sh.merge_i, total, tid, THREADS, sh.smin, sh.scount);
-    if (n_out > LIST_CAP) {
-      if (tid == 0) atomicOr(args.status, ST_LIST_OVERFLOW);
-      n_out = LIST_CAP;
-    }
-  }
-  const u64 slot = (u64)model * n_chunks + chunk;
+  if (KIND == PS_REDUCE_TOPK && list.n > 0) topk_compact(list, k_keep, lane, threshold, &sh.block_comm_limit);
+  __syncwarp();
+  const u64 slot = ((u64)model * n_chunks + chunk) * WARPS + warp;
   PartialEntry* dst = args.partial + slot * LIST_CAP;
-  for (int p = tid; p < n_out; p += THREADS) {
+  for (int p = lane; p < list.n; p += 32) {
     PartialEntry e;
-    e.a = sh.merge_a[p]; e.b = sh.merge_b[p]; e.i = sh.merge_i[p]; e.pad = 0;
+    e.a = list.a[p]; e.b = list.b[p]; e.i = list.i[p]; e.pad = 0;
     dst[p] = e;
   }
-  if (tid == 0) {
-    u32 s = 0;
-    for (int w = 0; w < WARPS; ++w) s += sh.warp_survivors[w];
-    args.partial_n[slot] = make_uint2((u32)n_out, s);
-  }
+  if (lane == 0) args.partial_n[slot] = make_uint2((u32)list.n, survivors);
 }
 
 // ------------------------------------------------------------------ merge + emit
-// One block per model: combine the n_chunks partial lists, then write the
-// entries of every capacity.  Each emitted point is evaluated again from its
-// index (host bytes and flags come from there; mem and comm must agree).
+// One block per model: combine the partial lists of the model's warps (n_lists
+// = blocks per model x warps per block), then write the entries of every
+// capacity.  Every list arrives sorted by key -- (mem, comm, idx) for Pareto,
+// where a staircase has distinct ascending bytes, (comm, mem, idx) for top-k --
+// and no point is in two lists, so an entry's place in the sorted union is its
+// place at home plus, for every other list, the number of entries below it
+// there: binary searches, no sort.  The union is then cut back (top-k: the k
+// smallest; Pareto: entries whose communication is below that of everything
+// before them).  Lists are taken in rounds of MERGE_LISTS beside what has been
+// kept so far, so any number can be combined.  Each emitted point is evaluated
+// again from its index (host bytes and flags come from there; mem and comm must
+// agree).
+constexpr int MERGE_THREADS = 256;
+constexpr int MERGE_LISTS = MERGE_CAP / LIST_CAP - 1;   // lists per round beside the kept entries
+
 struct MergeShared {
-  u64 a[MERGE_CAP];
-  u64 b[MERGE_CAP];
+  u64 in_a[MERGE_CAP], in_b[MERGE_CAP];     // the kept entries, then the round's lists
+  u32 in_i[MERGE_CAP];
+  u64 a[MERGE_CAP], b[MERGE_CAP];           // the sorted union; after the cut, the kept entries
   u32 i[MERGE_CAP];
-  u64 smin[THREADS];
-  int scount[THREADS];
+  int off[MERGE_LISTS + 2];                 // start of each list in in_*
+  u64 warp_min[MERGE_THREADS / 32];
+  int warp_sum[MERGE_THREADS / 32];
+  u32 survivors;
 };
 
+// exclusive prefix minimum / prefix sum over the threads of a block
+__device__ __forceinline__ u64 block_excl_min(u64 mine, u64* warp_min, int tid) {
+  const int lane = tid & 31, warp = tid >> 5;
+  u64 incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const u64 up = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl = min(incl, up);
+  }
+  u64 excl = __shfl_up_sync(0xffffffffu, incl, 1);
+  if (lane == 0) excl = U64MAX;
+  if (lane == 31) warp_min[warp] = incl;
+  __syncthreads();
+  for (int w = 0; w < warp; ++w) excl = min(excl, warp_min[w]);
+  __syncthreads();
+  return excl;
+}
+__device__ __forceinline__ int block_excl_sum(int mine, int* warp_sum, int tid, int* total) {
+  const int lane = tid & 31, warp = tid >> 5;
+  int incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int up = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += up;
+  }
+  if (lane == 31) warp_sum[warp] = incl;
+  __syncthreads();
+  int before = 0, all = 0;
+  for (int w = 0; w < MERGE_THREADS / 32; ++w) {
+    if (w < warp) before += warp_sum[w];
+    all += warp_sum[w];
+  }
+  __syncthreads();
+  *total = all;
+  return before + incl - mine;
+}
+
 template <int KIND>
-__global__ void __launch_bounds__(THREADS) k_sweep_merge(SpaceDev sp, MergeArgs args) {
+__global__ void __launch_bounds__(MERGE_THREADS) k_sweep_merge(SpaceDev sp, MergeArgs args) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   MergeShared& sh = *reinterpret_cast<MergeShared*>(smem_raw);
   const int tid = threadIdx.x;
   const u32 model = blockIdx.x;
-  const u32 n_chunks = args.n_chunks;
-  __shared__ int s_off[SWEEP_MAX_CHUNKS + 1];
-  __shared__ u32 s_survivors;
-  if (tid == 0) {
-    int off = 0;
+  const u32 n_lists = args.n_lists;
+  const uint2* list_n = args.partial_n + (u64)model * n_lists;
+  const PartialEntry* lists = args.partial + (u64)model * n_lists * LIST_CAP;
+  if (tid == 0) sh.survivors = 0;
+  __syncthreads();
+  {
     u32 surv = 0;
-    for (u32 c = 0; c < n_chunks; ++c) {
-      s_off[c] = off;
-      uint2 pn = args.partial_n[(u64)model * n_chunks + c];
-      off += (int)pn.x;
-      surv += pn.y;
-    }
-    s_off[n_chunks] = off;
-    s_survivors = surv;
+    for (u32 l = tid; l < n_lists; l += MERGE_THREADS) surv += list_n[l].y;
+    if (surv) atomicAdd(&sh.survivors, surv);
   }
-  __syncthreads();
-  const int total = s_off[n_chunks];
-  for (u32 c = 0; c < n_chunks; ++c) {
-    const PartialEntry* src = args.partial + ((u64)model * n_chunks + c) * LIST_CAP;
-    const int n = s_off[c + 1] - s_off[c];
-    for (int p = tid; p < n; p += THREADS) {
-      PartialEntry e = src[p];
-      sh.a[s_off[c] + p] = e.a; sh.b[s_off[c] + p] = e.b; sh.i[s_off[c] + p] = e.i;
+  int n_list = 0;                                  // entries kept so far: sh.a/b/i[0, n_list), sorted
+  for (u32 next = 0; next < n_lists; next += MERGE_LISTS) {
+    const int taken = (int)min((u32)MERGE_LISTS, n_lists - next);
+    // list 0 = the kept entries, lists 1..taken = this round's
+    if (tid <= taken + 1) {
+      int off = 0;
+      if (tid >= 1) off = n_list;
+      for (int c = 1; c < tid; ++c) off += min((int)list_n[next + c - 1].x, LIST_CAP);
+      sh.off[tid] = off;
     }
+    for (int p = tid; p < n_list; p += MERGE_THREADS) { sh.in_a[p] = sh.a[p]; sh.in_b[p] = sh.b[p]; sh.in_i[p] = sh.i[p]; }
+    __syncthreads();
+    const int total = sh.off[taken + 1];
+    for (int c = 1; c <= taken; ++c) {
+      const PartialEntry* src = lists + (u64)(next + c - 1) * LIST_CAP;
+      const int base = sh.off[c], n = sh.off[c + 1] - base;
+      for (int p = tid; p < n; p += MERGE_THREADS) {
+        const PartialEntry e = src[p];
+        sh.in_a[base + p] = e.a; sh.in_b[base + p] = e.b; sh.in_i[base + p] = e.i;
+      }
+    }
+    __syncthreads();
+    // place every entry in the sorted union
+    for (int e = tid; e < total; e += MERGE_THREADS) {
+      int home = 0;
+      while (sh.off[home + 1] <= e) ++home;
+      const Key key{sh.in_a[e], sh.in_b[e], sh.in_i[e]};
+      int rank = e - sh.off[home];
+      for (int c = 0; c <= taken; ++c) {
+        if (c == home) continue;
+        int lo = sh.off[c], hi = sh.off[c + 1];
+        const int base = lo;
+        while (lo < hi) {
+          const int mid = (lo + hi) >> 1;
+          const Key other{sh.in_a[mid], sh.in_b[mid], sh.in_i[mid]};
+          if (key_less(other, key)) lo = mid + 1; else hi = mid;
+        }
+        rank += lo - base;
+      }
+      sh.a[rank] = key.a; sh.b[rank] = key.b; sh.i[rank] = key.i;
+    }
+    __syncthreads();
+    if (KIND == PS_REDUCE_TOPK) {
+      n_list = min(total, (int)args.k_keep);
+    } else {
+      // an entry stays iff its communication is below that of every entry before it
+      constexpr int PER = (MERGE_CAP + MERGE_THREADS - 1) / MERGE_THREADS;
+      const int lo = min(tid * PER, total), hi = min(lo + PER, total);
+      u64 local = U64MAX;
+      for (int p = lo; p < hi; ++p) local = min(local, sh.b[p]);
+      const u64 before = block_excl_min(local, sh.warp_min, tid);
+      Key keep[PER];
+      int nk = 0;
+      u64 run = before;
+#pragma unroll
+      for (int k = 0; k < PER; ++k) {
+        const int p = lo + k;
+        if (p < hi && sh.b[p] < run) { run = sh.b[p]; keep[nk].a = sh.a[p]; keep[nk].b = sh.b[p]; keep[nk].i = sh.i[p]; ++nk; }
+      }
+      int kept_total;
+      const int offset = block_excl_sum(nk, sh.warp_sum, tid, &kept_total);   // barriers inside: all reads above are done
+      for (int k = 0; k < nk; ++k)
+        if (offset + k < MERGE_CAP) { sh.a[offset + k] = keep[k].a; sh.b[offset + k] = keep[k].b; sh.i[offset + k] = keep[k].i; }
+      n_list = kept_total;
+      if (n_list > LIST_CAP) {
+        if (tid == 0) atomicOr(args.status, ST_LIST_OVERFLOW);
+        n_list = LIST_CAP;
+      }
+    }
+    __syncthreads();
   }
-  const int n_pad = next_pow2(max(total, 1));
-  for (int p = total + tid; p < n_pad; p += THREADS) { sh.a[p] = U64MAX; sh.b[p] = U64MAX; sh.i[p] = 0xffffffffu; }
-  __syncthreads();
-  block_sort(sh.a, sh.b, sh.i, n_pad, tid, THREADS);
-  int n_list = total;
-  if (KIND == PS_REDUCE_PARETO)
-    n_list = block_pareto_prune(sh.a, sh.b, sh.i, total, tid, THREADS, sh.smin, sh.scount);
+  const u32 s_survivors = sh.survivors;
 
   const ModelRec rec = sp.recs[model];
   for (u32 ci = 0; ci < args.n_caps; ++ci) {
@@ -901,7 +931,7 @@ __global__ void __launch_bounds__(THREADS) k_sweep_merge(SpaceDev sp, MergeArgs 
       args.counts[(u64)model * args.n_caps_total + cap_slot] =
           (KIND == PS_REDUCE_PARETO) ? (u32)n_cap : s_survivors;
     const int n_emit = min(min(n_cap, (int)args.max_entries), KIND == PS_REDUCE_PARETO ? n_cap : (int)args.k_keep);
-    for (int p = tid; p < (int)args.max_entries; p += THREADS) {
+    for (int p = tid; p < (int)args.max_entries; p += MERGE_THREADS) {
       ps_front_entry e;
       e.mem = 0; e.comm = 0; e.host = 0; e.idx = 0; e.flags = 0; e.pad = 0;
       if (p < n_emit) {
@@ -927,16 +957,16 @@ __global__ void __launch_bounds__(THREADS) k_sweep_merge(SpaceDev sp, MergeArgs 
 }  // namespace
 
 // ------------------------------------------------------------------ launchers
-size_t sweep_shared_bytes() { return sizeof(SweepShared); }
-size_t merge_shared_bytes() { return sizeof(MergeShared); }
-
 template <int KIND, int NM>
 static cudaError_t launch_sweep_t(const SpaceDev& sp, const SweepArgs& a, u32 n_chunks, cudaStream_t stream) {
+  constexpr int WARPS = KIND == PS_REDUCE_PARETO ? SWEEP_WARPS_PARETO : SWEEP_WARPS_TOPK;
+  constexpr int MIN_BLOCKS = KIND == PS_REDUCE_PARETO ? SWEEP_BLOCKS_PARETO : SWEEP_BLOCKS_TOPK;
   dim3 grid(n_chunks, sp.n_models);
-  const size_t smem = sizeof(SweepShared);
-  cudaError_t e = cudaFuncSetAttribute(k_sweep<KIND, NM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const size_t smem = sizeof(SweepShared<WARPS>);
+  cudaError_t e = cudaFuncSetAttribute(k_sweep<KIND, NM, WARPS, MIN_BLOCKS>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  k_sweep<KIND, NM><<<grid, THREADS, smem, stream>>>(sp, a);
+  k_sweep<KIND, NM, WARPS, MIN_BLOCKS><<<grid, WARPS * 32, smem, stream>>>(sp, a);
   return cudaGetLastError();
 }
 
@@ -963,11 +993,11 @@ cudaError_t launch_sweep_merge(int kind, const SpaceDev& sp, const MergeArgs& a,
   if (kind == PS_REDUCE_PARETO) {
     e = cudaFuncSetAttribute(k_sweep_merge<PS_REDUCE_PARETO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    k_sweep_merge<PS_REDUCE_PARETO><<<sp.n_models, THREADS, smem, stream>>>(sp, a);
+    k_sweep_merge<PS_REDUCE_PARETO><<<sp.n_models, MERGE_THREADS, smem, stream>>>(sp, a);
   } else {
     e = cudaFuncSetAttribute(k_sweep_merge<PS_REDUCE_TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    k_sweep_merge<PS_REDUCE_TOPK><<<sp.n_models, THREADS, smem, stream>>>(sp, a);
+    k_sweep_merge<PS_REDUCE_TOPK><<<sp.n_models, MERGE_THREADS, smem, stream>>>(sp, a);
   }
   return cudaGetLastError();
 }
