@@ -130,6 +130,25 @@ typedef struct {
                                    2: {S, R}                                            */
   uint32_t mode_mask;           /* bit m set: mode m allowed on the data axis; != 0    */
   uint32_t tp_coll_per_layer;   /* all-reduces per layer per step on the tensor axis, <= 64 */
+  /* Two extensions the paper names without working them out.  Both apply to
+   * the whole space (sweep once per value to compare values); 0 means 1. */
+  uint32_t sstar_units;         /* 1 or 2: unit buffers a gathered (S*) state holds.  Theorem 1
+                                   charges one; its proof notes that an implementation which
+                                   gathers the next unit while the current one is in use needs
+                                   2 * s_unit.  Applies to all four states. */
+  uint32_t grad_accum_steps;    /* 1 .. 64: micro-batches per step (Section "Limitations":
+                                   gradient accumulation).  All figures stay per step.  Once
+                                   per step: every gradient synchronisation term, the update
+                                   and what it moves (gathered optimizer state, re-replicated
+                                   parameters, offloaded Omega and G, storing offloaded Theta).
+                                   Once per micro-batch: the two all-gathers of gathered
+                                   parameters (Theorem 2's third term), loading and gathering
+                                   offloaded parameters, moving offloaded activations, tensor-
+                                   and pipeline-axis traffic.  A placement whose only traffic
+                                   is gradient synchronisation therefore moves the same bytes
+                                   per step for g times the samples: the paper's "reduced by a
+                                   factor equal to the number of accumulation steps".  Memory
+                                   and the predicates do not change. */
 } ps_space_desc;
 
 /* survivors of a filter: mem <= cap_bytes, host <= host_cap and every bit of

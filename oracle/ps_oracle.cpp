@@ -60,6 +60,8 @@ struct ODesc {  // the design space
   u32 n_n;
   u32 t_enum_max, k_enum_max, tp_max_valid;
   u32 n_act_variants, n_tpa_variants, mode_mask, tp_coll_per_layer;
+  u32 sstar_units;       // 0 or 1: Theorem 1 as stated; 2: overlapped gathers (the proof's note)
+  u32 grad_accum_steps;  // 0 or 1: none; g: micro-batches per step ("Limitations")
 };
 
 struct OFilter {
@@ -144,11 +146,13 @@ ORecord derive_record(const OShape& s) {
 // ---------------------------------------------------------------- one point
 // Theorem 1 on the data axis: persistent and transient elements of a state of
 // E elements whose reconstruction unit is u, under mode pi over D devices.
-void mu_elems(int pi, u64 E, u64 u, u64 D, u64* persistent, u64* transient) {
+// The proof of case S* notes that an implementation which overlaps the gather
+// of the next unit with computation holds two unit buffers: gather_buffers.
+void mu_elems(int pi, u64 E, u64 u, u64 D, u64 gather_buffers, u64* persistent, u64* transient) {
   switch (pi) {
     case R:  *persistent = E;              *transient = 0; break;
     case S:  *persistent = ceil_div(E, D); *transient = 0; break;
-    case SG: *persistent = ceil_div(E, D); *transient = u; break;
+    case SG: *persistent = ceil_div(E, D); *transient = gather_buffers * u; break;
     case M:  *persistent = 0;              *transient = u; break;
     default: *persistent = 0;              *transient = 0; break;  // O
   }
@@ -156,8 +160,12 @@ void mu_elems(int pi, u64 E, u64 u, u64 D, u64* persistent, u64* transient) {
 
 OResult eval_point(const ORecord& m, u64 N, u64 T, u64 K, u64 D, int v, int tau,
                    int pi_theta, int pi_omega, int pi_grad, int pi_act,
-                   u32 tp_max_valid, u32 tp_coll_per_layer, bool axis_form_ok) {
+                   u32 tp_max_valid, u32 tp_coll_per_layer, bool axis_form_ok,
+                   u32 sstar_units = 1, u32 grad_accum_steps = 1) {
   OResult out;
+  // the two extensions: unit buffers of a gathered state, micro-batches per step
+  const u64 nbuf = sstar_units ? sstar_units : 1;
+  const u64 g = grad_accum_steps ? grad_accum_steps : 1;
   // Remark 4: tensor parallelism innermost, pipeline in the middle, data
   // outermost.  Table 2: both model axes shard Theta, Omega and G.
   u64 E1 = ceil_div(m.P, T);        // intra-layer split
@@ -171,27 +179,31 @@ OResult eval_point(const ORecord& m, u64 N, u64 T, u64 K, u64 D, int v, int tau,
 
   u64 p, t;
   out.mem = 0;
-  mu_elems(pi_theta, E2, u2, D, &p, &t); out.mem += (u64)m.w_theta * (p + t);
-  mu_elems(pi_omega, E2, u2, D, &p, &t); out.mem += (u64)m.w_omega * (p + t);
-  mu_elems(pi_grad,  E2, u2, D, &p, &t); out.mem += (u64)m.w_grad  * (p + t);
-  mu_elems(pi_act,   EA, uA, D, &p, &t); out.mem += p + t;   // already bytes
+  mu_elems(pi_theta, E2, u2, D, nbuf, &p, &t); out.mem += (u64)m.w_theta * (p + t);
+  mu_elems(pi_omega, E2, u2, D, nbuf, &p, &t); out.mem += (u64)m.w_omega * (p + t);
+  mu_elems(pi_grad,  E2, u2, D, nbuf, &p, &t); out.mem += (u64)m.w_grad  * (p + t);
+  mu_elems(pi_act,   EA, uA, D, nbuf, &p, &t); out.mem += p + t;   // already bytes
 
   u64 sh = ceil_div(E2, D);       // largest shard of Theta / Omega / G
   u64 x = ring_elems(E2, D);      // ring volume in elements
   u64 xT = x * m.w_theta, xO = x * m.w_omega, xG = x * m.w_grad;
 
-  // Theorem 2: the three priced transitions, nothing else
+  // Theorem 2: the three priced transitions, nothing else.  With gradient
+  // accumulation ("Limitations") a step runs g micro-batches and synchronises
+  // gradients once: the gradient terms stay, and whatever every micro-batch's
+  // forward and backward need is paid g times.  Per micro-batch the gradient
+  // terms are thus divided by g, as the paper says.
   out.comm_paper = 0;
-  if (pi_grad == R) out.comm_paper += 2 * xG;      // all-reduce
-  if (pi_grad == S) out.comm_paper += xG;          // reduce-scatter
-  if (pi_theta == SG) out.comm_paper += 2 * xT;    // gather for forward and backward
+  if (pi_grad == R) out.comm_paper += 2 * xG;          // all-reduce, once per step
+  if (pi_grad == S) out.comm_paper += xG;              // reduce-scatter, once per step
+  if (pi_theta == SG) out.comm_paper += g * 2 * xT;    // gather for forward and backward of every micro-batch
 
   // the update is committed on a shard when Omega's home is a shard
   bool update_on_shard = (pi_omega == S || pi_omega == SG || pi_omega == O);
 
   // traffic of the execution model that Theorem 2 does not price
   u64 ext_data = 0;
-  if (pi_theta == O) ext_data += 2 * xT;                     // gather after each host load
+  if (pi_theta == O) ext_data += g * 2 * xT;                 // gather after each host load, every micro-batch
   if (pi_theta == R && update_on_shard) ext_data += xT;      // re-replicate updated shards
   if (pi_grad == SG) ext_data += 2 * xG;                     // reduce-scatter, then gather
   if (pi_grad == M) ext_data += (update_on_shard ? 1 : 2) * xG;
@@ -200,14 +212,14 @@ OResult eval_point(const ORecord& m, u64 N, u64 T, u64 K, u64 D, int v, int tau,
   u64 layers_per_stage = ceil_div(m.L, K);
   u64 ext_tp = layers_per_stage * tp_coll_per_layer * 2 * ring_elems(m.Sbh, T) * m.w_act;
   u64 ext_pp = (K > 1) ? 2 * ceil_div(m.Sbh, tau == 0 ? T : 1) * m.w_act : 0;
-  out.comm_ext = ext_data + ext_tp + ext_pp;
+  out.comm_ext = ext_data + g * (ext_tp + ext_pp);           // model-axis traffic of every micro-batch
 
   // host-link bytes (mode O): shards live on the hosts
   out.host = 0;
-  if (pi_theta == O) out.host += 3 * sh * m.w_theta;   // load for fwd, load for bwd, store
+  if (pi_theta == O) out.host += (2 * g + 1) * sh * m.w_theta;   // load for fwd and bwd of every micro-batch, one store
   if (pi_omega == O) out.host += 2 * sh * m.w_omega;   // load, store
   if (pi_grad == O)  out.host += 2 * sh * m.w_grad;    // store, load at the update
-  if (pi_act == O)   out.host += 2 * EA;               // store after fwd, load for bwd
+  if (pi_act == O)   out.host += g * 2 * EA;           // store after fwd, load for bwd, every micro-batch
 
   // Theorems 3 and 4 as static predicates over the placement
   bool omega_full = (pi_omega == R) || (D == 1 && (pi_omega == S || pi_omega == SG));
@@ -318,7 +330,7 @@ struct Space {
     Decoded p = decode(idx);
     ORecord rec = derive_record(d->models[p.model]);
     return eval_point(rec, p.N, p.T, p.K, p.D, p.v, p.tau, p.pi[0], p.pi[1], p.pi[2], p.pi[3],
-                      d->tp_max_valid, d->tp_coll_per_layer, true);
+                      d->tp_max_valid, d->tp_coll_per_layer, true, d->sstar_units, d->grad_accum_steps);
   }
 };
 
@@ -490,7 +502,8 @@ void orc_check_composition(const OShape* shape, u32 N, u32 T, u32 K, u32 D, u32 
 // whose toy models have no transformer shape).  rec: P, unit, A0, A1, UA0,
 // UA1, Sbh, L, heads, w_theta, w_omega, w_grad, w_act as 13 u64.
 void orc_eval_record(const u64* rec, u32 N, u32 T, u32 K, u32 D, u32 v, u32 tau, u32 code,
-                     u32 tp_max_valid, u32 tp_coll_per_layer, u64* out5) {
+                     u32 tp_max_valid, u32 tp_coll_per_layer, u32 sstar_units, u32 grad_accum_steps,
+                     u64* out5) {
   ORecord m;
   m.P = rec[0]; m.unit = rec[1]; m.A[0] = rec[2]; m.A[1] = rec[3]; m.UA[0] = rec[4]; m.UA[1] = rec[5];
   m.Sbh = rec[6]; m.L = (u32)rec[7]; m.heads = (u32)rec[8];
@@ -498,7 +511,7 @@ void orc_eval_record(const u64* rec, u32 N, u32 T, u32 K, u32 D, u32 v, u32 tau,
   int pi[4];
   for (int s = 0; s < 4; ++s) { pi[s] = code % 5; code /= 5; }
   OResult r = eval_point(m, N, T, K, D, (int)v, (int)tau, pi[0], pi[1], pi[2], pi[3],
-                         tp_max_valid, tp_coll_per_layer, true);
+                         tp_max_valid, tp_coll_per_layer, true, sstar_units, grad_accum_steps);
   out5[0] = r.mem; out5[1] = r.comm_paper; out5[2] = r.comm_ext; out5[3] = r.host; out5[4] = r.flags;
 }
 

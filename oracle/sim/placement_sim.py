@@ -155,19 +155,21 @@ def adam(omega, grad, t, lr=0.05, b1=0.9, b2=0.999, eps=1e-8):
     return np.stack([master, m, v])
 
 
-def make_problem(units, h, b, D, seed):
+def make_problem(units, h, b, D, seed, accum=1):
+    """xs[j][i], ys[j][i]: micro-batch j of device i (accum micro-batches per step)."""
     rng = np.random.default_rng(seed)
     theta0 = rng.uniform(0.5, 1.5, units * h)
-    xs = [rng.normal(size=(b, h)) for _ in range(D)]
-    ys = [rng.uniform(-0.8, 0.8, size=(b, h)) for _ in range(D)]
+    xs = [[rng.normal(size=(b, h)) for _ in range(D)] for _ in range(accum)]
+    ys = [[rng.uniform(-0.8, 0.8, size=(b, h)) for _ in range(D)] for _ in range(accum)]
     return theta0, xs, ys
 
 
 def run_single(units, h, xs, ys, theta0, steps):
-    """The single-device run on the global batch (Definition 4's yardstick)."""
+    """The single-device run on the global batch (Definition 4's yardstick):
+    all micro-batches of all devices in one batch."""
     model = ToyModel(units, h)
-    x = np.concatenate(xs)
-    y = np.concatenate(ys)
+    x = np.concatenate([xi for xj in xs for xi in xj])
+    y = np.concatenate([yi for yj in ys for yi in yj])
     omega = np.stack([theta0.copy(), np.zeros_like(theta0), np.zeros_like(theta0)])
     theta = theta0.copy()
     traj = []
@@ -183,8 +185,11 @@ def run_single(units, h, xs, ys, theta0, steps):
 class Placed:
     """D devices executing one placement (pi_theta, pi_omega, pi_grad, pi_act)."""
 
-    def __init__(self, units, h, b, D, code, theta0):
+    def __init__(self, units, h, b, D, code, theta0, gather_buffers=1):
         self.model = ToyModel(units, h)
+        # unit buffers a gathered state holds: 2 when the next unit is fetched while
+        # the current one is in use (only possible with at least two units)
+        self.nbuf = min(gather_buffers, units)
         self.units, self.h, self.b, self.D = units, h, b, D
         self.pT, self.pO, self.pG, self.pA = code % 5, (code // 5) % 5, (code // 25) % 5, code // 125
         self.P = units * h
@@ -244,7 +249,7 @@ class Placed:
                     pieces.append(shards[i][s0 - lo:s1 - lo] if s1 > s0 else np.zeros(0))
                 got = ring_all_gather(pieces, W_THETA, books, None, sent)
                 if self.pT == SG:
-                    books.unit_buffer("theta", h * W_THETA)
+                    books.unit_buffer("theta", self.nbuf * h * W_THETA)
                 for i in range(D):
                     fulls[i][a:b_] = got[i]
             books.phases.append(("gather theta " + tag, sent))
@@ -263,6 +268,19 @@ class Placed:
         return out
 
     def step(self, t, xs, ys, books):
+        """One optimizer step over len(xs) micro-batches per device: forward and
+        backward run per micro-batch, the local gradients add up (that buffer is
+        not a placed state), everything from (4) on happens once."""
+        D, P = self.D, self.P
+        accum = len(xs)
+        local = [np.zeros(P) for _ in range(D)]
+        for j in range(accum):
+            mb = self.micro_batch(xs[j], ys[j], books)
+            for i in range(D):
+                local[i] += mb[i] / accum
+        self.finish_step(t, local, books)
+
+    def micro_batch(self, xs, ys, books):
         D, P, h, b = self.D, self.P, self.h, self.b
         model = self.model
         # (1) forward
@@ -293,14 +311,17 @@ class Placed:
                 # gather from the peers: their slices belong to other samples
                 sent = np.zeros(D, dtype=np.int64)
                 got = ring_all_gather(slices, 1, books, None, sent)
-                books.unit_buffer("act", b * h)
+                books.unit_buffer("act", self.nbuf * b * h)
                 kept = [g.reshape(acts[0].shape) for g in got]
         # (3) Theta again for backward
         th_b = self.theta_for_compute(books, "bwd")
         if self.pA == M:
             books.unit_buffer("act", b * h)
             kept = [model.forward(th_b[i], xs[i])[0] for i in range(D)]   # recomputed
-        local = [model.backward(th_b[i], kept[i], ys[i]) for i in range(D)]
+        return [model.backward(th_b[i], kept[i], ys[i]) for i in range(D)]
+
+    def finish_step(self, t, local, books):
+        D, P, h, b = self.D, self.P, self.h, self.b
         # (4) synchronise / deliver gradients (mean over the D replicas)
         grad = [np.zeros(P) for _ in range(D)]     # what the update will read
         cut = self.cut
@@ -331,7 +352,7 @@ class Placed:
                     s0, s1 = max(a, cut[i]), min(b_, cut[i + 1])
                     pieces.append(red[i][s0 - cut[i]:s1 - cut[i]] if s1 > s0 else np.zeros(0))
                 got = ring_all_gather(pieces, W_GRAD, books, None, sent)
-                books.unit_buffer("grad", h * W_GRAD)
+                books.unit_buffer("grad", self.nbuf * h * W_GRAD)
                 for i in range(D):
                     grad[i][a:b_] = got[i] / D
             books.phases.append(("grad all-gather before use", sent))
@@ -383,7 +404,7 @@ class Placed:
                     pieces.append(self.omega_gpu[i][0, s0 - cut[i]:s1 - cut[i]] if s1 > s0 else np.zeros(0))
                 for _row in range(3):          # master, m, v: 3 x 4 bytes per element
                     ring_all_gather(pieces, W_OMEGA // 3, books, None, sent)
-                books.unit_buffer("omega", h * W_OMEGA)
+                books.unit_buffer("omega", self.nbuf * h * W_OMEGA)
             books.phases.append(("gather omega", sent))
             for i in range(D):
                 lo, hi = cut[i], cut[i + 1]
@@ -433,13 +454,15 @@ class Placed:
         return thetas, omegas
 
 
-def simulate(units, h, b, D, code, steps=3, seed=0):
-    """Run `steps` steps; returns dict(match, mem, comm, host) where match says
-    whether every step's reassembled Theta and Omega equal the single-device
-    run to 1e-12 relative, and the byte figures are those of the last step."""
-    theta0, xs, ys = make_problem(units, h, b, D, seed)
+def simulate(units, h, b, D, code, steps=3, seed=0, accum=1, gather_buffers=1):
+    """Run `steps` steps of `accum` micro-batches each; returns dict(match, mem,
+    comm, host) where match says whether every step's reassembled Theta and Omega
+    equal the single-device run to 1e-12 relative, and the byte figures are those
+    of the last step.  gather_buffers = 2: a gathered state prefetches the next
+    unit while the current one is in use."""
+    theta0, xs, ys = make_problem(units, h, b, D, seed, accum)
     ref = run_single(units, h, xs, ys, theta0, steps)
-    job = Placed(units, h, b, D, code, theta0)
+    job = Placed(units, h, b, D, code, theta0, gather_buffers)
     match = True
     books = None
     for t in range(1, steps + 1):

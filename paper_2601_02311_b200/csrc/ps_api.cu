@@ -35,7 +35,7 @@ struct DeviceGuard {
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 // the supported ranges of a shape (the same limits the derivation kernel checks)
-bool shape_in_range(const ps_model_shape& s, u32 tp_coll) {
+bool shape_in_range(const ps_model_shape& s, u32 tp_coll, u32 accum = 1) {
   if (s.layers < 1 || s.layers > (1u << 10)) return false;
   if (s.hidden < 1 || s.hidden > (1u << 16)) return false;
   if (s.heads < 1 || s.heads > (1u << 16)) return false;
@@ -54,9 +54,12 @@ bool shape_in_range(const ps_model_shape& s, u32 tp_coll) {
   if (s.act_enabled) {
     const u128 A0 = L * (34 * S * b * H + 5 * a * S * S * b);
     if (A0 > ((u128)1 << 58)) return false;
+    if (2 * A0 * accum > ((u128)1 << 62)) return false;        // host bytes of offloaded activations
   } else if (5 * a * S * S * b > ((u128)1 << 58)) {
     return false;
   }
+  // tensor- and pipeline-axis bytes per step
+  if ((L * 2 * tp_coll * s.w_act + 2 * s.w_act) * S * b * H * accum > ((u128)1 << 62)) return false;
   return true;
 }
 
@@ -190,8 +193,10 @@ int ps_space_create(ps_ctx* ctx, const ps_space_desc* desc, ps_space** out) {
   if (desc->tp_coll_per_layer > 64) return PS_E_RANGE;
   for (u32 i = 0; i < desc->n_n; ++i)
     if (desc->n_values[i] < 1 || desc->n_values[i] > (1u << 24)) return PS_E_RANGE;
+  if (desc->sstar_units > 2 || desc->grad_accum_steps > 64) return PS_E_RANGE;
+  const u32 accum = desc->grad_accum_steps ? desc->grad_accum_steps : 1;
   for (u32 i = 0; i < desc->n_models; ++i)
-    if (!shape_in_range(desc->models[i], desc->tp_coll_per_layer)) return PS_E_RANGE;
+    if (!shape_in_range(desc->models[i], desc->tp_coll_per_layer, accum)) return PS_E_RANGE;
 
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return PS_E_CUDA;
@@ -241,6 +246,8 @@ int ps_space_create(ps_ctx* ctx, const ps_space_desc* desc, ps_space** out) {
   d.n_codes = d.n3 * nm;
   d.tp_max_valid = desc->tp_max_valid;
   d.tp_coll = desc->tp_coll_per_layer;
+  d.sstar_units = desc->sstar_units ? desc->sstar_units : 1;
+  d.accum = accum;
   const u64 ppm = (u64)d.n_facts * d.nvt * d.n_codes;
   if (ppm >= ((u64)1 << 32)) { delete sp; return PS_E_RANGE; }
   d.ppm = ppm;
@@ -264,7 +271,7 @@ int ps_space_set_models(ps_space* sp, const ps_model_shape* models, uint32_t n_m
   if (!sp || !models) return PS_E_NULLPTR;
   if (n_models != sp->dev.n_models) return PS_E_RANGE;
   for (u32 i = 0; i < n_models; ++i)
-    if (!shape_in_range(models[i], sp->dev.tp_coll)) return PS_E_RANGE;
+    if (!shape_in_range(models[i], sp->dev.tp_coll, sp->dev.accum)) return PS_E_RANGE;
   ps_ctx* ctx = sp->ctx;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return PS_E_CUDA;

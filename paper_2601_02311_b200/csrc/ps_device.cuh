@@ -43,6 +43,8 @@ struct SpaceDev {
   u32 n_codes;        // nm^4
   u32 n3;             // nm^3
   u32 tp_max_valid, tp_coll;
+  u32 sstar_units;    // unit buffers a gathered (S*) state holds at a time: 1, or 2 when gathers overlap computation
+  u32 accum;          // micro-batches per step (gradient accumulation), >= 1
 };
 
 enum : u32 {
@@ -173,19 +175,23 @@ __device__ __forceinline__ ActBase act_base_pow2(const ModelRec& r, const Pow2& 
 
 // tensor-axis and pipeline-axis traffic per step (not priced by Theorem 2):
 // per layer of a stage, tp_coll all-reduces of a boundary tensor over T
-// devices; one boundary tensor forward and one backward between stages
+// devices; one boundary tensor forward and one backward between stages; all of
+// it once per micro-batch (accum micro-batches per step)
 __device__ __forceinline__ u64 model_axis_traffic(const ModelRec& r, const Fact& f,
-                                                  const UnitBase& b, u32 tau, u32 tp_coll) {
+                                                  const UnitBase& b, u32 tau, u32 tp_coll,
+                                                  u32 accum = 1) {
   const u32 per_elem = 2 * tp_coll * r.wA;                 // <= 2 * 64 * 16
   const u64 tp = b.tp_x * (u64)(b.lps * per_elem);         // lps <= 2^10
   const u64 pp = (f.K > 1) ? (tau == 0 ? b.sbh_t : r.Sbh) * (u64)(2 * r.wA) : 0;
-  return tp + pp;
+  return (tp + pp) * accum;
 }
 
-// Theorem 1: persistent plus transient elements of a state under mode pi
-__device__ __forceinline__ u64 mu_elems(u32 pi, u64 full, u64 shard, u64 unit) {
+// Theorem 1: persistent plus transient elements of a state under mode pi.  A
+// gathered state (S*) holds sstar_units unit buffers: one, or two when the next
+// unit is gathered while the current one is in use (the theorem's proof, case S*).
+__device__ __forceinline__ u64 mu_elems(u32 pi, u64 full, u64 shard, u64 unit, u32 sstar_units = 1) {
   u64 p = (pi == PS_MODE_R) ? full : (in_set(SET_SHARDLIKE, pi) ? shard : 0);
-  u64 t = in_set(SET_TRANSIENT, pi) ? unit : 0;
+  u64 t = (pi == PS_MODE_SG) ? unit * sstar_units : (pi == PS_MODE_M ? unit : 0);
   return p + t;
 }
 
@@ -222,29 +228,35 @@ __device__ __forceinline__ u32 point_flags(u32 th, u32 om, u32 gr, u32 ac, bool 
 // The whole evaluation of one point, with nothing hoisted.  Used where single
 // points are needed (ps_check_composition, re-deriving host bytes and flags of
 // the few entries a sweep emits).
+// sstar_units: unit buffers of a gathered state; accum: micro-batches per step --
+// what happens once per micro-batch (gathering Theta for forward and backward,
+// loading offloaded Theta, moving activations to the host and back, tensor- and
+// pipeline-axis traffic) is counted accum times, what happens once per step
+// (synchronising gradients, the update and what it moves) once.
 __device__ __forceinline__ PointOut eval_point(const ModelRec& r, const Fact& f, u32 v, u32 tau,
                                                u32 th, u32 om, u32 gr, u32 ac, u32 tp_max_valid,
-                                               u32 tp_coll, bool axis_form) {
+                                               u32 tp_coll, bool axis_form, u32 sstar_units = 1,
+                                               u32 accum = 1) {
   UnitBase b = unit_base(r, f, tp_max_valid, axis_form);
   ActBase a = act_base(r, f, v, tau);
   PointOut o;
-  o.mem = r.wT * mu_elems(th, b.E2, b.sh, b.u) + r.wO * mu_elems(om, b.E2, b.sh, b.u) +
-          r.wG * mu_elems(gr, b.E2, b.sh, b.u) + mu_elems(ac, a.EA, a.shA, a.uA);
+  o.mem = r.wT * mu_elems(th, b.E2, b.sh, b.u, sstar_units) + r.wO * mu_elems(om, b.E2, b.sh, b.u, sstar_units) +
+          r.wG * mu_elems(gr, b.E2, b.sh, b.u, sstar_units) + mu_elems(ac, a.EA, a.shA, a.uA, sstar_units);
   u64 xT = b.x * r.wT, xO = b.x * r.wO, xG = b.x * r.wG;
   // Theorem 2
   o.comm_paper = (gr == PS_MODE_R ? 2 * xG : 0) + (gr == PS_MODE_S ? xG : 0) +
-                 (th == PS_MODE_SG ? 2 * xT : 0);
+                 (th == PS_MODE_SG ? 2 * xT * accum : 0);
   bool on_shard = in_set(SET_UPDATE_ON_SHARD, om);
   u64 ext = 0;
-  if (th == PS_MODE_O) ext += 2 * xT;
+  if (th == PS_MODE_O) ext += 2 * xT * accum;
   if (th == PS_MODE_R && on_shard) ext += xT;
   if (gr == PS_MODE_SG) ext += 2 * xG;
   if (gr == PS_MODE_M) ext += on_shard ? xG : 2 * xG;
   if (gr == PS_MODE_O) ext += xG;
   if (om == PS_MODE_SG) ext += xO;
-  o.comm_ext = ext + model_axis_traffic(r, f, b, tau, tp_coll);
-  o.host = (th == PS_MODE_O ? 3 * b.sh * r.wT : 0) + (om == PS_MODE_O ? 2 * b.sh * r.wO : 0) +
-           (gr == PS_MODE_O ? 2 * b.sh * r.wG : 0) + (ac == PS_MODE_O ? 2 * a.EA : 0);
+  o.comm_ext = ext + model_axis_traffic(r, f, b, tau, tp_coll, accum);
+  o.host = (th == PS_MODE_O ? (2 * accum + 1) * b.sh * r.wT : 0) + (om == PS_MODE_O ? 2 * b.sh * r.wO : 0) +
+           (gr == PS_MODE_O ? 2 * b.sh * r.wG : 0) + (ac == PS_MODE_O ? 2 * a.EA * accum : 0);
   o.flags = point_flags(th, om, gr, ac, b.d1, b.cv, ext == 0);
   return o;
 }

@@ -185,22 +185,24 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
         for (int s = 0; s < 3; ++s) {        // Theorem 1: R holds E, S and S* a shard, S* and M a unit
           if (modes[s] == PS_MODE_R) ca += width[s];
           if (in_set(SET_SHARDLIKE, modes[s])) cb += width[s];
-          if (in_set(SET_TRANSIENT, modes[s])) cc += width[s];
+          if (modes[s] == PS_MODE_SG) cc += width[s] * sp.sstar_units;   // one or two unit buffers
+          if (modes[s] == PS_MODE_M) cc += width[s];
         }
         ka[r] = ca; kb[r] = cb; kc[r] = cc;
-        // Theorem 2: all-reduce (2x) or reduce-scatter (1x) of G, two all-gathers of gathered Theta
-        kp[r] = (th[r] == PS_MODE_SG ? 2 * rec.wT : 0) +
+        // Theorem 2: all-reduce (2x) or reduce-scatter (1x) of G, two all-gathers of gathered
+        // Theta for every micro-batch
+        kp[r] = (th[r] == PS_MODE_SG ? 2 * sp.accum * rec.wT : 0) +
                 (gr[r] == PS_MODE_R ? 2 * rec.wG : (gr[r] == PS_MODE_S ? rec.wG : 0));
         // what the execution model moves beyond that
         u32 e = 0;
-        if (th[r] == PS_MODE_O) e += 2 * rec.wT;
+        if (th[r] == PS_MODE_O) e += 2 * sp.accum * rec.wT;
         if (th[r] == PS_MODE_R && on_shard) e += rec.wT;
         if (om[r] == PS_MODE_SG) e += rec.wO;
         if (gr[r] == PS_MODE_SG) e += 2 * rec.wG;
         if (gr[r] == PS_MODE_M) e += (on_shard ? 1 : 2) * rec.wG;
         if (gr[r] == PS_MODE_O) e += rec.wG;
         ke[r] = e;
-        kh[r] = (th[r] == PS_MODE_O ? 3 * rec.wT : 0) + (om[r] == PS_MODE_O ? 2 * rec.wO : 0) +
+        kh[r] = (th[r] == PS_MODE_O ? (2 * sp.accum + 1) * rec.wT : 0) + (om[r] == PS_MODE_O ? 2 * rec.wO : 0) +
                 (gr[r] == PS_MODE_O ? 2 * rec.wG : 0);
         st_many[r] = triple_static(th[r], om[r], gr[r], false);
         st_one[r] = triple_static(th[r], om[r], gr[r], true);
@@ -213,11 +215,11 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
     const UnitBase ub = p2.all ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
                                : unit_base(rec, f, sp.tp_max_valid, true);
     const ActBase ab = p2.all ? act_base_pow2(rec, p2, v, tau) : act_base(rec, f, v, tau);
-    const u64 c_axis = model_axis_traffic(rec, f, ub, tau, sp.tp_coll);
+    const u64 c_axis = model_axis_traffic(rec, f, ub, tau, sp.tp_coll, sp.accum);
     u64 act[NM];
 #pragma unroll
-    for (int d = 0; d < NM; ++d) act[d] = mu_elems(digit_mode(sp.modemap, d), ab.EA, ab.shA, ab.uA);
-    const u64 act_host = 2 * ab.EA;
+    for (int d = 0; d < NM; ++d) act[d] = mu_elems(digit_mode(sp.modemap, d), ab.EA, ab.shA, ab.uA, sp.sstar_units);
+    const u64 act_host = 2 * ab.EA * sp.accum;
     const u32 avail = ub.d1 ? ((1u << NM) - 1u) : own;     // digits with PS_F_ACT_AVAIL
 
     u64 mem3[R], paper3[R], ext3[R], host3[R];

@@ -378,21 +378,22 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
     for (int st = 0; st < 3; ++st) {
       if (modes[st] == PS_MODE_R) a += width[st];
       if (in_set(SET_SHARDLIKE, modes[st])) b += width[st];
-      if (in_set(SET_TRANSIENT, modes[st])) c += width[st];
+      if (modes[st] == PS_MODE_SG) c += width[st] * sp.sstar_units;   // one or two unit buffers
+      if (modes[st] == PS_MODE_M) c += width[st];
     }
     // Theorem 2: all-reduce of replicated gradients, reduce-scatter of sharded
-    // ones, two all-gathers of gathered parameters
-    u32 ct = (th == PS_MODE_SG) ? 2 : 0, co = 0;
+    // ones, two all-gathers of gathered parameters for each micro-batch
+    u32 ct = (th == PS_MODE_SG) ? 2 * sp.accum : 0, co = 0;
     u32 cg = (gr == PS_MODE_R) ? 2 : (gr == PS_MODE_S ? 1 : 0);
     if (ext_in_objective) {                  // traffic the theorem does not price
-      if (th == PS_MODE_O) ct += 2;
+      if (th == PS_MODE_O) ct += 2 * sp.accum;
       if (th == PS_MODE_R && on_shard) ct += 1;
       if (om == PS_MODE_SG) co = 1;
       if (gr == PS_MODE_SG) cg += 2;
       if (gr == PS_MODE_M) cg += on_shard ? 1 : 2;
       if (gr == PS_MODE_O) cg += 1;
     }
-    if (th == PS_MODE_O) h += 3 * rec.wT;
+    if (th == PS_MODE_O) h += (2 * sp.accum + 1) * rec.wT;
     if (om == PS_MODE_O) h += 2 * rec.wO;
     if (gr == PS_MODE_O) h += 2 * rec.wG;
     t_local[r] = tt;
@@ -435,16 +436,16 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
         ab.uA = tl_tau == 0 ? div_ceil(tl_UA, f.T) : tl_UA;
         ab.shA = div_ceil(ab.EA, f.D);
       }
-      const u64 am = mu_elems(tl_mode, ab.EA, ab.shA, ab.uA);
+      const u64 am = mu_elems(tl_mode, ab.EA, ab.shA, ab.uA, sp.sstar_units);
       if (tl_mine) {
         const u64 bound = am < cap_x ? cap_x - am : 0;
         tb.bound[tl_d][tl_vt] = bound;
         tb.bound_f64[tl_d][tl_vt] = (double)bound;
         tb.act[tl_vt][tl_d] = am;
         if (tl_d == 0) {
-          const u64 ah = 2 * ab.EA;                            // offload after fwd, reload for bwd
+          const u64 ah = 2 * ab.EA * sp.accum;                 // offload after fwd, reload for bwd, per micro-batch
           tb.host_bound[tl_vt] = ah < host_x ? host_x - ah : 0;
-          tb.c_axis[tl_vt] = ext_in_objective ? model_axis_traffic(rec, f, ub, tl_tau, sp.tp_coll) : 0;
+          tb.c_axis[tl_vt] = ext_in_objective ? model_axis_traffic(rec, f, ub, tl_tau, sp.tp_coll, sp.accum) : 0;
         }
       } else if (tl_vt < 4) {
         tb.bound[tl_d][tl_vt] = 0;
@@ -478,7 +479,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
     // that small (uniform test) the compares run on the fp64 pipe, which is idle
     // otherwise, and only the counting stays on the integer pipe.
     const bool small = cap_x < ((u64)1 << 53) &&
-                       (u64)(rec.wT + rec.wO + rec.wG) * (ub.E2 + ub.u) < ((u64)1 << 53);
+                       (u64)(rec.wT + rec.wO + rec.wG) * (ub.E2 + 2 * ub.u) < ((u64)1 << 53);
     if (small) {
       double mem_f64[R];
       float pass_f32[R];
@@ -563,19 +564,8 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
     // ---- reduction pass, only if some survivor of this warp can matter
     bool matters = false;
     if (KIND == PS_REDUCE_PARETO) {
-      // a triple's survivors hold at least the triple's own bytes and send at least
-      // its own volume plus the cheapest variant's axis traffic: if a point the
-      // block has already kept beats that bound strictly in bytes (a lower bucket
-      // of the coarse staircase) with no more communication, none of them can be
-      // on the frontier
-      const u64 least_axis = tb.c_axis[0];   // tau = 0 sends the smaller boundary tensor; v does not matter
 #pragma unroll
-      for (int r = 0; r < R; ++r) {
-        if (n_pass[r] != 0) {
-          const int bucket = stair_bucket(mem3[r]);
-          if (bucket == 0 || sh.stair[bucket - 1] > comm3[r] + least_axis) matters = true;
-        }
-      }
+      for (int r = 0; r < R; ++r) matters = matters || n_pass[r] != 0;
     } else {
       const u64 comm_limit = min(threshold.a, (u64)sh.block_comm_limit);
       const u64 least_axis = tb.c_axis[0];   // tau = 0 sends the smaller boundary tensor; v does not matter
@@ -940,7 +930,8 @@ __global__ void __launch_bounds__(MERGE_THREADS) k_sweep_merge(SpaceDev sp, Merg
         const Fact f = sp.facts[lp.unit];
         const PointOut po = eval_point(rec, f, lp.v, lp.tau, digit_mode(sp.modemap, lp.dth),
                                        digit_mode(sp.modemap, lp.dom), digit_mode(sp.modemap, lp.dgr),
-                                       digit_mode(sp.modemap, lp.dac), sp.tp_max_valid, sp.tp_coll, true);
+                                       digit_mode(sp.modemap, lp.dac), sp.tp_max_valid, sp.tp_coll, true,
+                                       sp.sstar_units, sp.accum);
         const u64 comm = args.comm_kind == PS_COMM_PAPER ? po.comm_paper : po.comm_paper + po.comm_ext;
         const u64 list_mem = (KIND == PS_REDUCE_PARETO) ? sh.a[p] : sh.b[p];
         const u64 list_comm = (KIND == PS_REDUCE_PARETO) ? sh.b[p] : sh.a[p];

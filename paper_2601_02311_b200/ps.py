@@ -55,7 +55,8 @@ class _SpaceDesc(C.Structure):
                 ("t_enum_max", C.c_uint32), ("k_enum_max", C.c_uint32),
                 ("tp_max_valid", C.c_uint32), ("n_act_variants", C.c_uint32),
                 ("n_tpa_variants", C.c_uint32), ("mode_mask", C.c_uint32),
-                ("tp_coll_per_layer", C.c_uint32)]
+                ("tp_coll_per_layer", C.c_uint32), ("sstar_units", C.c_uint32),
+                ("grad_accum_steps", C.c_uint32)]
 
 
 class _Filter(C.Structure):
@@ -203,7 +204,8 @@ class Space:
         desc = _SpaceDesc(models.ctypes.data, len(models), n_values.ctypes.data, len(n_values),
                           space["t_enum_max"], space["k_enum_max"], space["tp_max_valid"],
                           space["n_act_variants"], space["n_tpa_variants"], space["mode_mask"],
-                          space["tp_coll_per_layer"])
+                          space["tp_coll_per_layer"], space.get("sstar_units", 1),
+                          space.get("grad_accum_steps", 1))
         handle = C.c_void_p()
         _check(_lib.ps_space_create(ctx._h, C.byref(desc), C.byref(handle)), "ps_space_create")
         self._h = handle
