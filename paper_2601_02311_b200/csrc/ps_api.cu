@@ -89,10 +89,12 @@ int enqueue_status_copy(ps_ctx* ctx) {
 }
 
 u32 pick_chunks(const ps_ctx* ctx, const ps_space* sp, int kind) {
-  // enough blocks for about three waves of the resident blocks of every SM; every
-  // extra block of a model builds its lists from scratch and ends with a merge,
-  // so no more than that
-  const u64 target = (u64)ctx->sm_count * sweep_blocks_per_sm(kind) * 3;
+  // Blocks per model.  Every extra block of a model builds its lists from
+  // scratch -- a top-k block takes every survivor as a candidate until it has
+  // found its own first k -- so only as many as fill the GPU once (top-k) or
+  // twice (Pareto, whose blocks are fewer and longer).
+  const u64 waves = kind == PS_REDUCE_PARETO ? 2 : 1;
+  const u64 target = (u64)ctx->sm_count * sweep_blocks_per_sm(kind) * waves;
   u64 c = (target + sp->dev.n_models - 1) / sp->dev.n_models;
   if (c < 1) c = 1;
   if (c > SWEEP_MAX_CHUNKS) c = SWEEP_MAX_CHUNKS;
