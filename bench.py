@@ -55,8 +55,8 @@ BYTES_PER_POINT_MATERIALISE = 36
 # DRAM traffic of one launch from the ncu captures summarised under profiles/
 # (k_sweep<top-k> on the full stress configuration; k_eval<materialise> per point
 # of a 2^25-point window, where traffic grows in proportion to the points)
-NCU_SWEEP_DRAM_BYTES = 499_968
-NCU_MATERIALISE_DRAM_BYTES_PER_POINT = 1_268_337_000 / (1 << 25)
+NCU_SWEEP_DRAM_BYTES = 6_557_696
+NCU_MATERIALISE_DRAM_BYTES_PER_POINT = 1_400_919_560 / (1 << 25)
 
 
 def parse_args():
@@ -478,7 +478,7 @@ def run_ours(args):
                          "frac": alu_achieved / (int_peak / 1e12),
                          "traffic": NCU_SWEEP_DRAM_BYTES if args.workload == "C4" and args.models is None else None,
                          "ops_per_point": ALG_OPS_PER_POINT_SWEEP,
-                         "alu_pipe_active_ncu": 0.51, "issue_active_ncu": 0.65,
+                         "alu_pipe_active_ncu": 0.585, "issue_active_ncu": 0.752,
                          "peak_source": "k_int_peak (add+xor chains on both integer pipes) measured in this run"},
             "roofline_hbm": {"bound": "hbm", "kernel": "k_eval<materialise>", "achieved": mat_gbs,
                              "peak": hbm_peak, "unit": "GB/s", "frac": mat_gbs / hbm_peak,

@@ -77,20 +77,11 @@ __global__ void k_check_point(const ModelRec* rec, Fact f, u32 v, u32 tau, u32 c
   *out = e;
 }
 
-// Algorithm 1, one query per thread.  Thresholds are rationals; the comparisons
-// are carried out exactly in 128-bit integers.
-__global__ void __launch_bounds__(256) k_select(const ps_select_query* __restrict__ q, u64 n,
-                                                u32 head_num, u32 head_den, u32 layer_num,
-                                                u32 layer_den, u32 tp_degree,
-                                                ps_select_result* __restrict__ out) {
-  const u64 i = (u64)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  ps_select_query s;
-  {
-    const uint4* src = reinterpret_cast<const uint4*>(q + i);
-    uint4* dst = reinterpret_cast<uint4*>(&s);
-    dst[0] = __ldg(src); dst[1] = __ldg(src + 1);
-  }
+// Algorithm 1 for one query.  Thresholds are rationals; the comparisons are
+// carried out exactly in 128-bit integers.
+__device__ __forceinline__ ps_select_result select_one(const ps_select_query& s, u32 head_num,
+                                                       u32 head_den, u32 layer_num, u32 layer_den,
+                                                       u32 tp_degree) {
   typedef unsigned __int128 u128;
   const u32 wsum = (u32)s.w_param + s.w_grad + s.w_opt;
   const u128 m_model = (u128)wsum * s.param_elems;
@@ -110,19 +101,64 @@ __global__ void __launch_bounds__(256) k_select(const ps_select_query* __restric
       branch = 3;
     }
   }
-  ModelRec r;
-  r.P = s.param_elems; r.unit = s.layer_elems; r.A[0] = r.A[1] = r.UA[0] = r.UA[1] = 0;
-  r.Sbh = 1; r.L = 1; r.heads = T;
-  r.wT = s.w_param; r.wO = s.w_opt; r.wG = s.w_grad; r.wA = 1; r.ok = 1;
-  const Fact f{s.n_devices, T, 1, s.n_devices / T};
-  const PointOut p = eval_point(r, f, 0, 0, code % 5, (code / 5) % 5, (code / 25) % 5, (code / 125) % 5,
-                                0xffffffffu, 0, true);
+  // Theorem 1 and Theorem 2 for the choice, written out for the two specifications
+  // the algorithm can return (no activations, no pipeline axis): with E = ceil(P / T)
+  // elements per tensor rank over D = N / T replicas,
+  //   data parallel (R,R,R,R), T = 1:  bytes (w_T + w_O + w_G) P,  volume 2 x w_G
+  //   ZeRO-3 (S*,S,S,R):               bytes (w_T + w_O + w_G) ceil(E / D) + w_T ceil(unit / T),
+  //                                    volume x w_G + 2 x w_T
+  // where x = E - floor(E / D) is the ring volume in elements (Section 2.3).
+  const u32 D = s.n_devices / T;
+  const u64 E = div_ceil(s.param_elems, T);
+  const u64 quot = div_floor(E, D);
+  const u64 x = E - quot;
+  u64 mem, comm;
+  if (code == 0) {
+    mem = (u64)wsum * E;
+    comm = 2 * x * s.w_grad;
+  } else {
+    const u64 shard = quot + ((quot * D != E) ? 1 : 0);
+    mem = (u64)wsum * shard + (u64)s.w_param * div_ceil(s.layer_elems, T);
+    comm = x * s.w_grad + 2 * x * s.w_param;
+  }
   ps_select_result o;
-  o.mem = p.mem; o.comm = p.comm_paper; o.branch = branch; o.T = T; o.code_dp = code;
-  o.flags = p.mem <= s.device_bytes ? PS_F_FEASIBLE : 0;
-  uint4* dst = reinterpret_cast<uint4*>(out + i);
-  const uint4* src = reinterpret_cast<const uint4*>(&o);
-  dst[0] = src[0]; dst[1] = src[1];
+  o.mem = mem; o.comm = comm; o.branch = branch; o.T = T; o.code_dp = code;
+  o.flags = mem <= s.device_bytes ? PS_F_FEASIBLE : 0;
+  return o;
+}
+
+// Two queries per thread, SELECT_THREADS apart, so that four 16-byte loads are in
+// flight per thread before any arithmetic: the kernel streams 64 bytes per query.
+constexpr int SELECT_THREADS = 256;
+__global__ void __launch_bounds__(SELECT_THREADS) k_select(const ps_select_query* __restrict__ q, u64 n,
+                                                           u32 head_num, u32 head_den, u32 layer_num,
+                                                           u32 layer_den, u32 tp_degree,
+                                                           ps_select_result* __restrict__ out) {
+  const u64 i0 = (u64)blockIdx.x * (2 * SELECT_THREADS) + threadIdx.x;
+  const u64 i1 = i0 + SELECT_THREADS;
+  ps_select_query s0, s1;
+  if (i0 < n) {
+    const uint4* src = reinterpret_cast<const uint4*>(q + i0);
+    uint4* dst = reinterpret_cast<uint4*>(&s0);
+    dst[0] = __ldg(src); dst[1] = __ldg(src + 1);
+  }
+  if (i1 < n) {
+    const uint4* src = reinterpret_cast<const uint4*>(q + i1);
+    uint4* dst = reinterpret_cast<uint4*>(&s1);
+    dst[0] = __ldg(src); dst[1] = __ldg(src + 1);
+  }
+  if (i0 < n) {
+    const ps_select_result o = select_one(s0, head_num, head_den, layer_num, layer_den, tp_degree);
+    uint4* dst = reinterpret_cast<uint4*>(out + i0);
+    const uint4* src = reinterpret_cast<const uint4*>(&o);
+    dst[0] = src[0]; dst[1] = src[1];
+  }
+  if (i1 < n) {
+    const ps_select_result o = select_one(s1, head_num, head_den, layer_num, layer_den, tp_degree);
+    uint4* dst = reinterpret_cast<uint4*>(out + i1);
+    const uint4* src = reinterpret_cast<const uint4*>(&o);
+    dst[0] = src[0]; dst[1] = src[1];
+  }
 }
 
 // 8 independent chains per thread; each round applies to every chain an add
@@ -165,8 +201,9 @@ cudaError_t launch_check_point(const ModelRec* d_rec, Fact f, u32 v, u32 tau, u3
 
 cudaError_t launch_select(const ps_select_query* d_q, u64 n, u32 head_num, u32 head_den, u32 layer_num,
                           u32 layer_den, u32 tp_degree, ps_select_result* d_out, cudaStream_t stream) {
-  k_select<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(d_q, n, head_num, head_den, layer_num, layer_den,
-                                                             tp_degree, d_out);
+  const u64 per_block = 2 * SELECT_THREADS;
+  k_select<<<(unsigned)((n + per_block - 1) / per_block), SELECT_THREADS, 0, stream>>>(
+      d_q, n, head_num, head_den, layer_num, layer_den, tp_degree, d_out);
   return cudaGetLastError();
 }
 
