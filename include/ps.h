@@ -21,7 +21,9 @@
  *               composition validity (Theorems 6-7, Proposition 1, Remark 4)
  *               and their reasons.
  *
- * There is no floating point anywhere.  Shards are element-granular with the
+ * No result is ever rounded: every figure is an exact integer (a sweep compares
+ * on the fp64 pipe only where all numbers of a factorisation are below 2^53,
+ * which doubles hold exactly).  Shards are element-granular with the
  * boundaries of Definition 1 eq. (2); the per-device figure is the largest
  * shard, ceil(E/n); a ring reduce-scatter or all-gather (Section 2.3) moves
  * E - floor(E/n) elements on its busiest device; an all-reduce twice that.
