@@ -377,6 +377,7 @@ int ps_eval_batch(ps_ctx* ctx, const ps_space* sp, uint64_t first, uint64_t coun
     if (rc != PS_OK) return rc;
     a.tile_count = static_cast<u32*>(ctx->scratch);
     a.tile_offset = reinterpret_cast<u64*>(static_cast<char*>(ctx->scratch) + off_bytes);
+    eval_plan_runs(a);
     CUDA_OK(launch_eval_count(sp->dev, a, ctx->stream));
     CUDA_OK(launch_tile_scan(a, ctx->stream));
     CUDA_OK(launch_eval_write(sp->dev, a, ctx->stream));

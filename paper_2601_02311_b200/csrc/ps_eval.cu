@@ -16,10 +16,13 @@
 // (shared -> global, asynchronous), so the warp computes the next array while
 // the previous one drains.
 //
-// Compaction is count -> scan -> write: the count pass stores the survivors of
-// each group, a single-block scan turns them into offsets, the write pass
-// evaluates again and places survivors with ballot/popc prefix sums.  Output
-// order is the index order, so the result is unique.
+// Compaction is count -> scan -> write: the count pass (one warp per run of up to
+// 32 consecutive groups) stores the survivors of each group and of each run, a
+// single-block scan turns the runs' totals into offsets, the write pass skips
+// the groups without survivors, evaluates the others again and places their
+// survivors with ballot/popc prefix sums; a group's offset is its run's plus the
+// counts of the run's earlier groups.  Output order is the index order, so the
+// result is unique.
 #include "ps_device.cuh"
 #include "ps_internal.h"
 
@@ -28,14 +31,19 @@ namespace {
 // Launch shapes (blocks per SM; two are resident at a time).  Materialise is
 // fastest with about one group per warp: short-lived blocks keep the warps of an
 // SM at different stages (set-up, staging, draining stores) and the running
-// warps write neighbouring stretches of every output array.  Count and write
-// are arithmetic-bound and prefer long runs of groups per warp (the per-model
-// coefficients are then computed once).
+// warps write neighbouring stretches of every output array.  Count is
+// arithmetic-bound and prefers long runs of groups per warp (the per-model
+// coefficients are then computed once).  Write skips the groups without
+// survivors, which come in long stretches (invalid factorisations), so it takes
+// shorter runs to stay balanced.
 #ifndef EVAL_GRID_PER_SM_MATERIALISE
 #define EVAL_GRID_PER_SM_MATERIALISE 64
 #endif
 #ifndef EVAL_GRID_PER_SM_COMPACT
 #define EVAL_GRID_PER_SM_COMPACT 2
+#endif
+#ifndef EVAL_GRID_PER_SM_WRITE
+#define EVAL_GRID_PER_SM_WRITE 8
 #endif
 constexpr int THREADS = EVAL_THREADS;
 constexpr int WARPS = THREADS / 32;
@@ -130,9 +138,21 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
   const int lane = threadIdx.x & 31;
   const u32 warp_global = blockIdx.x * WARPS + (threadIdx.x >> 5);
   const u32 n_warps = gridDim.x * WARPS;
-  const u32 per_warp = (a.n_tiles + n_warps - 1) / n_warps;
-  const u32 seg_begin = min(warp_global * per_warp, a.n_tiles);
+  // count: one warp per run of the plan; otherwise the groups are dealt evenly
+  const u32 per_warp = MODE == MODE_COUNT ? a.run_len : (a.n_tiles + n_warps - 1) / n_warps;
+  const u32 seg_begin = (u32)min((u64)warp_global * per_warp, (u64)a.n_tiles);
   const u32 seg_end = min(seg_begin + per_warp, a.n_tiles);
+  u64 run_total = 0;                 // count: survivors of this warp's run
+  u64 write_next = 0;                // write: where the next group's survivors go
+  if (MODE == MODE_WRITE && seg_begin < seg_end) {
+    // survivors before this warp's first group = those of the runs before its run
+    // (scanned) plus those of the run's earlier groups
+    const u32 run = seg_begin / a.run_len;
+    u64 part = 0;
+    for (u32 j = run * a.run_len + lane; j < seg_begin; j += 32) part += a.tile_count[j];
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    write_next = a.tile_offset[run] + part;
+  }
   const u32 groups_per_model = sp.n_facts * sp.nvt;
 
   // the lane's triples: modes never change
@@ -164,6 +184,12 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
   u32 st_many[R], st_one[R];                      // static description for D > 1 and D = 1
 
   for (u32 seg = seg_begin; seg < seg_end; ++seg) {
+    // the count pass has evaluated every point of the group: nothing to place if none survived
+    u32 group_survivors = 0;
+    if (MODE == MODE_WRITE) {
+      group_survivors = a.tile_count[seg];
+      if (group_survivors == 0) continue;
+    }
     const u64 g = a.first_group + seg;
     const u32 model = (u32)(g / groups_per_model);
     const u32 gl = (u32)(g - (u64)model * groups_per_model);
@@ -242,7 +268,7 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
 
     u32 n_kept = 0;
     u64 write_base = 0;
-    if (MODE == MODE_WRITE) write_base = a.tile_offset[seg];
+    if (MODE == MODE_WRITE) { write_base = write_next; write_next += group_survivors; }
 
     // flags of a point = what the triple fixes | what the digit fixes | what needs both:
     //   gradient integrity needs the triple's two availability bits and the digit's,
@@ -343,28 +369,35 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
         }
       }
     }
-    if (MODE == MODE_COUNT && lane == 0) a.tile_count[seg] = n_kept;
+    if (MODE == MODE_COUNT) {
+      if (lane == 0) a.tile_count[seg] = n_kept;
+      run_total += n_kept;
+    }
   }
+  if (MODE == MODE_COUNT && lane == 0 && warp_global < a.n_runs) a.tile_offset[warp_global] = run_total;
   // the staging buffers must outlive the bulk stores that read them
   if (MODE == MODE_MATERIALISE && lane == 0) bulk_wait_all();
 }
 
-// exclusive prefix sum of the per-group survivor counts; one block that walks
-// the counts in tiles of 4096 with coalesced loads, a shuffle scan per warp and
-// one shared-memory pass per tile
-__global__ void __launch_bounds__(1024) k_tile_scan(EvalArgs a) {
+// exclusive prefix sum, in place, of the survivors of the count pass's runs
+// (a.tile_offset[0 .. n_runs)); the total goes to *a.n_out.  One block: there are
+// a few thousand runs, four per thread and tile.
+constexpr int SCAN_THREADS = 1024, SCAN_ITEMS = 4;
+__global__ void __launch_bounds__(SCAN_THREADS) k_tile_scan(EvalArgs a) {
   __shared__ u64 warp_sum[32];
   __shared__ u64 carry;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const u32 n = a.n_tiles;
+  const u32 n = a.n_runs;
   if (tid == 0) carry = 0;
   __syncthreads();
-  for (u32 tile = 0; tile < n; tile += 4096) {
-    const u32 i0 = tile + 4 * tid;
-    u32 c[4];
+  for (u32 tile = 0; tile < n; tile += SCAN_THREADS * SCAN_ITEMS) {
+    const u32 i0 = tile + SCAN_ITEMS * tid;
+    u64 c[SCAN_ITEMS];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) c[k] = (i0 + k < n) ? a.tile_count[i0 + k] : 0u;
-    const u64 mine = (u64)c[0] + c[1] + c[2] + c[3];
+    for (int k = 0; k < SCAN_ITEMS; ++k) c[k] = (i0 + k < n) ? a.tile_offset[i0 + k] : 0;
+    u64 mine = 0;
+#pragma unroll
+    for (int k = 0; k < SCAN_ITEMS; ++k) mine += c[k];
     u64 incl = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -377,12 +410,12 @@ __global__ void __launch_bounds__(1024) k_tile_scan(EvalArgs a) {
     for (int w = 0; w < warp; ++w) before += warp_sum[w];
     u64 run = before + incl - mine;
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
+    for (int k = 0; k < SCAN_ITEMS; ++k) {
       if (i0 + k < n) a.tile_offset[i0 + k] = run;
       run += c[k];
     }
     __syncthreads();
-    if (tid == 1023) carry = before + incl;
+    if (tid == SCAN_THREADS - 1) carry = before + incl;
     __syncthreads();
   }
   if (tid == 0) *a.n_out = carry;
@@ -393,9 +426,11 @@ cudaError_t launch_eval_t(const SpaceDev& sp, const EvalArgs& a, cudaStream_t st
   // one warp per run of groups; enough blocks to fill the GPU, no more than groups
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const unsigned needed = (a.n_tiles + WARPS - 1) / WARPS;
-  const unsigned most = (unsigned)sms * (MODE == MODE_MATERIALISE ? EVAL_GRID_PER_SM_MATERIALISE : EVAL_GRID_PER_SM_COMPACT);
-  const unsigned blocks = needed < most ? needed : most;
+  const unsigned needed = ((MODE == MODE_COUNT ? a.n_runs : a.n_tiles) + WARPS - 1) / WARPS;
+  const unsigned most = (unsigned)sms * (MODE == MODE_MATERIALISE ? EVAL_GRID_PER_SM_MATERIALISE
+                                         : MODE == MODE_WRITE     ? EVAL_GRID_PER_SM_WRITE
+                                                                  : EVAL_GRID_PER_SM_COMPACT);
+  const unsigned blocks = (MODE == MODE_COUNT || needed < most) ? needed : most;   // count: a warp per run
   constexpr int NC = NM * NM * NM * NM;
   const size_t smem = MODE == MODE_MATERIALISE ? (size_t)WARPS * 2 * Stage<NC>::BYTES : 0;
   if (smem > 48 * 1024) {
@@ -419,6 +454,20 @@ cudaError_t launch_eval_m(const SpaceDev& sp, const EvalArgs& a, cudaStream_t st
 
 }  // namespace
 
+// The count pass's runs: as many as fill the GPU with long-lived warps, but no
+// run longer than 32 groups (the write pass adds up the counts of a run's
+// earlier groups with one load per lane).
+void eval_plan_runs(EvalArgs& a) {
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const u32 target = (u32)sms * EVAL_GRID_PER_SM_COMPACT * WARPS;
+  u32 len = (a.n_tiles + target - 1) / target;
+  if (len < 1) len = 1;
+  if (len > 32) len = 32;
+  a.run_len = len;
+  a.n_runs = (a.n_tiles + len - 1) / len;
+}
+
 cudaError_t launch_eval_materialise(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream) {
   return launch_eval_m<MODE_MATERIALISE>(sp, a, stream);
 }
@@ -426,7 +475,7 @@ cudaError_t launch_eval_count(const SpaceDev& sp, const EvalArgs& a, cudaStream_
   return launch_eval_m<MODE_COUNT>(sp, a, stream);
 }
 cudaError_t launch_tile_scan(const EvalArgs& a, cudaStream_t stream) {
-  k_tile_scan<<<1, 1024, 0, stream>>>(a);
+  k_tile_scan<<<1, SCAN_THREADS, 0, stream>>>(a);
   return cudaGetLastError();
 }
 cudaError_t launch_eval_write(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream) {

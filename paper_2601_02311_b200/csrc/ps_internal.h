@@ -108,11 +108,15 @@ struct EvalArgs {
   u64* idx_out;
   u64* n_out;
   // compaction scratch
-  u32* tile_count;          // [n_tiles] survivors of each tile
-  u64* tile_offset;         // [n_tiles] exclusive prefix
+  // compaction: the count pass walks the groups in n_runs runs of run_len
+  // consecutive groups (one warp per run) -- set by eval_plan_runs
+  u32 n_runs, run_len;
+  u32* tile_count;          // [n_tiles] survivors of each group
+  u64* tile_offset;         // [n_runs <= n_tiles] survivors of each run, then (scan) of all runs before it
   u32* status;
 };
 
+void eval_plan_runs(EvalArgs& a);   // fills n_runs, run_len from n_tiles (current device)
 cudaError_t launch_eval_materialise(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream);
 cudaError_t launch_eval_count(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream);
 cudaError_t launch_tile_scan(const EvalArgs& a, cudaStream_t stream);

@@ -97,10 +97,12 @@ extern "C" int ps_eval_compact_noalloc(ps_ctx* ctx, const ps_space* sp, uint64_t
   a.require_flags = filter->require_flags & ~(u32)PS_F_FEASIBLE;
   a.tile_count = static_cast<u32*>(base);
   a.tile_offset = reinterpret_cast<u64*>(static_cast<unsigned char*>(base) + COUNT_BYTES);
+  eval_plan_runs(a);
   // The array still holds the previous call's numbers.  Every word this call
   // reads is written earlier in this call (the count pass stores a count for
-  // each group, the scan stores each offset); the counts are cleared anyway so
-  // that a stale value can never be mistaken for a fresh one.
+  // each group and a total for each run of groups, the scan turns the totals
+  // into offsets); the counts are cleared anyway so that a stale value can
+  // never be mistaken for a fresh one.
   if (cudaMemsetAsync(a.tile_count, 0, sizeof(u32) * n_groups, ctx->stream) != cudaSuccess) return PS_E_CUDA;
   if (launch_eval_count(sp->dev, a, ctx->stream) != cudaSuccess) return PS_E_CUDA;
   if (launch_tile_scan(a, ctx->stream) != cudaSuccess) return PS_E_CUDA;
