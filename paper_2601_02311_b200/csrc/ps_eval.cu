@@ -155,6 +155,9 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
   }
   const u32 groups_per_model = sp.n_facts * sp.nvt;
 
+  // with all five modes allowed digit d is mode d, and the compiler knows every
+  // per-digit property below
+  const u32 modemap = (NM == 5) ? 0x43210u : sp.modemap;
   // the lane's triples: modes never change
   u32 th[R], om[R], gr[R];
   bool live[R];
@@ -163,15 +166,15 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
     const u32 t = lane + 32 * r;
     live[r] = t < (u32)N3;
     const u32 tt = live[r] ? t : 0;
-    th[r] = digit_mode(sp.modemap, tt % NM);
-    om[r] = digit_mode(sp.modemap, (tt / NM) % NM);
-    gr[r] = digit_mode(sp.modemap, tt / N2);
+    th[r] = digit_mode(modemap, tt % NM);
+    om[r] = digit_mode(modemap, (tt / NM) % NM);
+    gr[r] = digit_mode(modemap, tt / N2);
   }
   // classes of the activation digit (Theorem 3: a replica needs its own activations)
   u32 own = 0, is_o = 0, not_mo = 0;
 #pragma unroll
   for (int d = 0; d < NM; ++d) {
-    const u32 ac = digit_mode(sp.modemap, d);
+    const u32 ac = digit_mode(modemap, d);
     if (in_set(SET_ACT_OWN, ac)) own |= 1u << d;
     if (ac == PS_MODE_O) is_o |= 1u << d;
     if (!in_set(SET_M_OR_O, ac)) not_mo |= 1u << d;
@@ -244,7 +247,7 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
     const u64 c_axis = model_axis_traffic(rec, f, ub, tau, sp.tp_coll, sp.accum);
     u64 act[NM];
 #pragma unroll
-    for (int d = 0; d < NM; ++d) act[d] = mu_elems(digit_mode(sp.modemap, d), ab.EA, ab.shA, ab.uA, sp.sstar_units);
+    for (int d = 0; d < NM; ++d) act[d] = mu_elems(digit_mode(modemap, d), ab.EA, ab.shA, ab.uA, sp.sstar_units);
     const u64 act_host = 2 * ab.EA * sp.accum;
     const u32 avail = ub.d1 ? ((1u << NM) - 1u) : own;     // digits with PS_F_ACT_AVAIL
 

@@ -342,11 +342,15 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
   constexpr u32 CV_BITS = PS_F_CV | PS_F_T_DIV_HEADS | PS_F_K_DIV_LAYERS | PS_F_TP_LE_MAX | PS_F_AXIS_FORM;
   const u32 req_cv = req & CV_BITS;
 
+  // with all five modes allowed digit d is mode d: the compiler then knows every
+  // per-digit property below (which digit offloads, which keep a replica's own
+  // activations) and drops the tests
+  const u32 modemap = (NM == 5) ? 0x43210u : sp.modemap;
   // activation-digit classes (Theorem 3: a replica needs its own activations)
   u32 all = (1u << NM) - 1u, own = 0, is_o = 0, not_mo = 0;
 #pragma unroll
   for (int d = 0; d < NM; ++d) {
-    const u32 ac = digit_mode(sp.modemap, d);
+    const u32 ac = digit_mode(modemap, d);
     if (in_set(SET_ACT_OWN, ac)) own |= 1u << d;
     if (ac == PS_MODE_O) is_o |= 1u << d;
     if (!in_set(SET_M_OR_O, ac)) not_mo |= 1u << d;
@@ -368,8 +372,8 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
     const u32 t = lane + 32 * r;
     const bool live = t < (u32)N3;
     const u32 tt = live ? t : 0;
-    const u32 modes[3] = {digit_mode(sp.modemap, tt % NM), digit_mode(sp.modemap, (tt / NM) % NM),
-                          digit_mode(sp.modemap, tt / N2)};
+    const u32 modes[3] = {digit_mode(modemap, tt % NM), digit_mode(modemap, (tt / NM) % NM),
+                          digit_mode(modemap, tt / N2)};
     const u32 width[3] = {rec.wT, rec.wO, rec.wG};
     const u32 th = modes[0], om = modes[1], gr = modes[2];
     const bool on_shard = in_set(SET_UPDATE_ON_SHARD, om);
@@ -411,7 +415,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
   const bool tl_mine = tl_vt < nvt;
   const u32 tl_v = tl_mine ? tl_vt / sp.nt : 0;
   const u32 tl_tau = tl_mine ? tl_vt - tl_v * sp.nt : 0;
-  const u32 tl_mode = digit_mode(sp.modemap, tl_d);
+  const u32 tl_mode = digit_mode(modemap, tl_d);
   const u64 tl_A = rec.A[tl_v], tl_UA = rec.UA[tl_v];
 
   // warps take the block's units in turn: the first one by warp number, then
