@@ -301,8 +301,9 @@ __device__ __forceinline__ u32 allowed_act_digits(u32 tb, u32 req, u32 all, u32 
 }
 
 // KIND: the reduction; NM: allowed modes; WARPS x 32 threads per block, compiled
-// for MIN_BLOCKS resident blocks per SM
-template <int KIND, int NM, int WARPS, int MIN_BLOCKS>
+// for MIN_BLOCKS resident blocks per SM; HOST_LIMITED: the filter has a host
+// budget (without one the host bytes are never formed)
+template <int KIND, int NM, int WARPS, int MIN_BLOCKS, bool HOST_LIMITED>
 __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, SweepArgs args) {
   constexpr int THREADS = WARPS * 32;
   constexpr int N2 = NM * NM, N3 = NM * NM * NM, NC = N3 * NM;
@@ -338,7 +339,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
   // capacities as exclusive bounds (memory and host bytes stay below 2^63)
   const u64 cap_x = min(args.cap_max, (u64)1 << 62) + 1;
   const u64 host_x = min(args.host_cap, (u64)1 << 62) + 1;
-  const bool host_limited = args.host_cap < ((u64)1 << 62);
+  constexpr bool host_limited = HOST_LIMITED;      // the launcher tests args.host_cap < 2^62
   constexpr u32 CV_BITS = PS_F_CV | PS_F_T_DIV_HEADS | PS_F_K_DIV_LAYERS | PS_F_TP_LE_MAX | PS_F_AXIS_FORM;
   const u32 req_cv = req & CV_BITS;
 
@@ -952,17 +953,23 @@ __global__ void __launch_bounds__(MERGE_THREADS) k_sweep_merge(SpaceDev sp, Merg
 }  // namespace
 
 // ------------------------------------------------------------------ launchers
-template <int KIND, int NM>
-static cudaError_t launch_sweep_t(const SpaceDev& sp, const SweepArgs& a, u32 n_chunks, cudaStream_t stream) {
+template <int KIND, int NM, bool HOST_LIMITED>
+static cudaError_t launch_sweep_h(const SpaceDev& sp, const SweepArgs& a, u32 n_chunks, cudaStream_t stream) {
   constexpr int WARPS = KIND == PS_REDUCE_PARETO ? SWEEP_WARPS_PARETO : SWEEP_WARPS_TOPK;
   constexpr int MIN_BLOCKS = KIND == PS_REDUCE_PARETO ? SWEEP_BLOCKS_PARETO : SWEEP_BLOCKS_TOPK;
   dim3 grid(n_chunks, sp.n_models);
   const size_t smem = sizeof(SweepShared<WARPS>);
-  cudaError_t e = cudaFuncSetAttribute(k_sweep<KIND, NM, WARPS, MIN_BLOCKS>,
+  cudaError_t e = cudaFuncSetAttribute(k_sweep<KIND, NM, WARPS, MIN_BLOCKS, HOST_LIMITED>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  k_sweep<KIND, NM, WARPS, MIN_BLOCKS><<<grid, WARPS * 32, smem, stream>>>(sp, a);
+  k_sweep<KIND, NM, WARPS, MIN_BLOCKS, HOST_LIMITED><<<grid, WARPS * 32, smem, stream>>>(sp, a);
   return cudaGetLastError();
+}
+
+template <int KIND, int NM>
+static cudaError_t launch_sweep_t(const SpaceDev& sp, const SweepArgs& a, u32 n_chunks, cudaStream_t stream) {
+  return a.host_cap < ((u64)1 << 62) ? launch_sweep_h<KIND, NM, true>(sp, a, n_chunks, stream)
+                                     : launch_sweep_h<KIND, NM, false>(sp, a, n_chunks, stream);
 }
 
 template <int KIND>
