@@ -768,7 +768,10 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
 // kept so far, so any number can be combined.  Each emitted point is evaluated
 // again from its index (host bytes and flags come from there; mem and comm must
 // agree).
-constexpr int MERGE_THREADS = 256;
+#ifndef SWEEP_MERGE_THREADS
+#define SWEEP_MERGE_THREADS 128
+#endif
+constexpr int MERGE_THREADS = SWEEP_MERGE_THREADS;
 constexpr int MERGE_LISTS = MERGE_CAP / LIST_CAP - 1;   // lists per round beside the kept entries
 
 struct MergeShared {
