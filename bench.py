@@ -58,7 +58,7 @@ BYTES_PER_POINT_MATERIALISE = 36
 # (k_sweep<top-k> on the full stress configuration; k_eval<materialise> per point
 # of a 2^25-point window, where traffic grows in proportion to the points)
 NCU_SWEEP_DRAM_BYTES = 5_313_792
-NCU_MATERIALISE_DRAM_BYTES_PER_POINT = 1_400_919_560 / (1 << 25)
+NCU_MATERIALISE_DRAM_BYTES_PER_POINT = 1_355_840_944 / (1 << 25)
 
 
 def parse_args():
