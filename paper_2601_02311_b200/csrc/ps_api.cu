@@ -250,6 +250,9 @@ int ps_space_create(ps_ctx* ctx, const ps_space_desc* desc, ps_space** out) {
   d.tp_coll = desc->tp_coll_per_layer;
   d.sstar_units = desc->sstar_units ? desc->sstar_units : 1;
   d.accum = accum;
+  d.all_pow2 = 1;
+  for (u32 i = 0; i < desc->n_n; ++i)
+    if (desc->n_values[i] & (desc->n_values[i] - 1)) d.all_pow2 = 0;
   const u64 ppm = (u64)d.n_facts * d.nvt * d.n_codes;
   if (ppm >= ((u64)1 << 32)) { delete sp; return PS_E_RANGE; }
   d.ppm = ppm;

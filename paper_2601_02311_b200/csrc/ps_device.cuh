@@ -45,6 +45,7 @@ struct SpaceDev {
   u32 tp_max_valid, tp_coll;
   u32 sstar_units;    // unit buffers a gathered (S*) state holds at a time: 1, or 2 when gathers overlap computation
   u32 accum;          // micro-batches per step (gradient accumulation), >= 1
+  u32 all_pow2;       // 1 if every device count of the space is a power of two (then every T, K, D is)
 };
 
 enum : u32 {

@@ -302,8 +302,9 @@ __device__ __forceinline__ u32 allowed_act_digits(u32 tb, u32 req, u32 all, u32 
 
 // KIND: the reduction; NM: allowed modes; WARPS x 32 threads per block, compiled
 // for MIN_BLOCKS resident blocks per SM; HOST_LIMITED: the filter has a host
-// budget (without one the host bytes are never formed)
-template <int KIND, int NM, int WARPS, int MIN_BLOCKS, bool HOST_LIMITED>
+// budget (without one the host bytes are never formed); POW2: every degree of
+// the space is a power of two (no division is compiled in)
+template <int KIND, int NM, int WARPS, int MIN_BLOCKS, bool HOST_LIMITED, bool POW2>
 __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, SweepArgs args) {
   constexpr int THREADS = WARPS * 32;
   constexpr int N2 = NM * NM, N3 = NM * NM * NM, NC = N3 * NM;
@@ -424,14 +425,14 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
   for (u32 unit = u_begin + warp; unit < u_end;) {
     const Fact f = sp.facts[unit];
     const Pow2 p2 = pow2_of(f);
-    const UnitBase ub = p2.all ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
+    const UnitBase ub = (POW2 || p2.all) ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
                                : unit_base(rec, f, sp.tp_max_valid, true);
     __syncwarp();
     {
       // lane (vt, d): activation bytes of digit d under variant vt, and the bound
       // a triple's own bytes must stay below for the sum to fit the capacity
       ActBase ab;
-      if (p2.all) {
+      if (POW2 || p2.all) {
         const u32 s = tl_tau == 0 ? p2.sT : 0;
         ab.EA = ceil_shift(tl_A, s);
         ab.uA = ceil_shift(tl_UA, s);
@@ -956,23 +957,27 @@ __global__ void __launch_bounds__(MERGE_THREADS) k_sweep_merge(SpaceDev sp, Merg
 }  // namespace
 
 // ------------------------------------------------------------------ launchers
-template <int KIND, int NM, bool HOST_LIMITED>
-static cudaError_t launch_sweep_h(const SpaceDev& sp, const SweepArgs& a, u32 n_chunks, cudaStream_t stream) {
+template <int KIND, int NM, bool HOST_LIMITED, bool POW2>
+static cudaError_t launch_sweep_p(const SpaceDev& sp, const SweepArgs& a, u32 n_chunks, cudaStream_t stream) {
   constexpr int WARPS = KIND == PS_REDUCE_PARETO ? SWEEP_WARPS_PARETO : SWEEP_WARPS_TOPK;
   constexpr int MIN_BLOCKS = KIND == PS_REDUCE_PARETO ? SWEEP_BLOCKS_PARETO : SWEEP_BLOCKS_TOPK;
   dim3 grid(n_chunks, sp.n_models);
   const size_t smem = sizeof(SweepShared<WARPS>);
-  cudaError_t e = cudaFuncSetAttribute(k_sweep<KIND, NM, WARPS, MIN_BLOCKS, HOST_LIMITED>,
+  cudaError_t e = cudaFuncSetAttribute(k_sweep<KIND, NM, WARPS, MIN_BLOCKS, HOST_LIMITED, POW2>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  k_sweep<KIND, NM, WARPS, MIN_BLOCKS, HOST_LIMITED><<<grid, WARPS * 32, smem, stream>>>(sp, a);
+  k_sweep<KIND, NM, WARPS, MIN_BLOCKS, HOST_LIMITED, POW2><<<grid, WARPS * 32, smem, stream>>>(sp, a);
   return cudaGetLastError();
 }
 
 template <int KIND, int NM>
 static cudaError_t launch_sweep_t(const SpaceDev& sp, const SweepArgs& a, u32 n_chunks, cudaStream_t stream) {
-  return a.host_cap < ((u64)1 << 62) ? launch_sweep_h<KIND, NM, true>(sp, a, n_chunks, stream)
-                                     : launch_sweep_h<KIND, NM, false>(sp, a, n_chunks, stream);
+  const bool host_limited = a.host_cap < ((u64)1 << 62);
+  if (sp.all_pow2)
+    return host_limited ? launch_sweep_p<KIND, NM, true, true>(sp, a, n_chunks, stream)
+                        : launch_sweep_p<KIND, NM, false, true>(sp, a, n_chunks, stream);
+  return host_limited ? launch_sweep_p<KIND, NM, true, false>(sp, a, n_chunks, stream)
+                      : launch_sweep_p<KIND, NM, false, false>(sp, a, n_chunks, stream);
 }
 
 template <int KIND>
