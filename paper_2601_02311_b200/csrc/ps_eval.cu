@@ -127,7 +127,8 @@ __device__ __forceinline__ void warp_bulk_store(T* __restrict__ dst, const T* bu
   if (lane == 0) asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 
-template <int MODE, int NM>
+// POW2: every degree of the space is a power of two (no division is compiled in)
+template <int MODE, int NM, bool POW2>
 __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
   constexpr int N2 = NM * NM, N3 = NM * NM * NM, NC = N3 * NM;
   constexpr int R = (N3 + 31) / 32;
@@ -241,9 +242,9 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
     // ---- per group: shard quantities (all divisions), activation bytes per digit
     const Fact f = sp.facts[unit];
     const Pow2 p2 = pow2_of(f);
-    const UnitBase ub = p2.all ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
+    const UnitBase ub = (POW2 || p2.all) ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
                                : unit_base(rec, f, sp.tp_max_valid, true);
-    const ActBase ab = p2.all ? act_base_pow2(rec, p2, v, tau) : act_base(rec, f, v, tau);
+    const ActBase ab = (POW2 || p2.all) ? act_base_pow2(rec, p2, v, tau) : act_base(rec, f, v, tau);
     const u64 c_axis = model_axis_traffic(rec, f, ub, tau, sp.tp_coll, sp.accum);
     u64 act[NM];
 #pragma unroll
@@ -424,8 +425,8 @@ __global__ void __launch_bounds__(SCAN_THREADS) k_tile_scan(EvalArgs a) {
   if (tid == 0) *a.n_out = carry;
 }
 
-template <int MODE, int NM>
-cudaError_t launch_eval_t(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream) {
+template <int MODE, int NM, bool POW2>
+cudaError_t launch_eval_p(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream) {
   // one warp per run of groups; enough blocks to fill the GPU, no more than groups
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -437,11 +438,16 @@ cudaError_t launch_eval_t(const SpaceDev& sp, const EvalArgs& a, cudaStream_t st
   constexpr int NC = NM * NM * NM * NM;
   const size_t smem = MODE == MODE_MATERIALISE ? (size_t)WARPS * 2 * Stage<NC>::BYTES : 0;
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(k_eval<MODE, NM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(k_eval<MODE, NM, POW2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  k_eval<MODE, NM><<<blocks, THREADS, smem, stream>>>(sp, a);
+  k_eval<MODE, NM, POW2><<<blocks, THREADS, smem, stream>>>(sp, a);
   return cudaGetLastError();
+}
+
+template <int MODE, int NM>
+cudaError_t launch_eval_t(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream) {
+  return sp.all_pow2 ? launch_eval_p<MODE, NM, true>(sp, a, stream) : launch_eval_p<MODE, NM, false>(sp, a, stream);
 }
 
 template <int MODE>
