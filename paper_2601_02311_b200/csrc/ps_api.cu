@@ -63,6 +63,17 @@ bool shape_in_range(const ps_model_shape& s, u32 tp_coll, u32 accum = 1) {
   return true;
 }
 
+// whether every byte count of a (Theta, Omega, G) triple of this model stays below 2^53
+bool shape_is_small(const ps_model_shape& s) {
+  typedef unsigned __int128 u128;
+  const u128 H = s.hidden;
+  const u128 P = s.param_elems_override ? (u128)s.param_elems_override
+                                        : 12 * (u128)s.layers * H * H + (u128)s.vocab * H;
+  const u128 unit = s.unit_from_shape ? 12 * H * H : 0;
+  const u128 wsum = (u128)s.w_param + s.w_grad + s.w_opt;
+  return wsum * (P + 2 * unit) < ((u128)1 << 53);
+}
+
 int ensure_scratch(ps_ctx* ctx, size_t bytes) {
   if (bytes <= ctx->scratch_bytes) return PS_OK;
   CUDA_OK(cudaStreamSynchronize(ctx->stream));
@@ -275,8 +286,12 @@ int ps_space_create(ps_ctx* ctx, const ps_space_desc* desc, ps_space** out) {
 int ps_space_set_models(ps_space* sp, const ps_model_shape* models, uint32_t n_models) {
   if (!sp || !models) return PS_E_NULLPTR;
   if (n_models != sp->dev.n_models) return PS_E_RANGE;
-  for (u32 i = 0; i < n_models; ++i)
+  u32 all_small = 1;
+  for (u32 i = 0; i < n_models; ++i) {
     if (!shape_in_range(models[i], sp->dev.tp_coll, sp->dev.accum)) return PS_E_RANGE;
+    if (!shape_is_small(models[i])) all_small = 0;
+  }
+  sp->dev.all_small = all_small;
   ps_ctx* ctx = sp->ctx;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return PS_E_CUDA;

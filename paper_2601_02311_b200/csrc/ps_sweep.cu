@@ -302,9 +302,10 @@ __device__ __forceinline__ u32 allowed_act_digits(u32 tb, u32 req, u32 all, u32 
 
 // KIND: the reduction; NM: allowed modes; WARPS x 32 threads per block, compiled
 // for MIN_BLOCKS resident blocks per SM; HOST_LIMITED: the filter has a host
-// budget (without one the host bytes are never formed); POW2: every degree of
-// the space is a power of two (no division is compiled in)
-template <int KIND, int NM, int WARPS, int MIN_BLOCKS, bool HOST_LIMITED, bool POW2>
+// budget (without one the host bytes are never formed); FAST: every degree of
+// the space is a power of two and every byte count is below 2^53 (no division
+// and no 64-bit integer compare is compiled into the evaluation)
+template <int KIND, int NM, int WARPS, int MIN_BLOCKS, bool HOST_LIMITED, bool FAST>
 __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, SweepArgs args) {
   constexpr int THREADS = WARPS * 32;
   constexpr int N2 = NM * NM, N3 = NM * NM * NM, NC = N3 * NM;
@@ -425,14 +426,14 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
   for (u32 unit = u_begin + warp; unit < u_end;) {
     const Fact f = sp.facts[unit];
     const Pow2 p2 = pow2_of(f);
-    const UnitBase ub = (POW2 || p2.all) ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
+    const UnitBase ub = (FAST || p2.all) ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
                                : unit_base(rec, f, sp.tp_max_valid, true);
     __syncwarp();
     {
       // lane (vt, d): activation bytes of digit d under variant vt, and the bound
       // a triple's own bytes must stay below for the sum to fit the capacity
       ActBase ab;
-      if (POW2 || p2.all) {
+      if (FAST || p2.all) {
         const u32 s = tl_tau == 0 ? p2.sT : 0;
         ab.EA = ceil_shift(tl_A, s);
         ab.uA = ceil_shift(tl_UA, s);
@@ -484,8 +485,8 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
     // Integers below 2^53 are exact in fp64, so when every quantity of the unit is
     // that small (uniform test) the compares run on the fp64 pipe, which is idle
     // otherwise, and only the counting stays on the integer pipe.
-    const bool small = cap_x < ((u64)1 << 53) &&
-                       (u64)(rec.wT + rec.wO + rec.wG) * (ub.E2 + 2 * ub.u) < ((u64)1 << 53);
+    const bool small = FAST || (cap_x < ((u64)1 << 53) &&
+                                (u64)(rec.wT + rec.wO + rec.wG) * (ub.E2 + 2 * ub.u) < ((u64)1 << 53));
     if (small) {
       double mem_f64[R];
       float pass_f32[R];
@@ -957,23 +958,24 @@ __global__ void __launch_bounds__(MERGE_THREADS) k_sweep_merge(SpaceDev sp, Merg
 }  // namespace
 
 // ------------------------------------------------------------------ launchers
-template <int KIND, int NM, bool HOST_LIMITED, bool POW2>
+template <int KIND, int NM, bool HOST_LIMITED, bool FAST>
 static cudaError_t launch_sweep_p(const SpaceDev& sp, const SweepArgs& a, u32 n_chunks, cudaStream_t stream) {
   constexpr int WARPS = KIND == PS_REDUCE_PARETO ? SWEEP_WARPS_PARETO : SWEEP_WARPS_TOPK;
   constexpr int MIN_BLOCKS = KIND == PS_REDUCE_PARETO ? SWEEP_BLOCKS_PARETO : SWEEP_BLOCKS_TOPK;
   dim3 grid(n_chunks, sp.n_models);
   const size_t smem = sizeof(SweepShared<WARPS>);
-  cudaError_t e = cudaFuncSetAttribute(k_sweep<KIND, NM, WARPS, MIN_BLOCKS, HOST_LIMITED, POW2>,
+  cudaError_t e = cudaFuncSetAttribute(k_sweep<KIND, NM, WARPS, MIN_BLOCKS, HOST_LIMITED, FAST>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  k_sweep<KIND, NM, WARPS, MIN_BLOCKS, HOST_LIMITED, POW2><<<grid, WARPS * 32, smem, stream>>>(sp, a);
+  k_sweep<KIND, NM, WARPS, MIN_BLOCKS, HOST_LIMITED, FAST><<<grid, WARPS * 32, smem, stream>>>(sp, a);
   return cudaGetLastError();
 }
 
 template <int KIND, int NM>
 static cudaError_t launch_sweep_t(const SpaceDev& sp, const SweepArgs& a, u32 n_chunks, cudaStream_t stream) {
   const bool host_limited = a.host_cap < ((u64)1 << 62);
-  if (sp.all_pow2)
+  // the fast case: powers of two everywhere, every byte count exact in a double
+  if (sp.all_pow2 && sp.all_small && a.cap_max < ((u64)1 << 53) - 1)
     return host_limited ? launch_sweep_p<KIND, NM, true, true>(sp, a, n_chunks, stream)
                         : launch_sweep_p<KIND, NM, false, true>(sp, a, n_chunks, stream);
   return host_limited ? launch_sweep_p<KIND, NM, true, false>(sp, a, n_chunks, stream)

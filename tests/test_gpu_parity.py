@@ -355,3 +355,18 @@ def test_smallest_possible_space(ctx, ps):
     filt = dict(require_flags=VALID)
     for kind_g, kind_o in ((ps.REDUCE_PARETO, O.KIND_PARETO), (ps.REDUCE_TOPK, O.KIND_TOPK)):
         assert_same_sweep(gs.sweep(filt, [O.NO_LIMIT], kind_g, 4), os_.sweep(filt, [O.NO_LIMIT], kind_o, 4))
+
+
+@pytest.mark.parametrize("cap", [(1 << 53) - 2, (1 << 53) - 1, 1 << 60])
+def test_sweeps_around_the_exact_double_limit(ctx, ps, cap):
+    """A power-of-two space runs kernels compiled for byte counts below 2^53 when
+    the capacity allows it and the general ones otherwise: same results."""
+    space = synth.config("C3", n_models=2)
+    gs, os_ = both(ctx, space)
+    caps = [192 * synth.GB, cap]
+    filt = dict(require_flags=VALID, host_cap=64 * synth.GB)
+    assert_same_sweep(gs.sweep(filt, caps, ps.REDUCE_PARETO, 64),
+                      os_.sweep(filt, caps, O.KIND_PARETO, 64, n_threads=8))
+    filt = dict(require_flags=VALID)
+    assert_same_sweep(gs.sweep(filt, [cap], ps.REDUCE_TOPK, 64),
+                      os_.sweep(filt, [cap], O.KIND_TOPK, 64, n_threads=8))
