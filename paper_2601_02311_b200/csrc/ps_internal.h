@@ -32,9 +32,11 @@ struct ps_space {
 
 // ---- sweep
 // Block shapes of the sweep: warps per block and the resident blocks per SM the
-// kernel is compiled for (which caps its registers).  The top-k sweep gains from
-// more resident warps (five blocks of four warps: 96 registers); the Pareto
-// sweep is fastest with two blocks of eight warps (128 registers).
+// kernel is compiled for (which caps its registers).  The top-k sweep is fastest
+// with five blocks of four warps (96 registers): many resident warps, few and
+// long lists per model.  The Pareto sweep is fastest with two blocks of ten
+// warps (96 registers): its warps share a block's coarse staircase, so larger
+// blocks reject more candidates early.
 #ifndef SWEEP_WARPS_TOPK
 #define SWEEP_WARPS_TOPK 4
 #endif
@@ -42,7 +44,7 @@ struct ps_space {
 #define SWEEP_BLOCKS_TOPK 5
 #endif
 #ifndef SWEEP_WARPS_PARETO
-#define SWEEP_WARPS_PARETO 8
+#define SWEEP_WARPS_PARETO 10
 #endif
 #ifndef SWEEP_BLOCKS_PARETO
 #define SWEEP_BLOCKS_PARETO 2
@@ -51,7 +53,7 @@ static inline int sweep_warps(int kind) { return kind == PS_REDUCE_PARETO ? SWEE
 static inline int sweep_blocks_per_sm(int kind) { return kind == PS_REDUCE_PARETO ? SWEEP_BLOCKS_PARETO : SWEEP_BLOCKS_TOPK; }
 #define SWEEP_LIST_CAP 128        /* entries of a warp's list and of a block's partial list */
 #define SWEEP_MAX_CHUNKS 16       /* blocks per model                                        */
-#define MERGE_CAP (9 * SWEEP_LIST_CAP)    /* entries the merge kernel combines at a time: what it
+#define MERGE_CAP (11 * SWEEP_LIST_CAP)   /* entries the merge kernel combines at a time: what it
                                      has kept plus the lists of one block of the sweep       */
 #define PS_MAX_CAPS 8
 
