@@ -465,10 +465,15 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
     const bool unit_ok = (ub.cv & req_cv) == req_cv;
     const u32 a_shift = ub.d1 ? 8 : 0;
     u64 mem3[R], comm3[R], host3[R];
+    double mem3_f64[R];
+    const double e2_f64 = (double)ub.E2, sh_f64 = (double)ub.sh, u_f64 = (double)ub.u;
     u32 allowed[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      mem3[r] = mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0)));
+      // the fast case forms the bytes as a double right away (three exact fused
+      // multiply-adds) and the integer only if the reduction pass needs it
+      if (FAST) mem3_f64[r] = fma((double)ka[r], e2_f64, fma((double)kb[r], sh_f64, (double)kc[r] * u_f64));
+      else mem3[r] = mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0)));
       comm3[r] = mad_small(ub.x, kx[r], 0);
       host3[r] = host_limited ? mad_small(ub.sh, kh[r], 0) : 0;
       allowed[r] = (unit_ok && host3[r] < host_x) ? ((t_allowed[r] >> a_shift) & all) : 0;
@@ -491,7 +496,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
       double mem_f64[R];
       float pass_f32[R];
 #pragma unroll
-      for (int r = 0; r < R; ++r) { mem_f64[r] = (double)mem3[r]; pass_f32[r] = 0.0f; }
+      for (int r = 0; r < R; ++r) { mem_f64[r] = FAST ? mem3_f64[r] : (double)mem3[r]; pass_f32[r] = 0.0f; }
 #pragma unroll
       for (int d = 0; d < NM; ++d) {
         const bool host_check = host_limited && ((is_o >> d) & 1u);
@@ -592,7 +597,8 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
       u32 l_allowed[R], l_triple[R], l_pass[R];
 #pragma unroll
       for (int r = 0; r < R; ++r) {
-        l_mem[r] = mem3[r]; l_comm[r] = comm3[r]; l_host[r] = host3[r];
+        l_mem[r] = FAST ? mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0))) : mem3[r];
+        l_comm[r] = comm3[r]; l_host[r] = host3[r];
         l_allowed[r] = allowed[r]; l_triple[r] = t_local[r];
       }
       if (KIND == PS_REDUCE_PARETO) {
