@@ -63,15 +63,17 @@ bool shape_in_range(const ps_model_shape& s, u32 tp_coll, u32 accum = 1) {
   return true;
 }
 
-// whether every byte count of a (Theta, Omega, G) triple of this model stays below 2^53
-bool shape_is_small(const ps_model_shape& s) {
+// whether every byte count of a (Theta, Omega, G) triple of this model -- device
+// bytes (at most wsum * (P + 2 unit)) and host bytes (at most (2 accum + 1) * wsum * P)
+// -- stays below 2^53
+bool shape_is_small(const ps_model_shape& s, u32 accum) {
   typedef unsigned __int128 u128;
   const u128 H = s.hidden;
   const u128 P = s.param_elems_override ? (u128)s.param_elems_override
                                         : 12 * (u128)s.layers * H * H + (u128)s.vocab * H;
   const u128 unit = s.unit_from_shape ? 12 * H * H : 0;
   const u128 wsum = (u128)s.w_param + s.w_grad + s.w_opt;
-  return wsum * (P + 2 * unit) < ((u128)1 << 53);
+  return (2 * (u128)accum + 1) * wsum * (P + 2 * unit) < ((u128)1 << 53);
 }
 
 int ensure_scratch(ps_ctx* ctx, size_t bytes) {
@@ -289,7 +291,7 @@ int ps_space_set_models(ps_space* sp, const ps_model_shape* models, uint32_t n_m
   u32 all_small = 1;
   for (u32 i = 0; i < n_models; ++i) {
     if (!shape_in_range(models[i], sp->dev.tp_coll, sp->dev.accum)) return PS_E_RANGE;
-    if (!shape_is_small(models[i])) all_small = 0;
+    if (!shape_is_small(models[i], sp->dev.accum)) all_small = 0;
   }
   sp->dev.all_small = all_small;
   ps_ctx* ctx = sp->ctx;

@@ -39,6 +39,7 @@ struct WarpTables {
   __align__(16) double bound_f64[5][4];
   u64 act[4][5];           // activation bytes of digit d
   u64 host_bound[4];       // a triple whose own host bytes are below this may offload activations
+  __align__(16) double host_bound_f64[4];   // the same as doubles (the fast case compares there)
   u64 c_axis[4];           // tensor + pipeline traffic of the variant (0 if not in the objective)
   // Pareto: for every set of digits the one with the least activation bytes
   // (lowest digit on ties), NM for the empty set
@@ -451,13 +452,15 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
         tb.act[tl_vt][tl_d] = am;
         if (tl_d == 0) {
           const u64 ah = 2 * ab.EA * sp.accum;                 // offload after fwd, reload for bwd, per micro-batch
-          tb.host_bound[tl_vt] = ah < host_x ? host_x - ah : 0;
+          const u64 hb = ah < host_x ? host_x - ah : 0;
+          tb.host_bound[tl_vt] = hb;
+          tb.host_bound_f64[tl_vt] = (double)hb;      // rounded only above 2^53, where no host figure of the fast case reaches
           tb.c_axis[tl_vt] = ext_in_objective ? model_axis_traffic(rec, f, ub, tl_tau, sp.tp_coll, sp.accum) : 0;
         }
       } else if (tl_vt < 4) {
         tb.bound[tl_d][tl_vt] = 0;
         tb.bound_f64[tl_d][tl_vt] = 0.0;
-        if (tl_d == 0) tb.host_bound[tl_vt] = 0;
+        if (tl_d == 0) { tb.host_bound[tl_vt] = 0; tb.host_bound_f64[tl_vt] = 0.0; }
       }
     }
     __syncwarp();
@@ -465,7 +468,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
     const bool unit_ok = (ub.cv & req_cv) == req_cv;
     const u32 a_shift = ub.d1 ? 8 : 0;
     u64 mem3[R], comm3[R], host3[R];
-    double mem3_f64[R];
+    double mem3_f64[R], host3_f64[R];
     const double e2_f64 = (double)ub.E2, sh_f64 = (double)ub.sh, u_f64 = (double)ub.u;
     u32 allowed[R];
 #pragma unroll
@@ -475,8 +478,14 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
       if (FAST) mem3_f64[r] = fma((double)ka[r], e2_f64, fma((double)kb[r], sh_f64, (double)kc[r] * u_f64));
       else mem3[r] = mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0)));
       comm3[r] = mad_small(ub.x, kx[r], 0);
-      host3[r] = host_limited ? mad_small(ub.sh, kh[r], 0) : 0;
-      allowed[r] = (unit_ok && host3[r] < host_x) ? ((t_allowed[r] >> a_shift) & all) : 0;
+      bool host_fits = true;                    // the triple's own host bytes against the budget
+      if (host_limited) {
+        if (FAST) { host3_f64[r] = (double)kh[r] * sh_f64; host_fits = host3_f64[r] < (double)host_x; }
+        else { host3[r] = mad_small(ub.sh, kh[r], 0); host_fits = host3[r] < host_x; }
+      } else {
+        host3[r] = 0;
+      }
+      allowed[r] = (unit_ok && host_fits) ? ((t_allowed[r] >> a_shift) & all) : 0;
     }
     const u32 unit_first = unit * per_unit;      // index of the unit's first point in the model
 
@@ -516,7 +525,9 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
               // offloading activations also has to fit the host budget of the variant
 #pragma unroll
               for (int vt = 0; vt < 4; ++vt)
-                if (mem_f64[r] < bound[vt] && host3[r] < tb.host_bound[vt]) c += 1.0f;
+                if (mem_f64[r] < bound[vt] &&
+                    (FAST ? host3_f64[r] < tb.host_bound_f64[vt] : host3[r] < tb.host_bound[vt]))
+                  c += 1.0f;
             } else {
 #pragma unroll
               for (int vt = 0; vt < 4; ++vt)
@@ -598,7 +609,8 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
 #pragma unroll
       for (int r = 0; r < R; ++r) {
         l_mem[r] = FAST ? mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0))) : mem3[r];
-        l_comm[r] = comm3[r]; l_host[r] = host3[r];
+        l_comm[r] = comm3[r];
+        l_host[r] = (FAST && host_limited) ? mad_small(ub.sh, kh[r], 0) : host3[r];
         l_allowed[r] = allowed[r]; l_triple[r] = t_local[r];
       }
       if (KIND == PS_REDUCE_PARETO) {
