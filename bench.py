@@ -51,14 +51,14 @@ UNIT = "evals/s"
 # the integer issue rate measured by k_int_peak in the same run -- i.e. how busy
 # the integer-capable issue slots are.  A lower figure at the same fraction is
 # the real win (it was 86 in the first correct kernel and 11.3 before the kernels
-# were compiled for their mode set and host budget).
-EXEC_OPS_PER_POINT_SWEEP = 9.22
+# were compiled for the cases the space and the filter allow).
+EXEC_OPS_PER_POINT_SWEEP = 8.43
 BYTES_PER_POINT_MATERIALISE = 36
 # DRAM traffic of one launch from the ncu captures summarised under profiles/
 # (k_sweep<top-k> on the full stress configuration; k_eval<materialise> per point
 # of a 2^25-point window, where traffic grows in proportion to the points)
-NCU_SWEEP_DRAM_BYTES = 5_313_792
-NCU_MATERIALISE_DRAM_BYTES_PER_POINT = 1_355_840_944 / (1 << 25)
+NCU_SWEEP_DRAM_BYTES = 7_202_304
+NCU_MATERIALISE_DRAM_BYTES_PER_POINT = 1_372_498_464 / (1 << 25)
 
 
 def parse_args():
@@ -491,7 +491,7 @@ def run_ours(args):
                          "ops_per_point": EXEC_OPS_PER_POINT_SWEEP,
                          "ops_per_point_source": "executed thread-instructions per point of this kernel "
                                                  "(ncu capture on the stress configuration, profiles/)",
-                         "alu_pipe_active_ncu": 0.548, "issue_active_ncu": 0.742,
+                         "alu_pipe_active_ncu": 0.541, "issue_active_ncu": 0.754,
                          "peak_source": "k_int_peak (add+xor chains on both integer pipes) measured in this run"},
             "roofline_hbm": {"bound": "hbm", "kernel": "k_eval<materialise>", "achieved": mat_gbs,
                              "peak": hbm_peak, "unit": "GB/s", "frac": mat_gbs / hbm_peak,
