@@ -64,8 +64,8 @@ bool shape_in_range(const ps_model_shape& s, u32 tp_coll, u32 accum = 1) {
 }
 
 // whether every byte count of a (Theta, Omega, G) triple of this model -- device
-// bytes (at most wsum * (P + 2 unit)) and host bytes (at most (2 accum + 1) * wsum * P)
-// -- stays below 2^53
+// bytes (at most wsum * (P + 2 unit)), host bytes (at most (2 accum + 1) * wsum * P)
+// and data-axis volume (at most (4 accum + 1) * wsum * P) -- stays below 2^53
 bool shape_is_small(const ps_model_shape& s, u32 accum) {
   typedef unsigned __int128 u128;
   const u128 H = s.hidden;
@@ -73,7 +73,7 @@ bool shape_is_small(const ps_model_shape& s, u32 accum) {
                                         : 12 * (u128)s.layers * H * H + (u128)s.vocab * H;
   const u128 unit = s.unit_from_shape ? 12 * H * H : 0;
   const u128 wsum = (u128)s.w_param + s.w_grad + s.w_opt;
-  return (2 * (u128)accum + 1) * wsum * (P + 2 * unit) < ((u128)1 << 53);
+  return (4 * (u128)accum + 1) * wsum * (P + 2 * unit) < ((u128)1 << 53);
 }
 
 int ensure_scratch(ps_ctx* ctx, size_t bytes) {

@@ -46,8 +46,9 @@ struct SpaceDev {
   u32 sstar_units;    // unit buffers a gathered (S*) state holds at a time: 1, or 2 when gathers overlap computation
   u32 accum;          // micro-batches per step (gradient accumulation), >= 1
   u32 all_pow2;       // 1 if every device count of the space is a power of two (then every T, K, D is)
-  u32 all_small;      // 1 if for every model (2 accum + 1) (w_T + w_O + w_G) (P + 2 unit) < 2^53: the device
-                      // and host bytes of a (Theta, Omega, G) triple are then exact in a double
+  u32 all_small;      // 1 if for every model (4 accum + 1) (w_T + w_O + w_G) (P + 2 unit) < 2^53: the device
+                      // bytes, host bytes and data-axis volume of a (Theta, Omega, G) triple are then
+                      // exact in a double
 };
 
 enum : u32 {

@@ -477,7 +477,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
       // multiply-adds) and the integer only if the reduction pass needs it
       if (FAST) mem3_f64[r] = fma((double)ka[r], e2_f64, fma((double)kb[r], sh_f64, (double)kc[r] * u_f64));
       else mem3[r] = mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0)));
-      comm3[r] = mad_small(ub.x, kx[r], 0);
+      if (!FAST) comm3[r] = mad_small(ub.x, kx[r], 0);   // the fast case forms it where it is needed
       bool host_fits = true;                    // the triple's own host bytes against the budget
       if (host_limited) {
         if (FAST) { host3_f64[r] = (double)kh[r] * sh_f64; host_fits = host3_f64[r] < (double)host_x; }
@@ -592,10 +592,23 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
     } else {
       const u64 comm_limit = min(threshold.a, (u64)sh.block_comm_limit);
       const u64 least_axis = tb.c_axis[0];   // tau = 0 sends the smaller boundary tensor; v does not matter
+      if (FAST) {
+        // a triple's volume is below 2^53 here, so it is compared as a double against
+        // what the limit leaves after the axis traffic (exact below 2^53, and above
+        // it every volume passes anyway)
+        const double room = comm_limit >= least_axis ? (double)(comm_limit - least_axis) : -1.0;
+        const double x_f64 = (double)ub.x;
 #pragma unroll
-      for (int r = 0; r < R; ++r) {
-        survivors += n_pass[r];
-        matters = matters || (n_pass[r] != 0 && comm3[r] + least_axis <= comm_limit);
+        for (int r = 0; r < R; ++r) {
+          survivors += n_pass[r];
+          matters = matters || (n_pass[r] != 0 && (double)kx[r] * x_f64 <= room);
+        }
+      } else {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          survivors += n_pass[r];
+          matters = matters || (n_pass[r] != 0 && comm3[r] + least_axis <= comm_limit);
+        }
       }
     }
     if (__any_sync(0xffffffffu, matters)) {
@@ -609,7 +622,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
 #pragma unroll
       for (int r = 0; r < R; ++r) {
         l_mem[r] = FAST ? mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0))) : mem3[r];
-        l_comm[r] = comm3[r];
+        l_comm[r] = FAST ? mad_small(ub.x, kx[r], 0) : comm3[r];
         l_host[r] = (FAST && host_limited) ? mad_small(ub.sh, kh[r], 0) : host3[r];
         l_allowed[r] = allowed[r]; l_triple[r] = t_local[r];
       }
