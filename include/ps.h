@@ -234,8 +234,10 @@ int ps_eval_batch(ps_ctx* ctx, const ps_space* space, uint64_t first, uint64_t c
  * d_out is [n_models][n_caps][max_entries] (device, 8-byte aligned); unused
  * slots are zeroed.  d_counts[n_models][n_caps] (device) receives the true
  * frontier length, or for top-k the number of survivors, even when that
- * exceeds max_entries.  A frontier longer than PS_FRONTIER_INTERNAL inside one
- * warp's share of a model makes ps_status return PS_E_CAPACITY.  n_caps <= 8. */
+ * exceeds max_entries.  A frontier longer than PS_FRONTIER_INTERNAL -- of a
+ * model under the largest capacity, or of the share of it one warp sweeps --
+ * makes ps_status return PS_E_CAPACITY.  n_caps <= 8.  The call may grow the
+ * context's scratch (one partial list per warp of the sweep). */
 int ps_sweep_pareto(ps_ctx* ctx, const ps_space* space, const ps_filter* filter,
                     const uint64_t* caps_bytes /* host */, uint32_t n_caps, uint32_t reduce_kind,
                     uint32_t max_entries, ps_front_entry* d_out, uint32_t* d_counts);
