@@ -229,9 +229,31 @@ __device__ __forceinline__ void topk_append(WarpList& w, bool cand, const Key& k
   __syncwarp();
 }
 
+// Fast case (every degree a power of two): what depends on the model and on the
+// tensor degree alone, or on the pipeline degree alone, for every possible
+// degree 2^s -- built once per block, so that a unit's prologue is a few loads
+// and the shifts by the remaining degrees.
+constexpr int MAX_LOG2_DEGREE = 25;        // device counts are at most 2^24
+struct __align__(16) TensorDegree {
+  u64 E1;        // ceil(P / T): elements of a state on one tensor rank
+  u64 u;         // ceil(unit / T)
+  u64 EA[2];     // ceil(A[v] / T): activations under sequence parallelism
+  u64 UA[2];     // ceil(UA[v] / T)
+  u64 tp_x;      // ring volume of a boundary tensor over T devices
+  u64 sbh_t;     // ceil(Sbh / T)
+  u32 t_heads;   // T divides the head count
+  u32 pad[3];
+};
+struct PipelineDegree {
+  u32 lps;       // ceil(L / K)
+  u32 k_layers;  // K divides the layer count
+};
+
 template <int WARPS>
 struct SweepShared {
   WarpTables tables[WARPS];
+  TensorDegree by_t[MAX_LOG2_DEGREE];
+  PipelineDegree by_k[MAX_LOG2_DEGREE];
   u64 list_a[WARPS * LIST_CAP];
   u64 list_b[WARPS * LIST_CAP];
   u32 list_i[WARPS * LIST_CAP];
@@ -326,6 +348,25 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
     for (int j = tid; j < STAIR; j += THREADS) sh.stair[j] = U64MAX;
   __syncthreads();
   const ModelRec& rec = sh.rec;
+  if (FAST) {
+    for (int sft = tid; sft < MAX_LOG2_DEGREE; sft += THREADS) {
+      TensorDegree t;
+      t.E1 = ceil_shift(rec.P, sft);
+      t.u = ceil_shift(rec.unit, sft);
+      t.EA[0] = ceil_shift(rec.A[0], sft); t.EA[1] = ceil_shift(rec.A[1], sft);
+      t.UA[0] = ceil_shift(rec.UA[0], sft); t.UA[1] = ceil_shift(rec.UA[1], sft);
+      t.tp_x = rec.Sbh - (rec.Sbh >> sft);
+      t.sbh_t = ceil_shift(rec.Sbh, sft);
+      t.t_heads = (rec.heads & ((1u << sft) - 1u)) == 0 ? 1u : 0u;
+      t.pad[0] = t.pad[1] = t.pad[2] = 0;
+      sh.by_t[sft] = t;
+      PipelineDegree k;
+      k.lps = (rec.L + ((1u << sft) - 1u)) >> sft;
+      k.k_layers = (rec.L & ((1u << sft) - 1u)) == 0 ? 1u : 0u;
+      sh.by_k[sft] = k;
+    }
+    __syncthreads();
+  }
 
   WarpTables& tb = sh.tables[warp];
   WarpList list{sh.list_a + warp * LIST_CAP, sh.list_b + warp * LIST_CAP,
@@ -427,14 +468,39 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
   for (u32 unit = u_begin + warp; unit < u_end;) {
     const Fact f = sp.facts[unit];
     const Pow2 p2 = pow2_of(f);
-    const UnitBase ub = (FAST || p2.all) ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
-                               : unit_base(rec, f, sp.tp_max_valid, true);
+    UnitBase ub;
+    if (FAST) {
+      // the tensor and pipeline parts come from the block's tables
+      const TensorDegree& td = sh.by_t[p2.sT];
+      const PipelineDegree kd = sh.by_k[p2.sK];
+      ub.E2 = ceil_shift(td.E1, p2.sK);
+      ub.sh = ceil_shift(ub.E2, p2.sD);
+      ub.x = ub.E2 - (ub.E2 >> p2.sD);
+      ub.u = td.u;
+      ub.tp_x = td.tp_x;
+      ub.sbh_t = td.sbh_t;
+      ub.lps = kd.lps;
+      const bool tp_le = f.T <= sp.tp_max_valid;
+      const bool whole = ((u64)f.T * f.K * f.D == (u64)f.N);
+      u32 cv = (td.t_heads ? PS_F_T_DIV_HEADS : 0) | (kd.k_layers ? PS_F_K_DIV_LAYERS : 0) |
+               (tp_le ? PS_F_TP_LE_MAX : 0) | PS_F_AXIS_FORM;
+      if (td.t_heads && kd.k_layers && tp_le && whole) cv |= PS_F_CV;
+      ub.cv = cv;
+      ub.d1 = (f.D == 1);
+    } else {
+      ub = p2.all ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true) : unit_base(rec, f, sp.tp_max_valid, true);
+    }
     __syncwarp();
     {
       // lane (vt, d): activation bytes of digit d under variant vt, and the bound
       // a triple's own bytes must stay below for the sum to fit the capacity
       ActBase ab;
-      if (FAST || p2.all) {
+      if (FAST) {
+        const TensorDegree& td = sh.by_t[tl_tau == 0 ? p2.sT : 0];     // degree 1 = not sharded
+        ab.EA = td.EA[tl_v];
+        ab.uA = td.UA[tl_v];
+        ab.shA = ceil_shift(ab.EA, p2.sD);
+      } else if (p2.all) {
         const u32 s = tl_tau == 0 ? p2.sT : 0;
         ab.EA = ceil_shift(tl_A, s);
         ab.uA = ceil_shift(tl_UA, s);
