@@ -53,8 +53,8 @@ static inline int sweep_warps(int kind) { return kind == PS_REDUCE_PARETO ? SWEE
 static inline int sweep_blocks_per_sm(int kind) { return kind == PS_REDUCE_PARETO ? SWEEP_BLOCKS_PARETO : SWEEP_BLOCKS_TOPK; }
 #define SWEEP_LIST_CAP 128        /* entries of a warp's list and of a block's partial list */
 #define SWEEP_MAX_CHUNKS 16       /* blocks per model                                        */
-#define MERGE_CAP (11 * SWEEP_LIST_CAP)   /* entries the merge kernel combines at a time: what it
-                                     has kept plus the lists of one block of the sweep       */
+#define MERGE_CAP (5 * SWEEP_LIST_CAP)    /* entries the merge kernel combines at a time: what it
+                                     has kept plus as many of the warps' lists as fit      */
 #define PS_MAX_CAPS 8
 
 struct PartialEntry {

@@ -863,7 +863,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
 // place at home plus, for every other list, the number of entries below it
 // there: binary searches, no sort.  The union is then cut back (top-k: the k
 // smallest; Pareto: entries whose communication is below that of everything
-// before them).  Lists are taken in rounds of MERGE_LISTS beside what has been
+// before them).  Lists are taken in rounds -- as many as fit beside what has been
 // kept so far, so any number can be combined.  Each emitted point is evaluated
 // again from its index (host bytes and flags come from there; mem and comm must
 // agree).
@@ -871,7 +871,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
 #define SWEEP_MERGE_THREADS 128
 #endif
 constexpr int MERGE_THREADS = SWEEP_MERGE_THREADS;
-constexpr int MERGE_LISTS = MERGE_CAP / LIST_CAP - 1;   // lists per round beside the kept entries
+constexpr int MERGE_LISTS = 16;             // most lists a round takes (they are usually far from full)
 
 struct MergeShared {
   u64 in_a[MERGE_CAP], in_b[MERGE_CAP];     // the kept entries, then the round's lists
@@ -879,6 +879,7 @@ struct MergeShared {
   u64 a[MERGE_CAP], b[MERGE_CAP];           // the sorted union; after the cut, the kept entries
   u32 i[MERGE_CAP];
   int off[MERGE_LISTS + 2];                 // start of each list in in_*
+  int taken;                                // lists of this round
   u64 warp_min[MERGE_THREADS / 32];
   int warp_sum[MERGE_THREADS / 32];
   u32 survivors;
@@ -938,17 +939,25 @@ __global__ void __launch_bounds__(MERGE_THREADS) k_sweep_merge(SpaceDev sp, Merg
     if (surv) atomicAdd(&sh.survivors, surv);
   }
   int n_list = 0;                                  // entries kept so far: sh.a/b/i[0, n_list), sorted
-  for (u32 next = 0; next < n_lists; next += MERGE_LISTS) {
-    const int taken = (int)min((u32)MERGE_LISTS, n_lists - next);
-    // list 0 = the kept entries, lists 1..taken = this round's
-    if (tid <= taken + 1) {
-      int off = 0;
-      if (tid >= 1) off = n_list;
-      for (int c = 1; c < tid; ++c) off += min((int)list_n[next + c - 1].x, LIST_CAP);
-      sh.off[tid] = off;
+  for (u32 next = 0; next < n_lists;) {
+    // list 0 = the kept entries, lists 1..taken = as many of the next lists as fit
+    // (at least one does: kept entries and a list are at most LIST_CAP each)
+    if (tid == 0) {
+      int off = n_list, c = 0;
+      sh.off[0] = 0;
+      while (c < MERGE_LISTS && next + c < n_lists) {
+        const int n = min((int)list_n[next + c].x, LIST_CAP);
+        if (off + n > MERGE_CAP) break;
+        sh.off[c + 1] = off;
+        off += n;
+        ++c;
+      }
+      sh.off[c + 1] = off;
+      sh.taken = c;
     }
     for (int p = tid; p < n_list; p += MERGE_THREADS) { sh.in_a[p] = sh.a[p]; sh.in_b[p] = sh.b[p]; sh.in_i[p] = sh.i[p]; }
     __syncthreads();
+    const int taken = sh.taken;
     const int total = sh.off[taken + 1];
     for (int c = 1; c <= taken; ++c) {
       const PartialEntry* src = lists + (u64)(next + c - 1) * LIST_CAP;
@@ -1006,6 +1015,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) k_sweep_merge(SpaceDev sp, Merg
         n_list = LIST_CAP;
       }
     }
+    next += (u32)taken;
     __syncthreads();
   }
   const u32 s_survivors = sh.survivors;
