@@ -57,7 +57,7 @@ BYTES_PER_POINT_MATERIALISE = 36
 # DRAM traffic of one launch from the ncu captures summarised under profiles/
 # (k_sweep<top-k> on the full stress configuration; k_eval<materialise> per point
 # of a 2^25-point window, where traffic grows in proportion to the points)
-NCU_SWEEP_DRAM_BYTES = 6_150_656
+NCU_SWEEP_DRAM_BYTES = 5_968_128
 NCU_MATERIALISE_DRAM_BYTES_PER_POINT = 1_372_498_464 / (1 << 25)
 
 
