@@ -145,9 +145,11 @@ class Context:
         self._h = handle
 
     def close(self):
-        if getattr(self, "_h", None):
+        # at interpreter shutdown the module's globals may be gone before the last
+        # handle: the process is ending, the driver releases the device memory
+        if getattr(self, "_h", None) and _lib is not None:
             _lib.ps_destroy(self._h)
-            self._h = None
+        self._h = None
 
     __del__ = close
 
@@ -212,7 +214,7 @@ class Space:
         self.n_models = len(models)
 
     def close(self):
-        if getattr(self, "_h", None) and getattr(self.ctx, "_h", None):
+        if getattr(self, "_h", None) and getattr(self.ctx, "_h", None) and _lib is not None:
             _lib.ps_space_destroy(self._h)
         self._h = None
 
