@@ -69,6 +69,14 @@ __device__ __forceinline__ u32 digit_mode(u32 modemap, u32 digit) { return (mode
 // the branch is uniform wherever a warp works on one factorisation.
 __device__ __forceinline__ u64 div_floor(u64 a, u32 d) {
   if ((d & (d - 1)) == 0) return a >> (31 - __clz(d));
+  if (a < ((u64)1 << 52)) {
+    // The correctly rounded double quotient is off by less than a half, and never
+    // below an integer the true quotient reaches, so its integer part is the
+    // quotient or one more; the remainder tells which.
+    u64 q = (u64)__double2ll_rz((double)(long long)a / (double)d);
+    if ((long long)(a - q * d) < 0) --q;
+    return q;
+  }
   return a / d;
 }
 __device__ __forceinline__ u64 div_ceil(u64 a, u32 d) { return div_floor(a + (d - 1), d); }
