@@ -303,9 +303,9 @@ int ps_select(ps_ctx* ctx, const ps_select_query* d_queries, uint64_t n, uint32_
  * device-wide synchronisation of cudaFree/cudaMalloc.  ps_eval_batch may do
  * both when its scratch has to grow.  This function never calls cudaMalloc,
  * cudaFree or any allocating routine: its two scratch tables (a survivor count
- * and a prefix sum per group of |mode_mask|^4 consecutive points) sit in a
- * fixed 1.5 MiB array inside the library image, which every GPU that loads the
- * library holds until the process ends.
+ * per group of |mode_mask|^4 consecutive points, and a prefix sum per run of up
+ * to 32 groups) sit in a fixed 1.5 MiB array inside the library image, which
+ * every GPU that loads the library holds until the process ends.
  *
  * Arguments, outputs, order of the survivors and error behaviour are those of
  * ps_eval_batch with a non-null filter (which is required here).  Limits and

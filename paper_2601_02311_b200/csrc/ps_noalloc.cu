@@ -1,7 +1,7 @@
 // ps_eval_compact_noalloc: the filter-and-compact path of ps_eval_batch for
 // callers that must not allocate device memory.  The per-group survivor counts
-// and their prefix sums live in a fixed array that is part of the library image
-// instead of in the context's growable scratch.
+// and the prefix sums over runs of groups live in a fixed array that is part of
+// the library image instead of in the context's growable scratch.
 #include <cuda_runtime.h>
 #include <string.h>
 #include <mutex>
@@ -16,7 +16,8 @@ constexpr size_t COUNT_BYTES = sizeof(u32) * (size_t)PS_NOALLOC_MAX_GROUPS;
 constexpr size_t OFFSET_BYTES = sizeof(u64) * (size_t)PS_NOALLOC_MAX_GROUPS;
 
 // 1.5 MiB on every GPU that loads the library, for the life of the process:
-// [0, COUNT_BYTES) survivor count of each group, then the exclusive prefix sums.
+// [0, COUNT_BYTES) survivor count of each group, then the exclusive prefix sums
+// (one per run of groups, so at most one per group).
 static __device__ __align__(256) unsigned char g_fixed_scratch[COUNT_BYTES + OFFSET_BYTES];
 
 constexpr int MAX_DEVICES = 64;
