@@ -60,3 +60,25 @@ def test_window_is_inside_the_space_and_not_group_aligned():
     first, count = bench.window_of(6_963_200_000, 25)
     assert count == 1 << 25 and first % 625 != 0 and first + count <= 6_963_200_000
     assert bench.window_of(4375, 25) == (0, 4375)
+
+
+def test_reference_arm_prints_the_contract_line():
+    """Rank 0 of the reference arm prints one JSON line with the keys the bench
+    contract names; its value is the oracle's own throughput."""
+    import json
+    env = dict(os.environ, RANK="0", WORLD_SIZE="1")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "1",
+                        "--steps", "1", "--warmup", "1", "--workload", "C3", "--models", "2"],
+                       env=env, capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
+    lines = [ln for ln in r.stdout.splitlines() if ln.strip()]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    for key in ("impl", "metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step",
+                "higher_is_better", "scaling", "vs_baseline", "dtype", "data", "config", "cpu_baseline", "e2e"):
+        assert key in line, key
+    assert line["impl"] == "reference" and line["value"] > 0 and line["vs_baseline"] is None
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["value"] == line["value"]
+    assert line["e2e"] == {"value": line["value"], "unit": line["unit"], "h2d_bytes_per_step": 0,
+                           "d2h_bytes_per_step": 0}
+    assert "workload" in line["config"]
