@@ -53,11 +53,13 @@ UNIT = "evals/s"
 # the real win (it was 86 in the first correct kernel and 11.3 before the kernels
 # were compiled for the cases the space and the filter allow).
 EXEC_OPS_PER_POINT_SWEEP = 7.90
+EXEC_OPS_PER_POINT_PARETO = 10.45     # the same figure for the Pareto sweep
 BYTES_PER_POINT_MATERIALISE = 36
 # DRAM traffic of one launch from the ncu captures summarised under profiles/
 # (k_sweep<top-k> on the full stress configuration; k_eval<materialise> per point
 # of a 2^25-point window, where traffic grows in proportion to the points)
 NCU_SWEEP_DRAM_BYTES = 5_968_128
+NCU_PARETO_DRAM_BYTES = 2_008_320
 NCU_MATERIALISE_DRAM_BYTES_PER_POINT = 1_372_498_464 / (1 << 25)
 
 
@@ -493,6 +495,13 @@ def run_ours(args):
                                                  "(ncu capture on the stress configuration, profiles/)",
                          "alu_pipe_active_ncu": 0.490, "issue_active_ncu": 0.752,
                          "peak_source": "k_int_peak (add+xor chains on both integer pipes) measured in this run"},
+            "roofline_pareto": {"bound": "alu", "kernel": "k_sweep<Pareto> (+ merge)",
+                                "achieved": EXEC_OPS_PER_POINT_PARETO * size / (phase_ms["pareto"] * 1e-3) / 1e12,
+                                "peak": int_peak / 1e12, "unit": "T thread-instructions/s",
+                                "frac": EXEC_OPS_PER_POINT_PARETO * size / (phase_ms["pareto"] * 1e-3) / int_peak,
+                                "traffic": NCU_PARETO_DRAM_BYTES if args.workload == "C4" and args.models is None else None,
+                                "ops_per_point": EXEC_OPS_PER_POINT_PARETO,
+                                "alu_pipe_active_ncu": 0.509, "issue_active_ncu": 0.714},
             "roofline_hbm": {"bound": "hbm", "kernel": "k_eval<materialise>", "achieved": mat_gbs,
                              "peak": hbm_peak, "unit": "GB/s", "frac": mat_gbs / hbm_peak,
                              "traffic": int(NCU_MATERIALISE_DRAM_BYTES_PER_POINT * count),
