@@ -370,3 +370,15 @@ def test_sweeps_around_the_exact_double_limit(ctx, ps, cap):
     filt = dict(require_flags=VALID)
     assert_same_sweep(gs.sweep(filt, [cap], ps.REDUCE_TOPK, 64),
                       os_.sweep(filt, [cap], O.KIND_TOPK, 64, n_threads=8))
+
+
+@pytest.mark.parametrize("host_cap", [0, 8 * synth.GB, 200 * synth.GB])
+def test_topk_with_a_host_budget_on_a_power_of_two_space(ctx, ps, host_cap):
+    """The top-k kernels compiled for a host budget, in the power-of-two case."""
+    space = synth.config("C4", n_models=2)
+    gs, os_ = both(ctx, space)
+    for comm_kind in (O.COMM_PAPER, O.COMM_PAPER_PLUS_EXT):
+        filt = dict(require_flags=VALID, host_cap=host_cap, comm_kind=comm_kind)
+        caps = [80 * synth.GB]
+        assert_same_sweep(gs.sweep(filt, caps, ps.REDUCE_TOPK, 64),
+                          os_.sweep(filt, caps, O.KIND_TOPK, 64, n_threads=8))
