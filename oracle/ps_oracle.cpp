@@ -26,11 +26,17 @@
 // checkpointing); offloaded state lives as shards on the hosts.
 //
 // Pins: tests/test_oracle_pins.py (the paper's printed numbers, closed forms,
-// invariants, Table 2) and tests/test_oracle_vs_sim.py (a brute-force fp64
-// training simulator with explicit shard bookkeeping).  Unpinned against the
-// paper (it prints no such number): the activation formula, the host-link byte
-// counts and the tensor/pipeline traffic -- "parity unpinned" for those three
-// readings; they are pinned only by closed forms and by the simulator.
+// invariants, Table 2), tests/test_oracle_vs_sim.py (a brute-force fp64
+// training simulator with explicit shard bookkeeping) and
+// tests/test_oracle_vs_composition_sim.py (a tensor x pipeline x data grid run
+// of a small network whose rings and stage-to-stage transfers count the bytes
+// they send: pins the tensor- and pipeline-axis traffic, with the number of
+// all-reduces per layer left a parameter).  The paper prints no activation
+// size, no host-link figure and no model-axis volume, so against the paper
+// these three stay readings.  "parity unpinned": the coefficients of the
+// activation formula (34 S b H + 5 a S^2 b; 2 S b H) -- only their wiring into
+// the rules (times L, checkpoint variant, unit = one layer, tensor-axis split)
+// is pinned.
 
 #include <algorithm>
 #include <cstdint>
@@ -211,7 +217,12 @@ OResult eval_point(const ORecord& m, u64 N, u64 T, u64 K, u64 D, int v, int tau,
   if (pi_omega == SG) ext_data += xO;                        // gather Omega for the update
   u64 layers_per_stage = ceil_div(m.L, K);
   u64 ext_tp = layers_per_stage * tp_coll_per_layer * 2 * ring_elems(m.Sbh, T) * m.w_act;
-  u64 ext_pp = (K > 1) ? 2 * ceil_div(m.Sbh, tau == 0 ? T : 1) * m.w_act : 0;
+  // between pipeline stages a device passes on what it holds of the boundary tensor
+  // (all of it, or its 1/T shard under sequence parallelism): an interior stage sends
+  // one forward and one gradient backward, the first and the last stage only one of
+  // the two -- bytes sent by the busiest device, as for the rings (Section 2.3)
+  u64 boundary_sends = (K >= 3) ? 2 : (K == 2 ? 1 : 0);
+  u64 ext_pp = boundary_sends * ceil_div(m.Sbh, tau == 0 ? T : 1) * m.w_act;
   out.comm_ext = ext_data + g * (ext_tp + ext_pp);           // model-axis traffic of every micro-batch
 
   // host-link bytes (mode O): shards live on the hosts

@@ -2,8 +2,8 @@
 
 ``python -m paper_2601_02311_b200.build [--verbose]``
 
-Extra compiler flags (for instance ``-DEVAL_GRID_PER_SM=4`` to try another launch
-shape) can be given in the environment variable ``PS_NVCC_FLAGS``.
+Extra compiler flags (for instance ``-DEVAL_GRID_PER_SM_WRITE=4`` to try another
+launch shape) can be given in the environment variable ``PS_NVCC_FLAGS``.
 """
 from __future__ import annotations
 
@@ -18,7 +18,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libps_b200.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "--use_fast_math", "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared"]
+              "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared"]
 
 
 def sources():

@@ -90,11 +90,14 @@ int ensure_scratch(ps_ctx* ctx, size_t bytes) {
 
 // a kernel-reported problem seen by an earlier status copy
 int pending_device_error(ps_ctx* ctx) {
-  const u32 st = *ctx->h_status;
+  const u32 st = *ctx->h_status & ~(u32)ST_TRUNCATED;     // a truncated frontier blocks nothing
   if (st & ST_LIST_OVERFLOW) return PS_E_CAPACITY;
   if (st) return PS_E_DEVICE;
   return PS_OK;
 }
+
+// flag bits a filter may require
+constexpr u32 KNOWN_FLAGS = (PS_F_PAPER_PRICED << 1) - 1u;
 
 int enqueue_status_copy(ps_ctx* ctx) {
   CUDA_OK(cudaMemcpyAsync(ctx->h_status, ctx->d_status, sizeof(u32), cudaMemcpyDeviceToHost, ctx->stream));
@@ -186,7 +189,8 @@ int ps_status(ps_ctx* ctx) {
   if (!guard.ok) return PS_E_CUDA;
   CUDA_OK(cudaMemcpyAsync(ctx->h_status, ctx->d_status, sizeof(u32), cudaMemcpyDeviceToHost, ctx->stream));
   CUDA_OK(cudaStreamSynchronize(ctx->stream));
-  const int rc = pending_device_error(ctx);
+  int rc = pending_device_error(ctx);
+  if (rc == PS_OK && (*ctx->h_status & ST_TRUNCATED)) rc = PS_E_TRUNCATED;
   if (rc != PS_OK) {
     *ctx->h_status = 0;
     CUDA_OK(cudaMemsetAsync(ctx->d_status, 0, sizeof(u32), ctx->stream));
@@ -363,7 +367,8 @@ int ps_eval_batch(ps_ctx* ctx, const ps_space* sp, uint64_t first, uint64_t coun
   if (!aligned(out.mem, 8) || !aligned(out.comm_paper, 8) || !aligned(out.comm_ext, 8) ||
       !aligned(out.host, 8) || !aligned(out.flags, 4) || !aligned(d_idx_out, 8) || !aligned(d_n_out, 8))
     return PS_E_ALIGN;
-  if (filter && filter->comm_kind > PS_COMM_PAPER_PLUS_EXT) return PS_E_RANGE;
+  if (filter && (filter->comm_kind > PS_COMM_PAPER_PLUS_EXT || (filter->require_flags & ~KNOWN_FLAGS)))
+    return PS_E_RANGE;
   int rc = pending_device_error(ctx);
   if (rc != PS_OK) return rc;
   DeviceGuard guard(ctx->device);
@@ -414,7 +419,7 @@ int ps_sweep_pareto(ps_ctx* ctx, const ps_space* sp, const ps_filter* filter,
   if (n_caps < 1 || n_caps > PS_MAX_CAPS || max_entries < 1) return PS_E_RANGE;
   if (reduce_kind != PS_REDUCE_PARETO && reduce_kind != PS_REDUCE_TOPK) return PS_E_RANGE;
   if (reduce_kind == PS_REDUCE_TOPK && max_entries > PS_TOPK_MAX) return PS_E_RANGE;
-  if (filter->comm_kind > PS_COMM_PAPER_PLUS_EXT) return PS_E_RANGE;
+  if (filter->comm_kind > PS_COMM_PAPER_PLUS_EXT || (filter->require_flags & ~KNOWN_FLAGS)) return PS_E_RANGE;
   if (!aligned(d_out, 8) || !aligned(d_counts, 4)) return PS_E_ALIGN;
   int rc = pending_device_error(ctx);
   if (rc != PS_OK) return rc;

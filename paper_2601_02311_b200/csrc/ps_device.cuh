@@ -187,14 +187,17 @@ __device__ __forceinline__ ActBase act_base_pow2(const ModelRec& r, const Pow2& 
 
 // tensor-axis and pipeline-axis traffic per step (not priced by Theorem 2):
 // per layer of a stage, tp_coll all-reduces of a boundary tensor over T
-// devices; one boundary tensor forward and one backward between stages; all of
-// it once per micro-batch (accum micro-batches per step)
+// devices; between stages the boundary tensor goes forward and its gradient
+// comes back, so the busiest device sends two of them when it has a neighbour on
+// either side (K >= 3) and one when there are two stages; all of it once per
+// micro-batch (accum micro-batches per step)
 __device__ __forceinline__ u64 model_axis_traffic(const ModelRec& r, const Fact& f,
                                                   const UnitBase& b, u32 tau, u32 tp_coll,
                                                   u32 accum = 1) {
   const u32 per_elem = 2 * tp_coll * r.wA;                 // <= 2 * 64 * 16
   const u64 tp = b.tp_x * (u64)(b.lps * per_elem);         // lps <= 2^10
-  const u64 pp = (f.K > 1) ? (tau == 0 ? b.sbh_t : r.Sbh) * (u64)(2 * r.wA) : 0;
+  const u32 sends = f.K >= 3 ? 2u : f.K - 1;                // K >= 1
+  const u64 pp = (tau == 0 ? b.sbh_t : r.Sbh) * (u64)(sends * r.wA);
   return (tp + pp) * accum;
 }
 
@@ -297,5 +300,6 @@ __device__ __forceinline__ LocalPoint decode_local(const SpaceDev& sp, u32 lidx)
 enum : u32 {
   ST_BAD_SHAPE = 1u << 0,      // a model shape outside the supported ranges
   ST_LIST_OVERFLOW = 1u << 1,  // a per-warp or per-block list was too short
-  ST_SELF_CHECK = 1u << 2      // an emitted entry did not re-evaluate to itself
+  ST_SELF_CHECK = 1u << 2,     // an emitted entry did not re-evaluate to itself
+  ST_TRUNCATED = 1u << 3       // a frontier was longer than the caller's max_entries (a notice, not a fault)
 };

@@ -1034,9 +1034,12 @@ __global__ void __launch_bounds__(MERGE_THREADS) k_sweep_merge(SpaceDev sp, Merg
     }
     const u32 cap_slot = (KIND == PS_REDUCE_PARETO) ? ci : args.cap_index;
     ps_front_entry* out = args.out + ((u64)model * args.n_caps_total + cap_slot) * args.max_entries;
-    if (tid == 0)
+    if (tid == 0) {
       args.counts[(u64)model * args.n_caps_total + cap_slot] =
           (KIND == PS_REDUCE_PARETO) ? (u32)n_cap : s_survivors;
+      // a frontier that does not fit the caller's rows: its head is written, the count is the true one
+      if (KIND == PS_REDUCE_PARETO && n_cap > (int)args.max_entries) atomicOr(args.status, ST_TRUNCATED);
+    }
     const int n_emit = min(min(n_cap, (int)args.max_entries), KIND == PS_REDUCE_PARETO ? n_cap : (int)args.k_keep);
     for (int p = tid; p < (int)args.max_entries; p += MERGE_THREADS) {
       ps_front_entry e;

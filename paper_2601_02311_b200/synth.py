@@ -182,17 +182,19 @@ def ragged_space(seed: int, n_models: int = 3) -> dict:
 
 
 def select_queries(n: int, seed: int) -> np.ndarray:
-    """Queries for the batched Algorithm 1 as an (n, 8) uint64 array: P, layer
-    elements (12 H^2 of a shape with that many parameters, roughly), device bytes
-    in {16, 24, 40, 80, 141, 192} GB, N a power of two up to 2^14 (or an odd
-    count now and then), byte widths 2/2/12, fast interconnect or not."""
+    """Queries for the batched Algorithm 1 as an (n, 8) uint64 array: parameter
+    count P (a mantissa in [1, 10) times a power of ten between 1e8 and 1e12),
+    elements of one layer (a fraction of P between 1/160 and 1/12, or 0 now and
+    then), device bytes in {16, 24, 40, 80, 141, 192} GB, N a power of two up to
+    2^14 (or an odd count now and then), byte widths 2/2/12, fast interconnect or
+    not.  Both sizes are drawn, not derived from a shape."""
     rng = SplitMix64(seed)
     out = np.zeros((n, 8), dtype=np.uint64)
     for i in range(n):
+        params = rng.uniform(1000, 9999) * 10 ** rng.uniform(5, 9)
         layers = rng.uniform(12, 160)
-        hidden = 128 * rng.uniform(6, 256)
-        out[i, 0] = 12 * layers * hidden * hidden + rng.uniform(32000, 256000) * hidden
-        out[i, 1] = 12 * hidden * hidden if rng.next() % 8 else 0
+        out[i, 0] = params
+        out[i, 1] = params // layers if rng.next() % 8 else 0
         out[i, 2] = rng.choice([16, 24, 40, 80, 141, 192]) * GB
         out[i, 3] = (1 << rng.uniform(0, 14)) if rng.next() % 6 else rng.uniform(1, 3000)
         out[i, 4], out[i, 5], out[i, 6] = 2, 2, 12
