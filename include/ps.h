@@ -52,11 +52,11 @@ enum {
   PS_E_ALIGN = -2,         /* a device pointer is not aligned to its element     */
   PS_E_RANGE = -3,         /* a size, shape or count is outside the stated range */
   PS_E_BADINDEX = -4,      /* [first, first+count) leaves the space              */
-  PS_E_TRUNCATED = -5,     /* an output held fewer entries than were found       */
+  PS_E_TRUNCATED = -5,     /* a notice from ps_status: some Pareto frontier was longer than
+                              max_entries (its head was written, d_counts is true)    */
   PS_E_CUDA = -6,          /* a CUDA runtime call failed                          */
   PS_E_UNIMPLEMENTED = -7,
   PS_E_DEVICE = -8,        /* a kernel reported an inconsistency (status word)   */
-  PS_E_CAPACITY = -9,      /* an internal fixed-size list overflowed             */
   PS_E_NOALLOC_LIMIT = -10 /* the window is too large for ps_eval_compact_noalloc's
                               fixed scratch array (PS_NOALLOC_MAX_GROUPS groups)  */
 };
@@ -94,7 +94,8 @@ enum { PS_REDUCE_PARETO = 0, PS_REDUCE_TOPK = 1 };
 
 #define PS_NO_LIMIT UINT64_MAX
 #define PS_TOPK_MAX 64           /* largest max_entries of a top-k sweep            */
-#define PS_FRONTIER_INTERNAL 128 /* longest frontier one warp or one block can hold */
+#define PS_FRONTIER_FAST 128     /* a model whose frontier (or the part of it one warp of the
+                                    sweep finds) is longer is reduced by a slow exact path */
 
 /* ------------------------------------------------------------------ types */
 typedef struct ps_ctx ps_ctx;     /* opaque: device, borrowed stream, scratch memory      */
@@ -234,9 +235,11 @@ int ps_eval_batch(ps_ctx* ctx, const ps_space* space, uint64_t first, uint64_t c
  * d_out is [n_models][n_caps][max_entries] (device, 8-byte aligned); unused
  * slots are zeroed.  d_counts[n_models][n_caps] (device) receives the true
  * frontier length, or for top-k the number of survivors, even when that
- * exceeds max_entries.  A frontier longer than PS_FRONTIER_INTERNAL -- of a
- * model under the largest capacity, or of the share of it one warp sweeps --
- * makes ps_status return PS_E_CAPACITY.  n_caps <= 8.  The call may grow the
+ * exceeds max_entries; a Pareto frontier longer than max_entries also makes the
+ * next ps_status return PS_E_TRUNCATED once (a notice: the head of the frontier
+ * was written and later calls are not affected).  Frontiers of any length are
+ * exact; one longer than PS_FRONTIER_FAST is computed by a slow path (one pass
+ * over the model's points per entry).  n_caps <= 8.  The call may grow the
  * context's scratch (one partial list per warp of the sweep). */
 int ps_sweep_pareto(ps_ctx* ctx, const ps_space* space, const ps_filter* filter,
                     const uint64_t* caps_bytes /* host */, uint32_t n_caps, uint32_t reduce_kind,

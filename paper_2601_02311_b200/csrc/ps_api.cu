@@ -91,7 +91,6 @@ int ensure_scratch(ps_ctx* ctx, size_t bytes) {
 // a kernel-reported problem seen by an earlier status copy
 int pending_device_error(ps_ctx* ctx) {
   const u32 st = *ctx->h_status & ~(u32)ST_TRUNCATED;     // a truncated frontier blocks nothing
-  if (st & ST_LIST_OVERFLOW) return PS_E_CAPACITY;
   if (st) return PS_E_DEVICE;
   return PS_OK;
 }
@@ -111,7 +110,7 @@ u32 pick_chunks(const ps_ctx* ctx, const ps_space* sp, int kind) {
   // twice (Pareto, whose blocks are fewer and longer).
   const u64 waves = kind == PS_REDUCE_PARETO ? 2 : 1;
   const u64 target = (u64)ctx->sm_count * sweep_blocks_per_sm(kind) * waves;
-  u64 c = (target + sp->dev.n_models - 1) / sp->dev.n_models;
+  u64 c = (target + sp->dev.n_models / 2) / sp->dev.n_models;       // to the nearest: one block too few is cheaper than a second list
   if (c < 1) c = 1;
   if (c > SWEEP_MAX_CHUNKS) c = SWEEP_MAX_CHUNKS;
   const u64 by_units = (sp->dev.n_facts + sweep_warps(kind) - 1) / sweep_warps(kind);   // a unit per warp at least
@@ -135,7 +134,6 @@ const char* ps_strerror(int code) {
     case PS_E_CUDA: return "a CUDA runtime call failed";
     case PS_E_UNIMPLEMENTED: return "not implemented";
     case PS_E_DEVICE: return "a kernel reported an inconsistency";
-    case PS_E_CAPACITY: return "an internal fixed-size list overflowed";
     case PS_E_NOALLOC_LIMIT:
       return "the window needs more scratch than the no-allocation entry point's fixed array holds";
     default: return "unknown error";
@@ -445,6 +443,8 @@ int ps_sweep_pareto(ps_ctx* ctx, const ps_space* sp, const ps_filter* filter,
   m.partial = s.partial;
   m.partial_n = s.partial_n;
   m.n_lists = n_chunks * sweep_warps((int)reduce_kind);
+  m.host_cap = filter->host_cap;
+  m.require_flags = s.require_flags;
   m.n_caps_total = n_caps;
   m.max_entries = max_entries;
   m.k_keep = s.k_keep;
@@ -456,6 +456,7 @@ int ps_sweep_pareto(ps_ctx* ctx, const ps_space* sp, const ps_filter* filter,
     u64 cap_max = 0;
     for (u32 c = 0; c < n_caps; ++c) { m.caps[c] = caps_bytes[c]; if (caps_bytes[c] > cap_max) cap_max = caps_bytes[c]; }
     s.cap_max = cap_max;
+    m.cap_max = cap_max;
     m.n_caps = n_caps;
     CUDA_OK(launch_sweep(PS_REDUCE_PARETO, sp->dev, s, n_chunks, ctx->stream));
     CUDA_OK(launch_sweep_merge(PS_REDUCE_PARETO, sp->dev, m, ctx->stream));
@@ -465,6 +466,7 @@ int ps_sweep_pareto(ps_ctx* ctx, const ps_space* sp, const ps_filter* filter,
       m.caps[0] = caps_bytes[c];
       m.n_caps = 1;
       m.cap_index = c;
+      m.cap_max = caps_bytes[c];
       CUDA_OK(launch_sweep(PS_REDUCE_TOPK, sp->dev, s, n_chunks, ctx->stream));
       CUDA_OK(launch_sweep_merge(PS_REDUCE_TOPK, sp->dev, m, ctx->stream));
     }

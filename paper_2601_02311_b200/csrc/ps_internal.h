@@ -32,16 +32,18 @@ struct ps_space {
 
 // ---- sweep
 // Block shapes of the sweep: warps per block and the resident blocks per SM the
-// kernel is compiled for (which caps its registers).  The top-k sweep is fastest
-// with five blocks of four warps (96 registers): many resident warps, few and
-// long lists per model.  The Pareto sweep is fastest with two blocks of ten
-// warps (96 registers): its warps share a block's coarse staircase, so larger
-// blocks reject more candidates early.
+// kernel is compiled for (which caps its registers at 96 either way: 21 warps fit
+// an SM).  The top-k sweep is fastest with seven blocks of three warps: many
+// resident blocks (1036 at a time, so that a thousand models run as one wave and
+// four thousand as four full ones), few and long lists per model.  The Pareto
+// sweep is fastest with two blocks of ten warps: its warps share a block's coarse
+// staircase, so larger blocks reject more candidates early (3 x 7, 4 x 5 and 7 x 3
+// were 4 to 30 % slower).
 #ifndef SWEEP_WARPS_TOPK
-#define SWEEP_WARPS_TOPK 4
+#define SWEEP_WARPS_TOPK 3
 #endif
 #ifndef SWEEP_BLOCKS_TOPK
-#define SWEEP_BLOCKS_TOPK 5
+#define SWEEP_BLOCKS_TOPK 7
 #endif
 #ifndef SWEEP_WARPS_PARETO
 #define SWEEP_WARPS_PARETO 10
@@ -78,6 +80,8 @@ struct MergeArgs {
   const PartialEntry* partial;
   const uint2* partial_n;
   u64 caps[PS_MAX_CAPS];
+  u64 cap_max, host_cap;  // the filter again, for the slow exact path
+  u32 require_flags;
   u32 n_lists;          // partial lists per model: blocks per model x warps per block
   u32 n_caps;           // capacities this launch emits
   u32 n_caps_total;     // capacities of the output layout

@@ -71,7 +71,7 @@ extern "C" int ps_eval_compact_noalloc(ps_ctx* ctx, const ps_space* sp, uint64_t
   if (filter->comm_kind > PS_COMM_PAPER_PLUS_EXT || (filter->require_flags & ~((PS_F_PAPER_PRICED << 1) - 1u)))
     return PS_E_RANGE;
   const u32 seen = *ctx->h_status & ~(u32)ST_TRUNCATED;   // a kernel-reported problem of an earlier call
-  if (seen) return (seen & ST_LIST_OVERFLOW) ? PS_E_CAPACITY : PS_E_DEVICE;
+  if (seen) return PS_E_DEVICE;
   CurrentDevice guard(ctx->device);
   if (!guard.ok) return PS_E_CUDA;
   if (count == 0) {

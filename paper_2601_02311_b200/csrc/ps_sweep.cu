@@ -17,14 +17,16 @@
 // and inserts the few that pass warp-cooperatively.  A warp that has run out of
 // units writes its list to global scratch and is done -- the warps of a block
 // never wait for one another; k_sweep_merge combines the partial lists of a
-// model (one block per model: sort, prune) and emits entries, re-evaluating
-// each emitted point from its index as a self-check.
+// model (one block per model: rank merge, prune) and emits entries,
+// re-evaluating each emitted point from its index as a self-check.  A frontier
+// that outgrows a list is handed to a slow exact path in the merge kernel.
 #include "ps_device.cuh"
 #include "ps_internal.h"
 
 namespace {
 
 constexpr int LIST_CAP = SWEEP_LIST_CAP;       // entries per warp list / per partial list
+constexpr u32 LIST_OVERFLOWED = 0xffffffffu;   // length of a partial list whose staircase outgrew LIST_CAP
 constexpr u64 U64MAX = ~0ull;
 
 // per-warp tables, rebuilt for every unit: what depends on the activation
@@ -62,6 +64,7 @@ struct WarpList {
   u64* b;
   u32* i;
   int n;
+  int over;   // Pareto: the staircase outgrew the list (the merge kernel then takes the slow exact path)
 };
 
 // Pareto staircase: a = mem ascending, b = comm strictly descending.
@@ -84,7 +87,7 @@ __device__ __forceinline__ void stair_publish(unsigned long long* stair, u64 m, 
 // warp-cooperative insertion; all lanes hold the same (m, c, idx).  Entries are
 // handled 32 at a time, so a short staircase (the usual case) takes one round.
 __device__ __noinline__ void pareto_insert(WarpList& w, u64 m, u64 c, u32 idx, int lane,
-                                           u32* status, unsigned long long* stair) {
+                                           unsigned long long* stair) {
   constexpr int PER = LIST_CAP / 32;
   const int rounds = (w.n + 31) >> 5;
   u64 ea[PER], eb[PER];
@@ -112,7 +115,7 @@ __device__ __noinline__ void pareto_insert(WarpList& w, u64 m, u64 c, u32 idx, i
   if (__any_sync(0xffffffffu, dominated)) { __syncwarp(); return; }
   const int n_new = w.n - killed + 1;
   if (n_new > LIST_CAP) {
-    if (lane == 0) atomicOr(status, ST_LIST_OVERFLOW);
+    w.over = 1;
     return;
   }
   __syncwarp();
@@ -370,7 +373,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
 
   WarpTables& tb = sh.tables[warp];
   WarpList list{sh.list_a + warp * LIST_CAP, sh.list_b + warp * LIST_CAP,
-                sh.list_i + warp * LIST_CAP, 0};
+                sh.list_i + warp * LIST_CAP, 0, 0};
   const int k_keep = (int)args.k_keep;
   Key threshold{U64MAX, U64MAX, 0xffffffffu};
   u32 survivors = 0;
@@ -707,8 +710,13 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
         __syncwarp();
       }
 
+      // Variants in an order in which later ones seldom beat earlier ones (the result
+      // does not depend on the order, the work does): the tensor axis that shards
+      // activations first, and full checkpointing before stored activations -- fewer
+      // bytes at the same communication.
 #pragma unroll 1
-      for (u32 vt = 0; vt < nvt; ++vt) {
+      for (u32 vt_step = 0; vt_step < nvt; ++vt_step) {
+        const u32 vt = (sp.nv - 1 - vt_step % sp.nv) * sp.nt + vt_step / sp.nv;
         const u64 c_axis = tb.c_axis[vt], host_bound = tb.host_bound[vt];
         const u32 vt_first = unit_first + vt * NC;
         // every point of (triple, variant): digit d is a survivor if the triple's
@@ -766,7 +774,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
                 const u64 pm = __shfl_sync(0xffffffffu, m, src);
                 const u64 pc = __shfl_sync(0xffffffffu, c, src);
                 const u32 pi = __shfl_sync(0xffffffffu, idx, src);
-                pareto_insert(list, pm, pc, pi, lane, args.status, sh.stair);
+                pareto_insert(list, pm, pc, pi, lane, sh.stair);
               }
             }
           }
@@ -815,9 +823,11 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
             list.n += (int)total;
             __syncwarp();
           } else {
-            // does not fit in one go: one (triple round, digit) at a time, compacting as needed
+            // does not fit in one go: one (triple round, digit) at a time, compacting as
+            // needed; digits downwards, because the higher modes (offloaded, recomputed,
+            // sharded) keep fewer activation bytes, so that what comes later seldom gets in
 #pragma unroll 1
-            for (u32 d = 0; d < (u32)NM; ++d) {
+            for (int d = NM - 1; d >= 0; --d) {
               const u64 am = tb.act[vt][d];
 #pragma unroll 1
               for (int r = 0; r < R; ++r) {
@@ -851,7 +861,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
     e.a = list.a[p]; e.b = list.b[p]; e.i = list.i[p]; e.pad = 0;
     dst[p] = e;
   }
-  if (lane == 0) args.partial_n[slot] = make_uint2((u32)list.n, survivors);
+  if (lane == 0) args.partial_n[slot] = make_uint2(list.over ? LIST_OVERFLOWED : (u32)list.n, survivors);
 }
 
 // ------------------------------------------------------------------ merge + emit
@@ -867,19 +877,32 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
 // kept so far, so any number can be combined.  Each emitted point is evaluated
 // again from its index (host bytes and flags come from there; mem and comm must
 // agree).
+//
+// A frontier with more than LIST_CAP entries -- in one warp's share of a model
+// or after merging -- does not fit these lists.  The block then computes the
+// model's frontier by the definition instead, one entry per pass over the
+// model's points: the next entry is the survivor with the fewest bytes among
+// those with more bytes and less communication than the last entry (fewest
+// communication, then smallest index, on ties).  Slow (passes = frontier
+// length), bounded memory, any length.
 #ifndef SWEEP_MERGE_THREADS
 #define SWEEP_MERGE_THREADS 128
 #endif
 constexpr int MERGE_THREADS = SWEEP_MERGE_THREADS;
 constexpr int MERGE_LISTS = 16;             // most lists a round takes (they are usually far from full)
+constexpr int MERGE_MAX_LISTS = SWEEP_MAX_CHUNKS * (SWEEP_WARPS_PARETO > SWEEP_WARPS_TOPK ? SWEEP_WARPS_PARETO : SWEEP_WARPS_TOPK);
 
 struct MergeShared {
+  Key pass_best[MERGE_THREADS / 32];        // slow path: the warps' best candidates of a pass
   u64 in_a[MERGE_CAP], in_b[MERGE_CAP];     // the kept entries, then the round's lists
   u32 in_i[MERGE_CAP];
   u64 a[MERGE_CAP], b[MERGE_CAP];           // the sorted union; after the cut, the kept entries
   u32 i[MERGE_CAP];
   int off[MERGE_LISTS + 2];                 // start of each list in in_*
+  int from[MERGE_LISTS + 1];                // which of the model's lists sits there
   int taken;                                // lists of this round
+  int next;                                 // first list the next round looks at
+  unsigned short len[MERGE_MAX_LISTS];      // entries of every list of the model
   u64 warp_min[MERGE_THREADS / 32];
   int warp_sum[MERGE_THREADS / 32];
   u32 survivors;
@@ -922,6 +945,73 @@ __device__ __forceinline__ int block_excl_sum(int mine, int* warp_sum, int tid, 
   return before + incl - mine;
 }
 
+// one point of a model from its index, as an output entry; the objective is returned through *comm
+__device__ __forceinline__ PointOut eval_local(const SpaceDev& sp, const ModelRec& rec, u32 lidx) {
+  const LocalPoint lp = decode_local(sp, lidx);
+  const Fact f = sp.facts[lp.unit];
+  return eval_point(rec, f, lp.v, lp.tau, digit_mode(sp.modemap, lp.dth), digit_mode(sp.modemap, lp.dom),
+                    digit_mode(sp.modemap, lp.dgr), digit_mode(sp.modemap, lp.dac), sp.tp_max_valid,
+                    sp.tp_coll, true, sp.sstar_units, sp.accum);
+}
+
+// The slow exact path for a model whose frontier outgrew the lists: see above.
+__device__ __noinline__ void frontier_by_definition(const SpaceDev& sp, const MergeArgs& args, u32 model,
+                                                    const ModelRec& rec, MergeShared& sh) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  u32 found[PS_MAX_CAPS];
+  for (u32 ci = 0; ci < PS_MAX_CAPS; ++ci) found[ci] = 0;
+  u64 last_mem = 0, last_comm = U64MAX;
+  bool have_last = false;
+  const u32 ppm = (u32)sp.ppm;
+  for (u32 pass = 0; pass <= ppm; ++pass) {             // a frontier has at most ppm entries
+    Key best{U64MAX, U64MAX, 0xffffffffu};
+    for (u32 lidx = tid; lidx < ppm; lidx += MERGE_THREADS) {
+      const PointOut po = eval_local(sp, rec, lidx);
+      const u64 comm = args.comm_kind == PS_COMM_PAPER ? po.comm_paper : po.comm_paper + po.comm_ext;
+      const bool survivor = po.mem <= args.cap_max && po.host <= args.host_cap &&
+                            (po.flags & args.require_flags) == args.require_flags;
+      const bool beyond = !have_last || (po.mem > last_mem && comm < last_comm);
+      const Key key{po.mem, comm, lidx};
+      if (survivor && beyond && key_less(key, best)) best = key;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const Key other = key_shfl_xor(best, o);
+      if (key_less(other, best)) best = other;
+    }
+    if (lane == 0) sh.pass_best[warp] = best;
+    __syncthreads();
+    best = sh.pass_best[0];
+    for (int w = 1; w < MERGE_THREADS / 32; ++w)
+      if (key_less(sh.pass_best[w], best)) best = sh.pass_best[w];
+    __syncthreads();
+    if (best.i == 0xffffffffu) break;                   // nothing beyond the last entry: done
+    for (u32 ci = 0; ci < args.n_caps; ++ci) {
+      if (best.a > args.caps[ci]) continue;
+      const u32 slot = found[ci]++;
+      if (slot < args.max_entries && tid == 0) {
+        const PointOut po = eval_local(sp, rec, best.i);
+        ps_front_entry e;
+        e.mem = po.mem; e.comm = best.b; e.host = po.host;
+        e.idx = (u64)model * sp.ppm + best.i;
+        e.flags = po.flags | PS_F_FEASIBLE; e.pad = 0;
+        args.out[((u64)model * args.n_caps_total + ci) * args.max_entries + slot] = e;
+      }
+    }
+    last_mem = best.a; last_comm = best.b; have_last = true;
+  }
+  for (u32 ci = 0; ci < args.n_caps; ++ci) {
+    ps_front_entry* out = args.out + ((u64)model * args.n_caps_total + ci) * args.max_entries;
+    ps_front_entry zero;
+    zero.mem = 0; zero.comm = 0; zero.host = 0; zero.idx = 0; zero.flags = 0; zero.pad = 0;
+    for (u32 p = found[ci] + tid; p < args.max_entries; p += MERGE_THREADS) out[p] = zero;
+    if (tid == 0) {
+      args.counts[(u64)model * args.n_caps_total + ci] = found[ci];
+      if (found[ci] > args.max_entries) atomicOr(args.status, ST_TRUNCATED);
+    }
+  }
+}
+
 template <int KIND>
 __global__ void __launch_bounds__(MERGE_THREADS) k_sweep_merge(SpaceDev sp, MergeArgs args) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -933,34 +1023,45 @@ __global__ void __launch_bounds__(MERGE_THREADS) k_sweep_merge(SpaceDev sp, Merg
   const PartialEntry* lists = args.partial + (u64)model * n_lists * LIST_CAP;
   if (tid == 0) sh.survivors = 0;
   __syncthreads();
+  bool overflowed = false;
   {
     u32 surv = 0;
-    for (u32 l = tid; l < n_lists; l += MERGE_THREADS) surv += list_n[l].y;
+    for (u32 l = tid; l < n_lists; l += MERGE_THREADS) {
+      const uint2 ln = list_n[l];
+      surv += ln.y;
+      overflowed = overflowed || ln.x == LIST_OVERFLOWED;
+      sh.len[l] = (unsigned short)min(ln.x, (u32)LIST_CAP);
+    }
     if (surv) atomicAdd(&sh.survivors, surv);
   }
+  overflowed = __syncthreads_or(overflowed) != 0;
   int n_list = 0;                                  // entries kept so far: sh.a/b/i[0, n_list), sorted
-  for (u32 next = 0; next < n_lists;) {
-    // list 0 = the kept entries, lists 1..taken = as many of the next lists as fit
-    // (at least one does: kept entries and a list are at most LIST_CAP each)
+  for (u32 next = 0; next < n_lists && !overflowed;) {
+    // list 0 = the kept entries, lists 1..taken = as many of the next non-empty lists as
+    // fit (at least one does: kept entries and a list are at most LIST_CAP each)
     if (tid == 0) {
       int off = n_list, c = 0;
+      u32 l = next;
       sh.off[0] = 0;
-      while (c < MERGE_LISTS && next + c < n_lists) {
-        const int n = min((int)list_n[next + c].x, LIST_CAP);
+      for (; c < MERGE_LISTS && l < n_lists; ++l) {
+        const int n = sh.len[l];
+        if (n == 0) continue;
         if (off + n > MERGE_CAP) break;
         sh.off[c + 1] = off;
+        sh.from[c + 1] = (int)l;
         off += n;
         ++c;
       }
       sh.off[c + 1] = off;
       sh.taken = c;
+      sh.next = (int)l;
     }
     for (int p = tid; p < n_list; p += MERGE_THREADS) { sh.in_a[p] = sh.a[p]; sh.in_b[p] = sh.b[p]; sh.in_i[p] = sh.i[p]; }
     __syncthreads();
     const int taken = sh.taken;
     const int total = sh.off[taken + 1];
     for (int c = 1; c <= taken; ++c) {
-      const PartialEntry* src = lists + (u64)(next + c - 1) * LIST_CAP;
+      const PartialEntry* src = lists + (u64)sh.from[c] * LIST_CAP;
       const int base = sh.off[c], n = sh.off[c + 1] - base;
       for (int p = tid; p < n; p += MERGE_THREADS) {
         const PartialEntry e = src[p];
@@ -1010,17 +1111,18 @@ __global__ void __launch_bounds__(MERGE_THREADS) k_sweep_merge(SpaceDev sp, Merg
       for (int k = 0; k < nk; ++k)
         if (offset + k < MERGE_CAP) { sh.a[offset + k] = keep[k].a; sh.b[offset + k] = keep[k].b; sh.i[offset + k] = keep[k].i; }
       n_list = kept_total;
-      if (n_list > LIST_CAP) {
-        if (tid == 0) atomicOr(args.status, ST_LIST_OVERFLOW);
-        n_list = LIST_CAP;
-      }
+      if (n_list > LIST_CAP) overflowed = true;      // the same for every thread
     }
-    next += (u32)taken;
+    next = (u32)sh.next;
     __syncthreads();
   }
   const u32 s_survivors = sh.survivors;
 
   const ModelRec rec = sp.recs[model];
+  if (KIND == PS_REDUCE_PARETO && overflowed) {
+    frontier_by_definition(sp, args, model, rec, sh);
+    return;
+  }
   for (u32 ci = 0; ci < args.n_caps; ++ci) {
     const u64 cap = args.caps[ci];
     // Pareto: a tighter capacity keeps the head of the staircase (dominance only
@@ -1046,12 +1148,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) k_sweep_merge(SpaceDev sp, Merg
       e.mem = 0; e.comm = 0; e.host = 0; e.idx = 0; e.flags = 0; e.pad = 0;
       if (p < n_emit) {
         const u32 lidx = sh.i[p];
-        const LocalPoint lp = decode_local(sp, lidx);
-        const Fact f = sp.facts[lp.unit];
-        const PointOut po = eval_point(rec, f, lp.v, lp.tau, digit_mode(sp.modemap, lp.dth),
-                                       digit_mode(sp.modemap, lp.dom), digit_mode(sp.modemap, lp.dgr),
-                                       digit_mode(sp.modemap, lp.dac), sp.tp_max_valid, sp.tp_coll, true,
-                                       sp.sstar_units, sp.accum);
+        const PointOut po = eval_local(sp, rec, lidx);
         const u64 comm = args.comm_kind == PS_COMM_PAPER ? po.comm_paper : po.comm_paper + po.comm_ext;
         const u64 list_mem = (KIND == PS_REDUCE_PARETO) ? sh.a[p] : sh.b[p];
         const u64 list_comm = (KIND == PS_REDUCE_PARETO) ? sh.b[p] : sh.a[p];

@@ -22,8 +22,8 @@ _lib = C.CDLL(LIB_PATH)
 
 # ---- constants of ps.h
 OK = 0
-E_NULLPTR, E_ALIGN, E_RANGE, E_BADINDEX, E_TRUNCATED, E_CUDA, E_UNIMPLEMENTED, E_DEVICE, E_CAPACITY = \
-    -1, -2, -3, -4, -5, -6, -7, -8, -9
+E_NULLPTR, E_ALIGN, E_RANGE, E_BADINDEX, E_TRUNCATED, E_CUDA, E_UNIMPLEMENTED, E_DEVICE = \
+    -1, -2, -3, -4, -5, -6, -7, -8
 E_NOALLOC_LIMIT = -10
 NOALLOC_MAX_GROUPS = 131072
 F_GI, F_SC, F_CV, F_FEASIBLE = 1, 2, 4, 8
@@ -156,8 +156,14 @@ class Context:
     def status(self) -> int:
         return _lib.ps_status(self._h)
 
-    def check_status(self):
-        _check(self.status(), "ps_status")
+    def check_status(self, allow_truncated: bool = False) -> int:
+        """Synchronise and raise on any error a kernel reported.  With
+        ``allow_truncated`` the notice that a frontier was longer than the caller's
+        rows (E_TRUNCATED: heads written, counts true) is returned instead of raised."""
+        rc = self.status()
+        if not (allow_truncated and rc == E_TRUNCATED):
+            _check(rc, "ps_status")
+        return rc
 
     def space(self, space: dict) -> "Space":
         return Space(self, space)
@@ -317,7 +323,7 @@ class Space:
         """Returns (entries[n_models, n_caps, max_entries] structured, counts[n_models, n_caps])."""
         d_out, d_counts = self.alloc_sweep(len(caps), max_entries)
         self.sweep_into(filt, caps, kind, max_entries, d_out, d_counts)
-        self.ctx.check_status()
+        self.last_sweep_status = self.ctx.check_status(allow_truncated=True)
         entries = d_out.cpu().numpy().view(ENTRY_DTYPE).reshape(self.n_models, len(caps), max_entries)
         counts = d_counts.cpu().numpy().view(np.uint32).reshape(self.n_models, len(caps))
         return entries, counts

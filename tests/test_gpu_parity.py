@@ -173,6 +173,10 @@ def test_pareto_many_caps_unsorted_and_truncated(ctx, ps):
     want = os_.sweep(filt, caps, O.KIND_PARETO, 3, n_threads=8)
     assert want[1].max() > 3
     assert_same_sweep(got, want)
+    assert gs.last_sweep_status == ps.E_TRUNCATED          # the notice; the next call is not blocked
+    got = gs.sweep(filt, caps, ps.REDUCE_PARETO, 64)
+    assert gs.last_sweep_status == ps.OK
+    assert_same_sweep(got, os_.sweep(filt, caps, O.KIND_PARETO, 64, n_threads=8))
 
 
 def test_pareto_without_requirements(ctx, ps):
@@ -382,3 +386,33 @@ def test_topk_with_a_host_budget_on_a_power_of_two_space(ctx, ps, host_cap):
         caps = [80 * synth.GB]
         assert_same_sweep(gs.sweep(filt, caps, ps.REDUCE_TOPK, 64),
                           os_.sweep(filt, caps, O.KIND_TOPK, 64, n_threads=8))
+
+
+def long_frontier_space():
+    """One model, 64 neighbouring device counts, no model axes: every device count
+    contributes two entries to the frontier and the single-device point one more --
+    129 entries, one more than the sweep's fast lists hold."""
+    models = synth.zoo(1, 5, max_layers=160, max_hidden_mult=256)
+    models["w_param"], models["w_grad"], models["w_opt"] = 2, 1, 2
+    return synth._space(models, list(range(100, 164)), t_enum_max=1, k_enum_max=1, n_act=1, n_tpa=1,
+                        mode_mask=0b1111)
+
+
+def test_pareto_frontier_longer_than_the_fast_lists(ctx, ps):
+    """A frontier beyond 128 entries takes the slow exact path and is still the oracle's."""
+    space = long_frontier_space()
+    gs, os_ = both(ctx, space)
+    filt = dict(require_flags=O.F_GI | O.F_SC, host_cap=0)
+    caps = [1 << 62, 30 * synth.GB]
+    want = os_.sweep(filt, caps, O.KIND_PARETO, 192, n_threads=8)
+    assert want[1][0, 0] > 128
+    assert_same_sweep(gs.sweep(filt, caps, ps.REDUCE_PARETO, 192), want)
+    assert gs.last_sweep_status == ps.OK
+    # rows shorter than the frontier: its head, the true count, and the notice
+    assert_same_sweep(gs.sweep(filt, caps, ps.REDUCE_PARETO, 16), os_.sweep(filt, caps, O.KIND_PARETO, 16, n_threads=8))
+    assert gs.last_sweep_status == ps.E_TRUNCATED
+    # the same model among ordinary ones: only it takes the slow path
+    mixed = dict(space)
+    mixed["models"] = np.concatenate([synth.zoo(2, 6), space["models"], synth.zoo(2, 7)])
+    gs, os_ = both(ctx, mixed)
+    assert_same_sweep(gs.sweep(filt, caps, ps.REDUCE_PARETO, 192), os_.sweep(filt, caps, O.KIND_PARETO, 192, n_threads=8))
