@@ -327,6 +327,59 @@ int ps_eval_compact_noalloc(ps_ctx* ctx, const ps_space* space, uint64_t first, 
                             const ps_filter* filter, ps_out_soa out, uint64_t* d_idx_out,
                             uint64_t* d_n_out);
 
+/* ------------------------------------------------------------------ verification protocol */
+/* The paper's verification protocol (Section 7.1: gradient-integrity check,
+ * state-consistency check, trajectory check) as a batched brute-force run.
+ * Every case trains a tiny layered network -- `units` layers of `h` parameters,
+ * layer l maps a to tanh(theta_l * a) elementwise, loss 0.5 |out - y|^2 -- with
+ * Adam in fp64 on D logical devices that hold Theta, Omega (master copy, first
+ * and second moment), G and A exactly as the placement code says (Definition 1:
+ * full copies, element shards with eq. (2)'s boundaries, nothing, or shards in a
+ * host arena), moving data through explicit rings that count the bytes each
+ * device sends (Section 2.3), and beside it the single-device run on the global
+ * batch (Definition 4).  What a placement leaves unavailable when it is needed
+ * reads as zeros.  A result says whether the reassembled Theta and Omega of
+ * every step equal the single-device state (Theorem 5: exactly the placements
+ * with gradient integrity and state consistency), and gives the last step's
+ * per-device bytes held (persistent high-water mark plus unit buffers, largest
+ * device), bytes sent (each collective charged to its busiest device) and bytes
+ * over the host link.  The kernel evaluates none of Theorems 1-4: it executes
+ * the mechanism, so its figures check the rules (ps_eval_batch,
+ * ps_check_composition) from outside.
+ *
+ * d_cases, d_data, d_out, d_theta_out are device pointers (8-byte aligned);
+ * d_theta_out (may be null) receives units * h doubles per case: the parameters
+ * the job holds after the last step.  A case's data sits at d_data +
+ * data_offset: theta0[units*h], then the inputs x[accum][D][b][h], then the
+ * targets y[accum][D][b][h].  A case with D outside 1..4, a code above 624 or
+ * data outside [0, data_len) gets a zero result and makes ps_status return
+ * PS_E_DEVICE; nothing is read or written out of bounds.  The call may grow the
+ * context's scratch (a workspace per case).  Ranges of the shape: see its
+ * comments; outside them PS_E_RANGE. */
+typedef struct {
+  uint32_t units, h, b;          /* layers 1..8, parameters per layer 1..32, samples per device and micro-batch 1..4 */
+  uint32_t accum, steps;         /* micro-batches per step 1..4, optimizer steps 1..16                              */
+  uint32_t gather_buffers;       /* unit buffers of a gathered state: 1, or 2 (Theorem 1's proof, case S*)           */
+  uint32_t w_theta, w_omega, w_grad; /* bytes per element, 1..16; w_omega a multiple of 3 (three rows)               */
+  uint32_t pad;
+  double lr, beta1, beta2, eps;  /* Adam                                                                             */
+  double rtol, atol;             /* equal means |got - want| <= atol + rtol * |want|                                 */
+} ps_verify_shape;
+typedef struct {
+  uint32_t code;                 /* data-axis placement code, 0..624                                                 */
+  uint32_t D;                    /* logical devices, 1..4                                                            */
+  uint64_t data_offset;          /* in doubles                                                                       */
+} ps_verify_case;                /* 16 bytes */
+typedef struct {
+  uint64_t mem, comm, host;      /* bytes, last step                                                                 */
+  uint32_t match;                /* 1: every step's state equals the single-device run                               */
+  uint32_t pad;
+  double max_rel_err;            /* largest relative deviation beyond atol that was seen                             */
+} ps_verify_result;              /* 40 bytes */
+int ps_verify_batch(ps_ctx* ctx, const ps_verify_shape* shape /* host */, const ps_verify_case* d_cases,
+                    uint64_t n, const double* d_data, uint64_t data_len, ps_verify_result* d_out,
+                    double* d_theta_out);
+
 /* ------------------------------------------------------------------ measurement */
 /* Integer-pipe microbenchmark: `blocks` x 256 threads each run `iters` rounds
  * of 8 independent 32-bit add/logic chains of 16 operations.  Returns through

@@ -454,6 +454,32 @@ class Placed:
         return thetas, omegas
 
 
+def simulate_problem(units, h, b, D, code, theta0, xs, ys, steps=3, gather_buffers=1):
+    """As simulate(), on a given problem (theta0[P]; xs[j][i], ys[j][i] = micro-batch j of
+    device i); also returns the parameters the job holds after the last step (first
+    holder's view, None if they are held nowhere)."""
+    ref = run_single(units, h, xs, ys, theta0, steps)
+    job = Placed(units, h, b, D, code, theta0, gather_buffers)
+    match = True
+    books = None
+    thetas = []
+    for t in range(1, steps + 1):
+        books = Books(D)
+        job.step(t, xs, ys, books)
+        thetas, omegas = job.reassemble()
+        rt, ro = ref[t - 1]
+        if not thetas or not omegas:
+            match = False
+        for th in thetas:
+            if not np.allclose(th, rt, rtol=1e-12, atol=1e-14):
+                match = False
+        for om in omegas:
+            if not np.allclose(om, ro, rtol=1e-12, atol=1e-14):
+                match = False
+    return dict(match=match, mem=books.memory(), comm=books.comm(), host=books.host_bytes(),
+                theta=thetas[0] if thetas else None, ref_theta=ref[-1][0])
+
+
 def simulate(units, h, b, D, code, steps=3, seed=0, accum=1, gather_buffers=1):
     """Run `steps` steps of `accum` micro-batches each; returns dict(match, mem,
     comm, host) where match says whether every step's reassembled Theta and Omega

@@ -529,6 +529,33 @@ int ps_select(ps_ctx* ctx, const ps_select_query* d_queries, uint64_t n, uint32_
   return PS_OK;
 }
 
+// ------------------------------------------------------------------ verification protocol
+int ps_verify_batch(ps_ctx* ctx, const ps_verify_shape* shape, const ps_verify_case* d_cases, uint64_t n,
+                    const double* d_data, uint64_t data_len, ps_verify_result* d_out, double* d_theta_out) {
+  if (!ctx || !shape || (n && (!d_cases || !d_data || !d_out))) return PS_E_NULLPTR;
+  if (!aligned(d_cases, 8) || !aligned(d_data, 8) || !aligned(d_out, 8) || !aligned(d_theta_out, 8)) return PS_E_ALIGN;
+  const ps_verify_shape& s = *shape;
+  if (s.units < 1 || s.units > 8 || s.h < 1 || s.h > 32 || s.b < 1 || s.b > 4 || s.accum < 1 || s.accum > 4 ||
+      s.steps < 1 || s.steps > 16 || s.gather_buffers < 1 || s.gather_buffers > 2)
+    return PS_E_RANGE;
+  if (s.w_theta < 1 || s.w_theta > 16 || s.w_grad < 1 || s.w_grad > 16 || s.w_omega < 3 || s.w_omega > 48 ||
+      s.w_omega % 3 != 0)
+    return PS_E_RANGE;
+  if (!(s.lr > 0) || !(s.beta1 >= 0 && s.beta1 < 1) || !(s.beta2 >= 0 && s.beta2 < 1) || !(s.eps > 0) ||
+      !(s.rtol >= 0) || !(s.atol >= 0) || n > ((u64)1 << 32))
+    return PS_E_RANGE;
+  int rc = pending_device_error(ctx);
+  if (rc != PS_OK) return rc;
+  if (n == 0) return PS_OK;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return PS_E_CUDA;
+  rc = ensure_scratch(ctx, sizeof(double) * verify_workspace_doubles(s) * (size_t)n);
+  if (rc != PS_OK) return rc;
+  CUDA_OK(launch_verify(s, d_cases, n, d_data, data_len, static_cast<double*>(ctx->scratch), d_theta_out, d_out,
+                        ctx->d_status, ctx->stream));
+  return enqueue_status_copy(ctx);
+}
+
 // ------------------------------------------------------------------ measurement
 int ps_int_peak(ps_ctx* ctx, uint32_t blocks, uint32_t iters, uint32_t* d_sink, uint64_t* thread_ops) {
   if (!ctx || !d_sink || !thread_ops) return PS_E_NULLPTR;

@@ -300,5 +300,6 @@ __device__ __forceinline__ LocalPoint decode_local(const SpaceDev& sp, u32 lidx)
 enum : u32 {
   ST_BAD_SHAPE = 1u << 0,      // a model shape outside the supported ranges
   ST_SELF_CHECK = 1u << 2,     // an emitted entry did not re-evaluate to itself
-  ST_TRUNCATED = 1u << 3       // a frontier was longer than the caller's max_entries (a notice, not a fault)
+  ST_TRUNCATED = 1u << 3,      // a frontier was longer than the caller's max_entries (a notice, not a fault)
+  ST_BAD_CASE = 1u << 4        // a verifier case outside the supported ranges or the given data
 };

@@ -137,3 +137,9 @@ cudaError_t launch_check_point(const ModelRec* d_rec, Fact f, u32 v, u32 tau, u3
 cudaError_t launch_select(const ps_select_query* d_q, u64 n, u32 head_num, u32 head_den, u32 layer_num,
                           u32 layer_den, u32 tp_degree, ps_select_result* d_out, cudaStream_t stream);
 cudaError_t launch_int_peak(u32 blocks, u32 iters, u32* d_sink, cudaStream_t stream);
+
+// ---- brute-force verifier
+size_t verify_workspace_doubles(const ps_verify_shape& s);     // per case
+cudaError_t launch_verify(const ps_verify_shape& s, const ps_verify_case* d_cases, u64 n, const double* d_data,
+                          u64 data_len, double* d_ws, double* d_theta_out, ps_verify_result* d_out, u32* status,
+                          cudaStream_t stream);

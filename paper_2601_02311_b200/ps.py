@@ -46,7 +46,8 @@ ENTRY_DTYPE = np.dtype([("mem", "<u8"), ("comm", "<u8"), ("host", "<u8"), ("idx"
 EXPORTS = ("ps_create", "ps_destroy", "ps_status", "ps_strerror", "ps_space_create",
            "ps_space_destroy", "ps_space_set_models", "ps_space_rederive", "ps_space_size",
            "ps_space_points_per_model", "ps_space_decode", "ps_eval_batch", "ps_sweep_pareto",
-           "ps_check_composition", "ps_int_peak", "ps_eval_compact_noalloc", "ps_select")
+           "ps_check_composition", "ps_int_peak", "ps_eval_compact_noalloc", "ps_select",
+           "ps_verify_batch")
 
 
 class _SpaceDesc(C.Structure):
@@ -67,6 +68,19 @@ class _Filter(C.Structure):
 class _OutSoa(C.Structure):
     _fields_ = [("mem", C.c_void_p), ("comm_paper", C.c_void_p), ("comm_ext", C.c_void_p),
                 ("host", C.c_void_p), ("flags", C.c_void_p)]
+
+
+class _VerifyShape(C.Structure):
+    _fields_ = [("units", C.c_uint32), ("h", C.c_uint32), ("b", C.c_uint32), ("accum", C.c_uint32),
+                ("steps", C.c_uint32), ("gather_buffers", C.c_uint32), ("w_theta", C.c_uint32),
+                ("w_omega", C.c_uint32), ("w_grad", C.c_uint32), ("pad", C.c_uint32),
+                ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
+                ("rtol", C.c_double), ("atol", C.c_double)]
+
+
+VERIFY_CASE_DTYPE = np.dtype([("code", "<u4"), ("D", "<u4"), ("data_offset", "<u8")])
+VERIFY_RESULT_DTYPE = np.dtype([("mem", "<u8"), ("comm", "<u8"), ("host", "<u8"), ("match", "<u4"),
+                                ("pad", "<u4"), ("max_rel_err", "<f8")])
 
 
 class _Point(C.Structure):
@@ -102,6 +116,8 @@ _lib.ps_check_composition.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_ui
                                       C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p]
 _lib.ps_select.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32,
                            C.c_uint32, C.c_uint32, C.c_void_p]
+_lib.ps_verify_batch.argtypes = [C.c_void_p, C.POINTER(_VerifyShape), C.c_void_p, C.c_uint64, C.c_void_p,
+                                 C.c_uint64, C.c_void_p, C.c_void_p]
 _lib.ps_int_peak.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_void_p,
                              C.POINTER(C.c_uint64)]
 
@@ -194,6 +210,32 @@ class Context:
         self.select_into(d_q, len(q), d_o, headroom, layer, tp_degree)
         self.check_status()
         return d_o.cpu().numpy()[:len(q) * 32].view(SELECT_RESULT_DTYPE)
+
+    def verify_batch(self, shape: dict, cases: np.ndarray, data: np.ndarray, want_theta: bool = False):
+        """ps_verify_batch: `cases` a VERIFY_CASE_DTYPE array, `data` a float64 array holding every
+        case's problem; returns VERIFY_RESULT_DTYPE records (and the final parameters)."""
+        sh = _VerifyShape(shape["units"], shape["h"], shape["b"], shape.get("accum", 1), shape.get("steps", 3),
+                          shape.get("gather_buffers", 1), shape.get("w_theta", 2), shape.get("w_omega", 12),
+                          shape.get("w_grad", 2), 0, shape.get("lr", 0.05), shape.get("beta1", 0.9),
+                          shape.get("beta2", 0.999), shape.get("eps", 1e-8), shape.get("rtol", 1e-12),
+                          shape.get("atol", 1e-14))
+        cases = np.ascontiguousarray(cases)
+        assert cases.dtype.itemsize == 16
+        data = np.ascontiguousarray(data, dtype=np.float64)
+        n = len(cases)
+        dev = self.torch_device
+        d_cases = torch.from_numpy(cases.view(np.uint8).reshape(-1).copy()).to(dev)
+        d_data = torch.from_numpy(data).to(dev)
+        d_out = torch.zeros(max(n, 1) * 40, dtype=torch.uint8, device=dev)
+        P = shape["units"] * shape["h"]
+        d_theta = torch.zeros(max(n, 1) * P, dtype=torch.float64, device=dev) if want_theta else None
+        _check(_lib.ps_verify_batch(self._h, C.byref(sh), _dptr(d_cases), n, _dptr(d_data), len(data),
+                                    _dptr(d_out), _dptr(d_theta)), "ps_verify_batch")
+        self.check_status()
+        res = d_out.cpu().numpy()[:n * 40].view(VERIFY_RESULT_DTYPE)
+        if want_theta:
+            return res, d_theta.cpu().numpy().reshape(-1, P)[:n]
+        return res
 
     def int_peak(self, blocks: int, iters: int, sink: torch.Tensor) -> int:
         ops = C.c_uint64()
