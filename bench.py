@@ -44,23 +44,19 @@ GB = synth.GB
 VALID = 1 | 2 | 4
 METRIC = "placement evaluations/sec (bit-exact vs oracle)"
 UNIT = "evals/s"
-# Integer work per point of the top-k sweep: the thread-instructions the kernel
-# executes per point (ncu, smsp__inst_executed x 32 / points, profiles/).  The
-# method's own need cannot be larger than what a correct kernel executes, so this
-# is the work figure used for the roofline: achieved = this x points/s, against
-# the integer issue rate measured by k_int_peak in the same run -- i.e. how busy
-# the integer-capable issue slots are.  A lower figure at the same fraction is
-# the real win (it was 86 in the first correct kernel and 11.3 before the kernels
-# were compiled for the cases the space and the filter allow).
-EXEC_OPS_PER_POINT_SWEEP = 7.90
-EXEC_OPS_PER_POINT_PARETO = 10.45     # the same figure for the Pareto sweep
 BYTES_PER_POINT_MATERIALISE = 36
-# DRAM traffic of one launch from the ncu captures summarised under profiles/
-# (k_sweep<top-k> on the full stress configuration; k_eval<materialise> per point
-# of a 2^25-point window, where traffic grows in proportion to the points)
-NCU_SWEEP_DRAM_BYTES = 5_968_128
-NCU_PARETO_DRAM_BYTES = 2_008_320
-NCU_MATERIALISE_DRAM_BYTES_PER_POINT = 1_372_498_464 / (1 << 25)
+
+
+def ncu_counters():
+    """Figures only a profiler can give (executed instructions per point, pipe
+    utilisation, DRAM traffic), from the tracked summary of the last capture.
+    They describe the kernels of the commit named there, on the stress
+    configuration; the bench prints that commit and uses them on that workload
+    only."""
+    try:
+        return json.load(open(os.path.join(ROOT, "profiles", "ncu_counters.json")))
+    except Exception:
+        return None
 
 
 def parse_args():
@@ -179,18 +175,26 @@ def oracle_step(osp, first, count, model_count, threads):
     return model_count * ppm * (len(TOPK_CAPS) + len(PARETO_CAPS)) + 2 * count
 
 
-def cpu_baseline(space, threads=None):
-    """The oracle as it stands, timed on a bounded sample of the workload."""
+def cpu_baseline(space, gpu_topk=None, threads=None):
+    """The oracle as it stands, timed on a bounded sample of the workload.  Its
+    result is not thrown away: the top-k tables of every model it sweeps are
+    compared with the GPU's (`gpu_topk` = (entries, counts)); returns the
+    baseline record and the number of models compared (None on a mismatch)."""
     from oracle import oracle as O
     threads = threads or O.hardware_threads()
     osp = O.Space(space)
     n_models = min(len(space["models"]), 96 * threads)      # about 15 s of CPU work
     t0 = time.perf_counter()
-    osp.sweep(TOPK_FILTER, TOPK_CAPS, O.KIND_TOPK, TOPK_K, model_count=n_models, n_threads=threads)
+    o_e, o_c = osp.sweep(TOPK_FILTER, TOPK_CAPS, O.KIND_TOPK, TOPK_K, model_count=n_models, n_threads=threads)
     dt = time.perf_counter() - t0
     evals = n_models * osp.points_per_model
+    compared = 0
+    if gpu_topk is not None:
+        g_e, g_c = gpu_topk
+        same = g_e[:n_models].tobytes() == o_e[:n_models].tobytes() and np.array_equal(g_c[:n_models], o_c[:n_models])
+        compared = n_models if same else None
     return {"value": evals / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
-            "sample": f"top-k sweep of the first {n_models} models ({evals} points) in {dt:.2f} s"}
+            "sample": f"top-k sweep of the first {n_models} models ({evals} points) in {dt:.2f} s"}, compared
 
 
 def run_reference(args):
@@ -304,7 +308,8 @@ def run_ours(args):
         if err:
             print(json.dumps({"metric": METRIC, "value": None, "unit": UNIT, "error": "parity: " + err}))
             sys.exit(1)
-        parity = "bit-exact on sampled models and windows"
+        parity = ("bit-exact: top-k and Pareto tables of 3 sampled models, a 2^18-point window materialised "
+                  "and compacted")
 
     # device buffers (caller-owned outputs)
     topk_out, topk_cnt = gs.alloc_sweep(len(TOPK_CAPS), TOPK_K)
@@ -449,6 +454,24 @@ def run_ours(args):
     torch.cuda.synchronize()
     select_ms = s0.elapsed_time(s1) / 10
 
+    # ---- compaction with every point surviving (the output-bound case), beside the step
+    dense_filter = dict(require_flags=0)                                    # no capacity, no flags: all survive
+    for _ in range(3):
+        gs.eval_batch_into(first, count, cmp_out, dense_filter, cmp_idx, cmp_n)
+    torch.cuda.synchronize()
+    dense_ms = []
+    for _ in range(10):
+        flush.fill_(1)
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record(stream)
+        gs.eval_batch_into(first, count, cmp_out, dense_filter, cmp_idx, cmp_n)
+        d1.record(stream)
+        torch.cuda.synchronize()
+        dense_ms.append(d0.elapsed_time(d1))
+    dense_ms = float(np.mean(dense_ms))
+    dense_survivors = int(cmp_n.item())
+    ctx.check_status()
+
     # ---- aggregate over ranks: max time, summed points
     value, e2e_value, total_ms_max, e2e_ms_max = aggregate_over_ranks(
         dist, dev, total_ms, e2e_s * 1e3, world, points_per_step, args.steps, e2e_steps)
@@ -461,8 +484,31 @@ def run_ours(args):
             pass
         hbm_peak = peaks.get("hbm_gbs", 6650.0)
         hbm_src = "measured" if "hbm_gbs" in peaks else "fallback"
-        sweep_ms = phase_ms["topk"]
-        alu_achieved = EXEC_OPS_PER_POINT_SWEEP * size / (sweep_ms * 1e-3) / 1e12
+        ncu = ncu_counters()
+        on_captured_workload = args.workload == "C4" and args.models is None and ncu is not None
+        ncu_commit = ncu["captured_at_commit"] if ncu else None
+
+        def alu_roofline(kernel_key, label, ms):
+            """The sweep against the integer issue rate measured in this run.  `frac` is the
+            issue-slot fraction: executed thread-instructions of all kinds per point (ncu) x
+            points/s over the add/xor issue peak.  `alu_pipe_frac` is ncu's ALU-pipe
+            utilisation (integer and logic instructions only) -- the figure to hold against
+            an integer-ALU target.  Both come from the capture named in `counters_commit`
+            and are given on the workload of that capture only."""
+            k = ncu["kernels"][kernel_key] if on_captured_workload else None
+            ops = k["thread_instr_per_point"] if k else None
+            achieved = ops * size / (ms * 1e-3) / 1e12 if k else None
+            return {"bound": "alu", "kernel": label, "achieved": achieved, "peak": int_peak / 1e12,
+                    "unit": "T thread-instructions/s", "frac": achieved / (int_peak / 1e12) if k else None,
+                    "frac_is": "issue-slot fraction (all executed instructions)",
+                    "alu_pipe_frac": k["alu_pipe_active"] if k else None,
+                    "alu_pipe_frac_is": "ncu ALU-pipe utilisation of the captured launch",
+                    "issue_active_ncu": k["issue_active"] if k else None,
+                    "traffic": k["dram_bytes_per_launch"] if k else None,
+                    "ops_per_point": ops, "counters_commit": ncu_commit if k else None,
+                    "evals_per_s": size / (ms * 1e-3),
+                    "peak_source": "k_int_peak (add+xor chains on both integer pipes) measured in this run"}
+
         mat_gbs = BYTES_PER_POINT_MATERIALISE * count / (phase_ms["materialise"] * 1e-3) / 1e9
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -486,32 +532,38 @@ def run_ours(args):
             "e2e": {"value": e2e_value, "unit": UNIT,
                     "h2d_bytes_per_step": int(models_pinned.numel()), "d2h_bytes_per_step": int(d2h)},
             "gpu_launches": launches_per_step * args.steps,
-            "roofline": {"bound": "alu", "kernel": "k_sweep<top-k> (+ merge)",
-                         "achieved": alu_achieved, "peak": int_peak / 1e12, "unit": "T thread-instructions/s",
-                         "frac": alu_achieved / (int_peak / 1e12),
-                         "traffic": NCU_SWEEP_DRAM_BYTES if args.workload == "C4" and args.models is None else None,
-                         "ops_per_point": EXEC_OPS_PER_POINT_SWEEP,
-                         "ops_per_point_source": "executed thread-instructions per point of this kernel "
-                                                 "(ncu capture on the stress configuration, profiles/)",
-                         "alu_pipe_active_ncu": 0.490, "issue_active_ncu": 0.752,
-                         "peak_source": "k_int_peak (add+xor chains on both integer pipes) measured in this run"},
-            "roofline_pareto": {"bound": "alu", "kernel": "k_sweep<Pareto> (+ merge)",
-                                "achieved": EXEC_OPS_PER_POINT_PARETO * size / (phase_ms["pareto"] * 1e-3) / 1e12,
-                                "peak": int_peak / 1e12, "unit": "T thread-instructions/s",
-                                "frac": EXEC_OPS_PER_POINT_PARETO * size / (phase_ms["pareto"] * 1e-3) / int_peak,
-                                "traffic": NCU_PARETO_DRAM_BYTES if args.workload == "C4" and args.models is None else None,
-                                "ops_per_point": EXEC_OPS_PER_POINT_PARETO,
-                                "alu_pipe_active_ncu": 0.509, "issue_active_ncu": 0.714},
+            # the dominant kernel of a step is the Pareto sweep (its share is in phases_ms)
+            "roofline": alu_roofline("k_sweep_pareto", "k_sweep<Pareto> (+ merge)", phase_ms["pareto"]),
+            "roofline_topk": alu_roofline("k_sweep_topk", "k_sweep<top-k> (+ merge)", phase_ms["topk"]),
             "roofline_hbm": {"bound": "hbm", "kernel": "k_eval<materialise>", "achieved": mat_gbs,
                              "peak": hbm_peak, "unit": "GB/s", "frac": mat_gbs / hbm_peak,
-                             "traffic": int(NCU_MATERIALISE_DRAM_BYTES_PER_POINT * count),
+                             "traffic": (int(ncu["kernels"]["k_eval_materialise"]["dram_bytes_per_point"] * count)
+                                         if on_captured_workload else None),
+                             "counters_commit": ncu_commit if on_captured_workload else None,
                              "peak_source": hbm_src + " (of measured)" if hbm_src == "measured" else hbm_src + " (of fallback)"},
         }
+        dense_gbs = (BYTES_PER_POINT_MATERIALISE + 8) * dense_survivors / (dense_ms * 1e-3) / 1e9
+        line["roofline_compact_dense"] = {
+            "bound": "hbm", "kernel": "k_compact_count + k_tile_scan + k_eval<write>, every point survives",
+            "achieved": dense_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": dense_gbs / hbm_peak,
+            "ms": dense_ms, "survivors": dense_survivors, "bytes_per_survivor": BYTES_PER_POINT_MATERIALISE + 8,
+            "traffic": None}
         line["select"] = {"queries": n_sel, "ms": select_ms, "queries_per_s": n_sel / (select_ms * 1e-3),
                           "GB/s": 64 * n_sel / (select_ms * 1e-3) / 1e9,
                           "frac_of_hbm_peak": 64 * n_sel / (select_ms * 1e-3) / 1e9 / hbm_peak}
         if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = cpu_baseline(space)
+            gpu_topk = None
+            if not args.no_parity:
+                e = topk_out.cpu().numpy().view(ps.ENTRY_DTYPE).reshape(nm, len(TOPK_CAPS), TOPK_K)
+                c = topk_cnt.cpu().numpy().view(np.uint32).reshape(nm, len(TOPK_CAPS))
+                gpu_topk = (e, c)
+            line["cpu_baseline"], compared = cpu_baseline(space, gpu_topk)
+            if compared is None:
+                print(json.dumps({"metric": METRIC, "value": None, "unit": UNIT,
+                                  "error": "parity: top-k tables differ from the CPU-baseline sweep"}))
+                sys.exit(1)
+            if compared:
+                line["config"]["parity"] += f"; top-k tables of {compared} of {nm} models (the CPU-baseline sweep)"
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()

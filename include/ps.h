@@ -295,6 +295,44 @@ int ps_select(ps_ctx* ctx, const ps_select_query* d_queries, uint64_t n, uint32_
               uint32_t headroom_den, uint32_t layer_num, uint32_t layer_den, uint32_t tp_degree,
               ps_select_result* d_out);
 
+/* Algorithm 1 beside the exhaustive answer.  For every model of a space, run
+ * Algorithm 1 with the model's own parameter count, layer size and byte widths,
+ * the device count n_values[n_index] and M_d = device_bytes, take its choice as
+ * a point of the space (tensor degree T of branch 2 or 1, no pipeline axis,
+ * D = N / T, the space's first activation and tensor-axis variants, data-axis
+ * code 0 or 32), evaluate that point as the space does (Theorems 1-4, with
+ * activations and the traffic Theorem 2 does not price, per filter->comm_kind),
+ * and hold it against the model's Pareto frontier under the same capacity, as
+ * ps_sweep_pareto wrote it (d_frontier[n_models][n_caps][max_entries],
+ * d_counts[n_models][n_caps]; the capacity at cap_index must be device_bytes and
+ * the filter the sweep's).  Sweep a space whose only device count is that N to
+ * compare like with like.  status bits:
+ *   PS_SEL_IN_SPACE     the choice is a point of the space (alg_idx is its index)
+ *   PS_SEL_SURVIVOR     it fits device_bytes, the host budget and the required flags
+ *   PS_SEL_ON_FRONTIER  the frontier has an entry with its (mem, comm)
+ *   PS_SEL_DOMINATED    some entry is no worse in both and better in one
+ *   PS_SEL_FRONTIER_EMPTY / PS_SEL_FRONTIER_TRUNCATED (count > max_entries: only
+ *                       the written head was looked at)
+ * best_* is the frontier's last written entry: the least communication that fits.
+ * All pointers but filter are device pointers; d_out has n_models records. */
+enum {
+  PS_SEL_IN_SPACE = 1u << 0, PS_SEL_SURVIVOR = 1u << 1, PS_SEL_ON_FRONTIER = 1u << 2,
+  PS_SEL_DOMINATED = 1u << 3, PS_SEL_FRONTIER_EMPTY = 1u << 4, PS_SEL_FRONTIER_TRUNCATED = 1u << 5
+};
+typedef struct {
+  uint64_t alg_mem, alg_comm, alg_idx;     /* Algorithm 1's choice as the space evaluates it   */
+  uint64_t best_mem, best_comm, best_idx;  /* the frontier's least-communication entry          */
+  uint32_t branch, T, code_dp;             /* as in ps_select_result                            */
+  uint32_t alg_flags;                      /* PS_F_* of the choice (PS_F_FEASIBLE vs device_bytes) */
+  uint32_t status, pad;
+} ps_select_compare_result;                /* 72 bytes */
+int ps_select_compare(ps_ctx* ctx, const ps_space* space, uint32_t n_index, uint64_t device_bytes,
+                      uint32_t fast_interconnect, uint32_t headroom_num, uint32_t headroom_den,
+                      uint32_t layer_num, uint32_t layer_den, uint32_t tp_degree,
+                      const ps_filter* filter /* host */, const ps_front_entry* d_frontier,
+                      const uint32_t* d_counts, uint32_t n_caps, uint32_t cap_index,
+                      uint32_t max_entries, ps_select_compare_result* d_out);
+
 /* The filter-and-compact form of ps_eval_batch for callers that cannot
  * allocate device memory.  (The paper has no counterpart: this is a property of
  * the library, not of the method.)
@@ -305,10 +343,11 @@ int ps_select(ps_ctx* ctx, const ps_select_query* d_queries, uint64_t n, uint32_
  * can fail or fragment that pool; and a loop that cannot afford the implicit
  * device-wide synchronisation of cudaFree/cudaMalloc.  ps_eval_batch may do
  * both when its scratch has to grow.  This function never calls cudaMalloc,
- * cudaFree or any allocating routine: its two scratch tables (a survivor count
- * per group of |mode_mask|^4 consecutive points, and a prefix sum per run of up
- * to 32 groups) sit in a fixed 1.5 MiB array inside the library image, which
- * every GPU that loads the library holds until the process ends.
+ * cudaFree or any allocating routine: its scratch tables (a survivor count per
+ * group of |mode_mask|^4 consecutive points, the list of groups that have
+ * survivors, and a prefix sum per run of up to 32 groups) sit in a fixed 2 MiB
+ * array inside the library image, which every GPU that loads the library holds
+ * until the process ends.
  *
  * Arguments, outputs, order of the survivors and error behaviour are those of
  * ps_eval_batch with a non-null filter (which is required here).  Limits and

@@ -152,6 +152,24 @@ class Space:
         return entries, counts
 
 
+def select_compare(space: "Space", n_index: int, device_bytes: int, filt: dict, entries: np.ndarray,
+                   counts: np.ndarray, cap_index: int, fast: int = 1, headroom=(7, 10), layer=(3, 10),
+                   tp_degree: int = 8) -> np.ndarray:
+    """Algorithm 1's choice for every model, as a point of the space, against the frontier
+    (entries[n_models, n_caps, max_entries], counts[n_models, n_caps]).  Returns (n_models, 12)
+    uint64: alg mem, comm, idx; best mem, comm, idx; branch, T, code, flags, status, 0."""
+    entries = np.ascontiguousarray(entries)
+    counts = np.ascontiguousarray(counts, dtype=np.uint32)
+    nm, n_caps, max_entries = entries.shape
+    out = np.zeros((nm, 12), dtype=np.uint64)
+    f = _mk_filter(filt)
+    lib().orc_select_compare(C.byref(space.desc), C.c_uint32(n_index), C.c_uint64(device_bytes), C.c_uint32(fast),
+                             headroom[0], headroom[1], layer[0], layer[1], tp_degree, C.byref(f), _ptr(entries),
+                             _ptr(counts), C.c_uint32(n_caps), C.c_uint32(cap_index), C.c_uint32(max_entries),
+                             _ptr(out))
+    return out
+
+
 def _mk_filter(filt: dict) -> _Filter:
     return _Filter(filt.get("host_cap", NO_LIMIT), filt.get("require_flags", 0),
                    filt.get("comm_kind", COMM_PAPER_PLUS_EXT), filt.get("cap_bytes", NO_LIMIT))

@@ -570,6 +570,78 @@ void orc_select(const u64* query, u64 n, u32 hn, u32 hd, u32 ln, u32 ld, u32 tp_
   }
 }
 
+// Algorithm 1 beside the frontier: for every model, Algorithm 1's choice at device
+// count n_values[n_index] and M_d = device_bytes, taken as a point of the space
+// (K = 1, first variants), evaluated like any other point, and held against the
+// model's frontier under that capacity (frontier[n_models][n_caps][max_entries],
+// counts[n_models][n_caps]).  out: 12 u64 per model -- alg mem, comm, idx; best
+// mem, comm, idx (the frontier's last written entry); branch, T, code, point
+// flags, status (1 in space, 2 survivor, 4 on frontier, 8 dominated, 16 frontier
+// empty, 32 frontier truncated), 0.
+void orc_select_compare(const ODesc* d, u32 n_index, u64 Md, u32 fast, u32 hn, u32 hd, u32 ln, u32 ld,
+                        u32 tp_degree, const OFilter* f, const OEntry* frontier, const u32* counts,
+                        u32 n_caps, u32 cap_index, u32 max_entries, u64* out) {
+  Space sp(d);
+  const u64 N = d->n_values[n_index];
+  for (u32 model = 0; model < d->n_models; ++model) {
+    ORecord rec = derive_record(d->models[model]);
+    u64 query[8] = {rec.P, rec.unit, Md, N, rec.w_theta, rec.w_grad, rec.w_omega, fast ? 1ull : 0ull};
+    u64 pick[6];
+    orc_select(query, 1, hn, hd, ln, ld, tp_degree, pick);
+    const u32 branch = (u32)pick[2], T = (u32)pick[3], code = (u32)pick[4];
+    // is the choice a point of the space?  Walk the space's own order to find it.
+    bool in_space = false;
+    u64 idx = 0;
+    {
+      u64 at = (u64)model * sp.pts_per_model;
+      const u64 per_fact = (u64)d->n_act_variants * d->n_tpa_variants * sp.n_codes;
+      for (u32 i = 0; i < d->n_n && !in_space; ++i) {
+        for (size_t k = 0; k < sp.facts[i].size() && !in_space; ++k) {
+          const Fact& fa = sp.facts[i][k];
+          if (i == n_index && fa.T == T && fa.K == 1) {
+            // the code's modes as digits of the allowed-mode numbering
+            u64 digits = 0, weight = 1;
+            bool ok = true;
+            u32 c = code;
+            for (int st = 0; st < 4; ++st) {
+              int mode = c % 5; c /= 5;
+              int pos = -1;
+              for (size_t q = 0; q < sp.modes.size(); ++q) if (sp.modes[q] == mode) pos = (int)q;
+              if (pos < 0) ok = false;
+              digits += weight * (u64)(pos < 0 ? 0 : pos);
+              weight *= sp.modes.size();
+            }
+            if (ok) { in_space = true; idx = at + digits; }
+          }
+          at += per_fact;
+        }
+      }
+    }
+    int pi[4]; u32 c = code;
+    for (int st = 0; st < 4; ++st) { pi[st] = c % 5; c /= 5; }
+    OResult r = eval_point(rec, N, T, 1, N / T, 0, 0, pi[0], pi[1], pi[2], pi[3], d->tp_max_valid,
+                           d->tp_coll_per_layer, true, d->sstar_units, d->grad_accum_steps);
+    const u64 comm = objective_comm(r, *f);
+    u32 fl;
+    const bool survivor = passes(r, *f, Md, &fl);
+    u32 status = (in_space ? 1u : 0u) | (survivor ? 2u : 0u);
+    const u32 count = counts[(u64)model * n_caps + cap_index];
+    const OEntry* fr = frontier + ((u64)model * n_caps + cap_index) * max_entries;
+    const u32 written = std::min(count, max_entries);
+    if (count == 0) status |= 16u;
+    if (count > max_entries) status |= 32u;
+    for (u32 e = 0; e < written; ++e) {
+      if (fr[e].mem == r.mem && fr[e].comm == comm) status |= 4u;
+      else if (fr[e].mem <= r.mem && fr[e].comm <= comm) status |= 8u;
+    }
+    u64* o = out + 12 * (u64)model;
+    o[0] = r.mem; o[1] = comm; o[2] = in_space ? idx : 0;
+    o[3] = written ? fr[written - 1].mem : 0; o[4] = written ? fr[written - 1].comm : 0;
+    o[5] = written ? fr[written - 1].idx : 0;
+    o[6] = branch; o[7] = T; o[8] = code; o[9] = fl; o[10] = status; o[11] = 0;
+  }
+}
+
 u32 orc_hardware_threads() { return std::thread::hardware_concurrency(); }
 
 }  // extern "C"

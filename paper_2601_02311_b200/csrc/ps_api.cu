@@ -395,12 +395,18 @@ int ps_eval_batch(ps_ctx* ctx, const ps_space* sp, uint64_t first, uint64_t coun
     a.cap_bytes = filter->cap_bytes;
     a.host_cap = filter->host_cap;
     a.require_flags = filter->require_flags & ~(u32)PS_F_FEASIBLE;
-    const size_t off_bytes = (sizeof(u32) * n_groups + 15) & ~size_t(15);
-    rc = ensure_scratch(ctx, off_bytes + sizeof(u64) * n_groups);
+    // per group a count and a place in the list of groups with survivors, the list's length,
+    // per run of groups an offset
+    const size_t cnt_bytes = (sizeof(u32) * n_groups + 15) & ~size_t(15);
+    rc = ensure_scratch(ctx, 2 * cnt_bytes + 16 + sizeof(u64) * n_groups);
     if (rc != PS_OK) return rc;
-    a.tile_count = static_cast<u32*>(ctx->scratch);
-    a.tile_offset = reinterpret_cast<u64*>(static_cast<char*>(ctx->scratch) + off_bytes);
+    char* base = static_cast<char*>(ctx->scratch);
+    a.tile_count = reinterpret_cast<u32*>(base);
+    a.nonempty = reinterpret_cast<u32*>(base + cnt_bytes);
+    a.n_nonempty = reinterpret_cast<u32*>(base + 2 * cnt_bytes);
+    a.tile_offset = reinterpret_cast<u64*>(base + 2 * cnt_bytes + 16);
     eval_plan_runs(a);
+    CUDA_OK(cudaMemsetAsync(a.n_nonempty, 0, sizeof(u32), ctx->stream));
     CUDA_OK(launch_eval_count(sp->dev, a, ctx->stream));
     CUDA_OK(launch_tile_scan(a, ctx->stream));
     CUDA_OK(launch_eval_write(sp->dev, a, ctx->stream));
@@ -526,6 +532,31 @@ int ps_select(ps_ctx* ctx, const ps_select_query* d_queries, uint64_t n, uint32_
   if (!guard.ok) return PS_E_CUDA;
   CUDA_OK(launch_select(d_queries, n, headroom_num, headroom_den, layer_num, layer_den, tp_degree, d_out,
                         ctx->stream));
+  return PS_OK;
+}
+
+int ps_select_compare(ps_ctx* ctx, const ps_space* sp, uint32_t n_index, uint64_t device_bytes,
+                      uint32_t fast_interconnect, uint32_t headroom_num, uint32_t headroom_den,
+                      uint32_t layer_num, uint32_t layer_den, uint32_t tp_degree, const ps_filter* filter,
+                      const ps_front_entry* d_frontier, const uint32_t* d_counts, uint32_t n_caps,
+                      uint32_t cap_index, uint32_t max_entries, ps_select_compare_result* d_out) {
+  if (!ctx || !sp || !filter || !d_frontier || !d_counts || !d_out) return PS_E_NULLPTR;
+  if (sp->ctx != ctx) return PS_E_RANGE;
+  if (!aligned(d_frontier, 8) || !aligned(d_counts, 4) || !aligned(d_out, 8)) return PS_E_ALIGN;
+  if (n_index >= sp->n_values.size() || n_caps < 1 || n_caps > PS_MAX_CAPS || cap_index >= n_caps || max_entries < 1 ||
+      headroom_den < 1 || layer_den < 1 || tp_degree < 1 || headroom_num > (1u << 16) || headroom_den > (1u << 16) ||
+      layer_num > (1u << 16) || layer_den > (1u << 16) || device_bytes > ((u64)1 << 50) ||
+      filter->comm_kind > PS_COMM_PAPER_PLUS_EXT || (filter->require_flags & ~KNOWN_FLAGS))
+    return PS_E_RANGE;
+  int rc = pending_device_error(ctx);
+  if (rc != PS_OK) return rc;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return PS_E_CUDA;
+  CUDA_OK(launch_select_compare(sp->dev, sp->fact_begin[n_index], sp->fact_begin[n_index + 1], sp->n_values[n_index],
+                                device_bytes, fast_interconnect, headroom_num, headroom_den, layer_num, layer_den,
+                                tp_degree, filter->host_cap, filter->require_flags & ~(u32)PS_F_FEASIBLE,
+                                filter->comm_kind, d_frontier, d_counts, n_caps, cap_index, max_entries, d_out,
+                                ctx->stream));
   return PS_OK;
 }
 

@@ -276,6 +276,42 @@ __device__ __forceinline__ PointOut eval_point(const ModelRec& r, const Fact& f,
   return o;
 }
 
+// ---------------------------------------------------------------- filters on (Theta, Omega, G) triples
+// bits of a triple's static description
+enum : u32 {
+  T_THETA_AVAIL = 1u << 0, T_GRAD_COVER = 1u << 1, T_SC = 1u << 2, T_HOST = 1u << 3,
+  T_M_OR_O = 1u << 4, T_EXT0 = 1u << 5
+};
+
+__device__ __forceinline__ u32 triple_bits(u32 th, u32 om, u32 gr, bool d1) {
+  const bool on_shard = in_set(SET_UPDATE_ON_SHARD, om);
+  const bool omega_full = (om == PS_MODE_R) || (d1 && in_set(SET_SHARDLIKE, om));
+  const bool theta_avail = in_set(SET_THETA_ALWAYS, th) || (th == PS_MODE_S && d1) ||
+                           (th == PS_MODE_M && omega_full);
+  const bool grad_cover = d1 || on_shard || in_set(SET_GRAD_FULL, gr);
+  const u32 seen = (1u << th) | (1u << om) | (1u << gr);
+  // data-axis traffic beyond Theorem 2: none with a single replica (nothing moves)
+  const bool ext0 = d1 || !((th == PS_MODE_O) || (th == PS_MODE_R && on_shard) ||
+                            in_set((1u << PS_MODE_SG) | SET_M_OR_O, gr) || om == PS_MODE_SG);
+  return (theta_avail ? T_THETA_AVAIL : 0) | (grad_cover ? T_GRAD_COVER : 0) |
+         (om != PS_MODE_M ? T_SC : 0) | ((seen >> PS_MODE_O) & 1u ? T_HOST : 0) |
+         ((seen & SET_M_OR_O) ? T_M_OR_O : 0) | (ext0 ? T_EXT0 : 0);
+}
+
+// which activation digits give a point with every required flag, for a triple
+// with static bits `tb` (the composition bits are checked per unit)
+__device__ __forceinline__ u32 allowed_act_digits(u32 tb, u32 req, u32 all, u32 own, u32 is_o, u32 not_mo) {
+  u32 ok = all;
+  if ((req & PS_F_SC) && !(tb & T_SC)) ok = 0;
+  if ((req & PS_F_THETA_AVAIL) && !(tb & T_THETA_AVAIL)) ok = 0;
+  if ((req & PS_F_GRAD_COVER) && !(tb & T_GRAD_COVER)) ok = 0;
+  if (req & PS_F_GI) ok &= ((tb & T_THETA_AVAIL) && (tb & T_GRAD_COVER)) ? own : 0;
+  if (req & PS_F_ACT_AVAIL) ok &= own;
+  if (req & PS_F_USES_HOST) ok &= (tb & T_HOST) ? all : is_o;
+  if (req & PS_F_PAPER_PRICED) ok &= ((tb & T_EXT0) && !(tb & T_M_OR_O)) ? not_mo : 0;
+  return ok;
+}
+
 // linear index within a model -> unit, variant, digits of the data-axis code
 struct LocalPoint {
   u32 unit, v, tau, dth, dom, dgr, dac;

@@ -16,13 +16,16 @@
 // (shared -> global, asynchronous), so the warp computes the next array while
 // the previous one drains.
 //
-// Compaction is count -> scan -> write: the count pass (one warp per run of up to
-// 32 consecutive groups) stores the survivors of each group and of each run, a
-// single-block scan turns the runs' totals into offsets, the write pass skips
-// the groups without survivors, evaluates the others again and places their
-// survivors with ballot/popc prefix sums; a group's offset is its run's plus the
-// counts of the run's earlier groups.  Output order is the index order, so the
-// result is unique.
+// Compaction is count -> scan -> write.  The count pass (k_compact_count, one
+// warp per run of up to 32 consecutive groups) never forms a point's bytes or
+// flags: like the sweeps it compares a triple's own bytes with a per-(variant,
+// digit) bound and masks the result with the digits the required flags allow.
+// It stores the survivors of each group and of each run and appends the groups
+// that have survivors to a list.  A single-block scan turns the runs' totals
+// into offsets.  The write pass takes the listed groups one per warp, evaluates
+// them and places their survivors with ballot/popc prefix sums; a group's offset
+// is its run's plus the counts of the run's earlier groups.  Output order is the
+// index order, so the result is unique.
 #include "ps_device.cuh"
 #include "ps_internal.h"
 
@@ -31,11 +34,12 @@ namespace {
 // Launch shapes (blocks per SM; two are resident at a time).  Materialise is
 // fastest with about one group per warp: short-lived blocks keep the warps of an
 // SM at different stages (set-up, staging, draining stores) and the running
-// warps write neighbouring stretches of every output array.  Count is
-// arithmetic-bound and prefers long runs of groups per warp (the per-model
-// coefficients are then computed once).  Write skips the groups without
-// survivors, which come in long stretches (invalid factorisations), so it takes
-// shorter runs to stay balanced.
+// warps write neighbouring stretches of every output array.  The count pass
+// prefers long runs of groups per warp (what a model and a factorisation fix is
+// then computed once).  The write pass takes the listed groups round-robin; with
+// many short blocks the stores of neighbouring groups are in flight together
+// (every point surviving: 0.56 of the copy bandwidth with 4 blocks per SM, 0.62
+// with 32).
 #ifndef EVAL_GRID_PER_SM_MATERIALISE
 #define EVAL_GRID_PER_SM_MATERIALISE 64
 #endif
@@ -43,7 +47,7 @@ namespace {
 #define EVAL_GRID_PER_SM_COMPACT 2
 #endif
 #ifndef EVAL_GRID_PER_SM_WRITE
-#define EVAL_GRID_PER_SM_WRITE 8
+#define EVAL_GRID_PER_SM_WRITE 32
 #endif
 constexpr int THREADS = EVAL_THREADS;
 constexpr int WARPS = THREADS / 32;
@@ -78,7 +82,7 @@ __device__ __forceinline__ u32 triple_static(u32 th, u32 om, u32 gr, bool d1) {
          ((seen & SET_M_OR_O) ? X_MO3 : 0) | (ext0 ? X_EXT0 : 0);
 }
 
-enum { MODE_MATERIALISE = 0, MODE_COUNT = 1, MODE_WRITE = 2 };
+enum { MODE_MATERIALISE = 0, MODE_WRITE = 2 };
 
 // Staging for the materialise path.  A warp builds one output array of one
 // group (NC elements) in shared memory and hands it to the copy engine as a
@@ -139,21 +143,12 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
   const int lane = threadIdx.x & 31;
   const u32 warp_global = blockIdx.x * WARPS + (threadIdx.x >> 5);
   const u32 n_warps = gridDim.x * WARPS;
-  // count: one warp per run of the plan; otherwise the groups are dealt evenly
-  const u32 per_warp = MODE == MODE_COUNT ? a.run_len : (a.n_tiles + n_warps - 1) / n_warps;
-  const u32 seg_begin = (u32)min((u64)warp_global * per_warp, (u64)a.n_tiles);
-  const u32 seg_end = min(seg_begin + per_warp, a.n_tiles);
-  u64 run_total = 0;                 // count: survivors of this warp's run
-  u64 write_next = 0;                // write: where the next group's survivors go
-  if (MODE == MODE_WRITE && seg_begin < seg_end) {
-    // survivors before this warp's first group = those of the runs before its run
-    // (scanned) plus those of the run's earlier groups
-    const u32 run = seg_begin / a.run_len;
-    u64 part = 0;
-    for (u32 j = run * a.run_len + lane; j < seg_begin; j += 32) part += a.tile_count[j];
-    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-    write_next = a.tile_offset[run] + part;
-  }
+  // materialise: the window's groups are dealt evenly, a contiguous stretch per warp;
+  // write: the groups that have survivors, from the count pass's list, dealt round-robin
+  const u32 per_warp = (a.n_tiles + n_warps - 1) / n_warps;
+  const u32 it_begin = MODE == MODE_WRITE ? warp_global : (u32)min((u64)warp_global * per_warp, (u64)a.n_tiles);
+  const u32 it_end = MODE == MODE_WRITE ? *a.n_nonempty : min(it_begin + per_warp, a.n_tiles);
+  const u32 it_step = MODE == MODE_WRITE ? n_warps : 1u;
   const u32 groups_per_model = sp.n_facts * sp.nvt;
 
   // with all five modes allowed digit d is mode d, and the compiler knows every
@@ -187,13 +182,8 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
   u32 ka[R], kb[R], kc[R], kp[R], ke[R], kh[R];   // bytes (E, s, u), priced / unpriced comm (x), host (s)
   u32 st_many[R], st_one[R];                      // static description for D > 1 and D = 1
 
-  for (u32 seg = seg_begin; seg < seg_end; ++seg) {
-    // the count pass has evaluated every point of the group: nothing to place if none survived
-    u32 group_survivors = 0;
-    if (MODE == MODE_WRITE) {
-      group_survivors = a.tile_count[seg];
-      if (group_survivors == 0) continue;
-    }
+  for (u32 it = it_begin; it < it_end; it += it_step) {
+    const u32 seg = MODE == MODE_WRITE ? a.nonempty[it] : it;
     const u64 g = a.first_group + seg;
     const u32 model = (u32)(g / groups_per_model);
     const u32 gl = (u32)(g - (u64)model * groups_per_model);
@@ -272,7 +262,15 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
 
     u32 n_kept = 0;
     u64 write_base = 0;
-    if (MODE == MODE_WRITE) { write_base = write_next; write_next += group_survivors; }
+    if (MODE == MODE_WRITE) {
+      // survivors before this group = those of the runs before its run (scanned) plus
+      // those of the run's earlier groups
+      const u32 run = seg / a.run_len;
+      u64 part = 0;
+      for (u32 j = run * a.run_len + lane; j < seg; j += 32) part += a.tile_count[j];
+      for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+      write_base = a.tile_offset[run] + part;
+    }
 
     // flags of a point = what the triple fixes | what the digit fixes | what needs both:
     //   gradient integrity needs the triple's two availability bits and the digit's,
@@ -373,14 +371,172 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
         }
       }
     }
-    if (MODE == MODE_COUNT) {
-      if (lane == 0) a.tile_count[seg] = n_kept;
-      run_total += n_kept;
-    }
   }
-  if (MODE == MODE_COUNT && lane == 0 && warp_global < a.n_runs) a.tile_offset[warp_global] = run_total;
   // the staging buffers must outlive the bulk stores that read them
   if (MODE == MODE_MATERIALISE && lane == 0) bulk_wait_all();
+}
+
+// The count pass of the compaction.  One warp per run of consecutive groups.  What
+// a factorisation fixes is computed once for its (up to four) groups: the lanes'
+// triples' own bytes and host bytes, and for every (variant, digit) the bound the
+// own bytes must stay below for the point to fit the capacity (cap + 1 - activation
+// bytes) and the host budget.  A point then costs one compare, masked by the
+// digits the required flags allow for its triple (fixed for the whole kernel).
+struct CountTables {
+  u64 bound[5][4];       // [digit][variant]
+  u64 host_bound[4];     // the triple's own host bytes must stay below this to offload activations
+};
+
+template <int NM, bool POW2>
+__global__ void __launch_bounds__(THREADS, 2) k_compact_count(SpaceDev sp, EvalArgs a) {
+  constexpr int N2 = NM * NM, N3 = NM * NM * NM, NC = N3 * NM;
+  constexpr int R = (N3 + 31) / 32;
+  __shared__ CountTables tables[WARPS];
+  const int lane = threadIdx.x & 31;
+  const u32 run = blockIdx.x * WARPS + (threadIdx.x >> 5);
+  if (run >= a.n_runs) return;
+  CountTables& tb = tables[threadIdx.x >> 5];
+  const u32 seg_begin = run * a.run_len;
+  const u32 seg_end = min(seg_begin + a.run_len, a.n_tiles);
+  const u32 groups_per_model = sp.n_facts * sp.nvt;
+  const u32 modemap = (NM == 5) ? 0x43210u : sp.modemap;
+  const u32 req = a.require_flags;
+  constexpr u32 CV_BITS = PS_F_CV | PS_F_T_DIV_HEADS | PS_F_K_DIV_LAYERS | PS_F_TP_LE_MAX | PS_F_AXIS_FORM;
+  const u32 req_cv = req & CV_BITS;
+  // capacities as exclusive bounds (memory and host bytes stay below 2^62)
+  const u64 cap_x = min(a.cap_bytes, (u64)1 << 62) + 1;
+  const u64 host_x = min(a.host_cap, (u64)1 << 62) + 1;
+  u32 all = (1u << NM) - 1u, own = 0, is_o = 0, not_mo = 0;
+#pragma unroll
+  for (int d = 0; d < NM; ++d) {
+    const u32 ac = digit_mode(modemap, d);
+    if (in_set(SET_ACT_OWN, ac)) own |= 1u << d;
+    if (ac == PS_MODE_O) is_o |= 1u << d;
+    if (!in_set(SET_M_OR_O, ac)) not_mo |= 1u << d;
+  }
+  // the lane's triples: modes and the activation digits the required flags allow
+  // (bits 0..4 with several replicas, bits 8..12 with one), fixed for the kernel
+  u32 th[R], om[R], gr[R], t_allowed[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const u32 t = lane + 32 * r;
+    const bool live = t < (u32)N3;
+    const u32 tt = live ? t : 0;
+    th[r] = digit_mode(modemap, tt % NM);
+    om[r] = digit_mode(modemap, (tt / NM) % NM);
+    gr[r] = digit_mode(modemap, tt / N2);
+    const u32 a_many = allowed_act_digits(triple_bits(th[r], om[r], gr[r], false), req, all, own, is_o, not_mo);
+    const u32 a_one = allowed_act_digits(triple_bits(th[r], om[r], gr[r], true), req, all, all, is_o, not_mo);
+    t_allowed[r] = live ? (a_many | (a_one << 8)) : 0;
+  }
+  // this lane's table entry (variant, digit)
+  const u32 tl_vt = lane / NM, tl_d = lane - tl_vt * NM;
+  const bool tl_mine = tl_vt < sp.nvt;
+  const u32 tl_v = tl_mine ? tl_vt / sp.nt : 0;
+  const u32 tl_tau = tl_mine ? tl_vt - tl_v * sp.nt : 0;
+  const u32 tl_mode = digit_mode(modemap, tl_d);
+
+  u32 model_cur = 0xffffffffu, unit_cur = 0xffffffffu;
+  ModelRec rec;
+  u32 ka[R], kb[R], kc[R], kh[R];
+  u64 mem3[R], host3[R];
+  u32 allowed[R];
+  u64 run_total = 0;
+  u32 with_survivors = 0;                  // bit j: group seg_begin + j has survivors
+  const u64 window_end = a.first + a.count;
+
+  for (u32 seg = seg_begin; seg < seg_end; ++seg) {
+    const u64 g = a.first_group + seg;
+    const u32 model = (u32)(g / groups_per_model);
+    const u32 gl = (u32)(g - (u64)model * groups_per_model);
+    const u32 unit = gl / sp.nvt, vt = gl - unit * sp.nvt;
+    if (model != model_cur) {
+      model_cur = model;
+      unit_cur = 0xffffffffu;
+      const uint4* src = reinterpret_cast<const uint4*>(&sp.recs[model]);
+      uint4* dst = reinterpret_cast<uint4*>(&rec);
+#pragma unroll
+      for (int k = 0; k < 6; ++k) dst[k] = __ldg(src + k);
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const u32 modes[3] = {th[r], om[r], gr[r]};
+        const u32 width[3] = {rec.wT, rec.wO, rec.wG};
+        u32 ca = 0, cb = 0, cc = 0;
+#pragma unroll
+        for (int s = 0; s < 3; ++s) {        // Theorem 1: R holds E, S and S* a shard, S* and M a unit
+          if (modes[s] == PS_MODE_R) ca += width[s];
+          if (in_set(SET_SHARDLIKE, modes[s])) cb += width[s];
+          if (modes[s] == PS_MODE_SG) cc += width[s] * sp.sstar_units;
+          if (modes[s] == PS_MODE_M) cc += width[s];
+        }
+        ka[r] = ca; kb[r] = cb; kc[r] = cc;
+        kh[r] = (th[r] == PS_MODE_O ? (2 * sp.accum + 1) * rec.wT : 0) + (om[r] == PS_MODE_O ? 2 * rec.wO : 0) +
+                (gr[r] == PS_MODE_O ? 2 * rec.wG : 0);
+      }
+    }
+    if (unit != unit_cur) {
+      unit_cur = unit;
+      const Fact f = sp.facts[unit];
+      const Pow2 p2 = pow2_of(f);
+      const UnitBase ub = (POW2 || p2.all) ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
+                                           : unit_base(rec, f, sp.tp_max_valid, true);
+      __syncwarp();                            // the previous factorisation's bounds have been read
+      if (tl_mine) {
+        const ActBase ab = (POW2 || p2.all) ? act_base_pow2(rec, p2, tl_v, tl_tau) : act_base(rec, f, tl_v, tl_tau);
+        const u64 am = mu_elems(tl_mode, ab.EA, ab.shA, ab.uA, sp.sstar_units);
+        tb.bound[tl_d][tl_vt] = am < cap_x ? cap_x - am : 0;
+        if (tl_d == 0) {
+          const u64 ah = 2 * ab.EA * sp.accum;  // offloaded after forward, reloaded for backward, per micro-batch
+          tb.host_bound[tl_vt] = ah < host_x ? host_x - ah : 0;
+        }
+      }
+      __syncwarp();
+      const bool unit_ok = (ub.cv & req_cv) == req_cv;
+      const u32 shift = ub.d1 ? 8 : 0;
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        mem3[r] = mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0)));
+        host3[r] = mad_small(ub.sh, kh[r], 0);
+        allowed[r] = (unit_ok && host3[r] < host_x) ? ((t_allowed[r] >> shift) & all) : 0;
+      }
+    }
+    // the group's codes inside the window
+    const u64 group_first = g * NC;
+    const u32 code_lo = a.first > group_first ? (u32)(a.first - group_first) : 0u;
+    const u32 code_hi = window_end < group_first + NC ? (u32)(window_end - group_first) : (u32)NC;
+    const bool whole = code_lo == 0 && code_hi == (u32)NC;
+    const u64 host_bound = tb.host_bound[vt];
+    u32 n = 0;
+#pragma unroll
+    for (int d = 0; d < NM; ++d) {
+      const u64 bound = tb.bound[d][vt];
+      const bool offload = (is_o >> d) & 1u;
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        bool pass = ((allowed[r] >> d) & 1u) && mem3[r] < bound && (!offload || host3[r] < host_bound);
+        if (!whole) {
+          const u32 code = lane + 32 * r + d * N3;
+          pass = pass && code >= code_lo && code < code_hi;
+        }
+        n += pass ? 1u : 0u;
+      }
+    }
+    n = __reduce_add_sync(0xffffffffu, n);
+    if (lane == 0) a.tile_count[seg] = n;
+    run_total += n;
+    if (n) with_survivors |= 1u << (seg - seg_begin);
+  }
+  if (lane == 0) a.tile_offset[run] = run_total;
+  // the groups with survivors join the write pass's list (in any order: a group's place
+  // in the output comes from the scan, not from the list)
+  const u32 n_listed = __popc(with_survivors);
+  if (n_listed) {
+    u32 base = 0;
+    if (lane == 0) base = atomicAdd(a.n_nonempty, n_listed);
+    base = __shfl_sync(0xffffffffu, base, 0);
+    if ((with_survivors >> lane) & 1u)
+      a.nonempty[base + __popc(with_survivors & ((1u << lane) - 1u))] = seg_begin + lane;
+  }
 }
 
 // exclusive prefix sum, in place, of the survivors of the count pass's runs
@@ -430,11 +586,10 @@ cudaError_t launch_eval_p(const SpaceDev& sp, const EvalArgs& a, cudaStream_t st
   // one warp per run of groups; enough blocks to fill the GPU, no more than groups
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const unsigned needed = ((MODE == MODE_COUNT ? a.n_runs : a.n_tiles) + WARPS - 1) / WARPS;
+  const unsigned needed = (a.n_tiles + WARPS - 1) / WARPS;
   const unsigned most = (unsigned)sms * (MODE == MODE_MATERIALISE ? EVAL_GRID_PER_SM_MATERIALISE
-                                         : MODE == MODE_WRITE     ? EVAL_GRID_PER_SM_WRITE
-                                                                  : EVAL_GRID_PER_SM_COMPACT);
-  const unsigned blocks = (MODE == MODE_COUNT || needed < most) ? needed : most;   // count: a warp per run
+                                                                  : EVAL_GRID_PER_SM_WRITE);
+  const unsigned blocks = needed < most ? needed : most;
   constexpr int NC = NM * NM * NM * NM;
   const size_t smem = MODE == MODE_MATERIALISE ? (size_t)WARPS * 2 * Stage<NC>::BYTES : 0;
   if (smem > 48 * 1024) {
@@ -480,8 +635,21 @@ void eval_plan_runs(EvalArgs& a) {
 cudaError_t launch_eval_materialise(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream) {
   return launch_eval_m<MODE_MATERIALISE>(sp, a, stream);
 }
+template <int NM>
+static cudaError_t launch_count_t(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream) {
+  const unsigned blocks = (a.n_runs + WARPS - 1) / WARPS;       // a warp per run
+  if (sp.all_pow2) k_compact_count<NM, true><<<blocks, THREADS, 0, stream>>>(sp, a);
+  else k_compact_count<NM, false><<<blocks, THREADS, 0, stream>>>(sp, a);
+  return cudaGetLastError();
+}
 cudaError_t launch_eval_count(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream) {
-  return launch_eval_m<MODE_COUNT>(sp, a, stream);
+  switch (sp.nm) {
+    case 1: return launch_count_t<1>(sp, a, stream);
+    case 2: return launch_count_t<2>(sp, a, stream);
+    case 3: return launch_count_t<3>(sp, a, stream);
+    case 4: return launch_count_t<4>(sp, a, stream);
+    default: return launch_count_t<5>(sp, a, stream);
+  }
 }
 cudaError_t launch_tile_scan(const EvalArgs& a, cudaStream_t stream) {
   k_tile_scan<<<1, SCAN_THREADS, 0, stream>>>(a);

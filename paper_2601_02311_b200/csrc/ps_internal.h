@@ -118,6 +118,8 @@ struct EvalArgs {
   // consecutive groups (one warp per run) -- set by eval_plan_runs
   u32 n_runs, run_len;
   u32* tile_count;          // [n_tiles] survivors of each group
+  u32* nonempty;            // [n_tiles] the groups that have survivors, in any order
+  u32* n_nonempty;          // how many (zero before the count pass)
   u64* tile_offset;         // [n_runs <= n_tiles] survivors of each run, then (scan) of all runs before it
   u32* status;
 };
@@ -143,3 +145,9 @@ size_t verify_workspace_doubles(const ps_verify_shape& s);     // per case
 cudaError_t launch_verify(const ps_verify_shape& s, const ps_verify_case* d_cases, u64 n, const double* d_data,
                           u64 data_len, double* d_ws, double* d_theta_out, ps_verify_result* d_out, u32* status,
                           cudaStream_t stream);
+
+cudaError_t launch_select_compare(const SpaceDev& sp, u32 unit_begin, u32 unit_end, u32 N, u64 device_bytes, u32 fast,
+                                  u32 head_num, u32 head_den, u32 layer_num, u32 layer_den, u32 tp_degree,
+                                  u64 host_cap, u32 require_flags, u32 comm_kind, const ps_front_entry* d_frontier,
+                                  const u32* d_counts, u32 n_caps, u32 cap_index, u32 max_entries,
+                                  ps_select_compare_result* d_out, cudaStream_t stream);

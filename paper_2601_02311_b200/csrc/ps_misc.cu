@@ -161,6 +161,73 @@ __global__ void __launch_bounds__(SELECT_THREADS) k_select(const ps_select_query
   }
 }
 
+// Algorithm 1's choice for every model of a space, as a point of the space, against
+// the model's frontier (one thread per model).
+__global__ void __launch_bounds__(128) k_select_compare(SpaceDev sp, u32 unit_begin, u32 unit_end, u32 N,
+                                                        u64 device_bytes, u32 fast, u32 head_num, u32 head_den,
+                                                        u32 layer_num, u32 layer_den, u32 tp_degree, u64 host_cap,
+                                                        u32 require_flags, u32 comm_kind,
+                                                        const ps_front_entry* __restrict__ frontier,
+                                                        const u32* __restrict__ counts, u32 n_caps, u32 cap_index,
+                                                        u32 max_entries, ps_select_compare_result* __restrict__ out) {
+  const u32 model = blockIdx.x * blockDim.x + threadIdx.x;
+  if (model >= sp.n_models) return;
+  const ModelRec rec = sp.recs[model];
+  ps_select_query q;
+  q.param_elems = rec.P; q.layer_elems = rec.unit; q.device_bytes = device_bytes; q.n_devices = N;
+  q.w_param = (uint8_t)rec.wT; q.w_grad = (uint8_t)rec.wG; q.w_opt = (uint8_t)rec.wO;
+  q.fast_interconnect = (uint8_t)(fast ? 1 : 0);
+  const ps_select_result pick = select_one(q, head_num, head_den, layer_num, layer_den, tp_degree);
+  ps_select_compare_result r;
+  r.branch = pick.branch; r.T = pick.T; r.code_dp = pick.code_dp; r.pad = 0;
+  u32 status = 0;
+  // the choice as a point of the space: (N, T, K = 1), first variants, the code's modes as digits
+  const u32 modes[4] = {pick.code_dp % 5, (pick.code_dp / 5) % 5, (pick.code_dp / 25) % 5, pick.code_dp / 125};
+  u32 digits[4];
+  bool in_space = true;
+  for (int st = 0; st < 4; ++st) {
+    digits[st] = 0xffffffffu;
+    for (u32 d = 0; d < sp.nm; ++d)
+      if (digit_mode(sp.modemap, d) == modes[st]) digits[st] = d;
+    in_space = in_space && digits[st] != 0xffffffffu;
+  }
+  u32 unit = 0xffffffffu;
+  for (u32 u = unit_begin; u < unit_end; ++u) {
+    const Fact f = sp.facts[u];
+    if (f.N == N && f.T == pick.T && f.K == 1) { unit = u; break; }
+  }
+  in_space = in_space && unit != 0xffffffffu;
+  const Fact f = in_space ? sp.facts[unit] : Fact{N, pick.T, 1, N / pick.T};
+  const PointOut po = eval_point(rec, f, 0, 0, modes[0], modes[1], modes[2], modes[3], sp.tp_max_valid, sp.tp_coll,
+                                 true, sp.sstar_units, sp.accum);
+  const u64 comm = comm_kind == PS_COMM_PAPER ? po.comm_paper : po.comm_paper + po.comm_ext;
+  r.alg_mem = po.mem; r.alg_comm = comm;
+  r.alg_idx = 0;
+  if (in_space) {
+    const u32 code = digits[0] + sp.nm * (digits[1] + sp.nm * (digits[2] + sp.nm * digits[3]));
+    r.alg_idx = (u64)model * sp.ppm + (u64)unit * sp.nvt * sp.n_codes + code;
+    status |= PS_SEL_IN_SPACE;
+  }
+  const bool fits = po.mem <= device_bytes;
+  r.alg_flags = po.flags | (fits ? PS_F_FEASIBLE : 0);
+  if (fits && po.host <= host_cap && (po.flags & require_flags) == require_flags) status |= PS_SEL_SURVIVOR;
+  // the frontier of this model under this capacity
+  const u32 count = counts[(u64)model * n_caps + cap_index];
+  const ps_front_entry* fr = frontier + ((u64)model * n_caps + cap_index) * max_entries;
+  const u32 written = count < max_entries ? count : max_entries;
+  if (count == 0) status |= PS_SEL_FRONTIER_EMPTY;
+  if (count > max_entries) status |= PS_SEL_FRONTIER_TRUNCATED;
+  r.best_mem = 0; r.best_comm = 0; r.best_idx = 0;
+  for (u32 e = 0; e < written; ++e) {
+    const u64 m = fr[e].mem, c = fr[e].comm;
+    if (m == po.mem && c == comm) status |= PS_SEL_ON_FRONTIER;
+    else if (m <= po.mem && c <= comm) status |= PS_SEL_DOMINATED;
+  }
+  if (written) { r.best_mem = fr[written - 1].mem; r.best_comm = fr[written - 1].comm; r.best_idx = fr[written - 1].idx; }
+  r.status = status;
+  out[model] = r;
+}
+
 // 8 independent chains per thread; each round applies to every chain an add
 // and an xor with loop-carried values the compiler cannot fold, so a round is
 // 16 independent-across-chains 32-bit operations and a chain's operations are
@@ -209,5 +276,16 @@ cudaError_t launch_select(const ps_select_query* d_q, u64 n, u32 head_num, u32 h
 
 cudaError_t launch_int_peak(u32 blocks, u32 iters, u32* d_sink, cudaStream_t stream) {
   k_int_peak<<<blocks, 256, 0, stream>>>(iters, d_sink);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_select_compare(const SpaceDev& sp, u32 unit_begin, u32 unit_end, u32 N, u64 device_bytes, u32 fast,
+                                  u32 head_num, u32 head_den, u32 layer_num, u32 layer_den, u32 tp_degree,
+                                  u64 host_cap, u32 require_flags, u32 comm_kind, const ps_front_entry* d_frontier,
+                                  const u32* d_counts, u32 n_caps, u32 cap_index, u32 max_entries,
+                                  ps_select_compare_result* d_out, cudaStream_t stream) {
+  k_select_compare<<<(sp.n_models + 127) / 128, 128, 0, stream>>>(
+      sp, unit_begin, unit_end, N, device_bytes, fast, head_num, head_den, layer_num, layer_den, tp_degree, host_cap,
+      require_flags, comm_kind, d_frontier, d_counts, n_caps, cap_index, max_entries, d_out);
   return cudaGetLastError();
 }

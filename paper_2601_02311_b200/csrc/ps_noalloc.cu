@@ -13,12 +13,14 @@
 namespace {
 
 constexpr size_t COUNT_BYTES = sizeof(u32) * (size_t)PS_NOALLOC_MAX_GROUPS;
+constexpr size_t LENGTH_BYTES = 256;
 constexpr size_t OFFSET_BYTES = sizeof(u64) * (size_t)PS_NOALLOC_MAX_GROUPS;
 
-// 1.5 MiB on every GPU that loads the library, for the life of the process:
-// [0, COUNT_BYTES) survivor count of each group, then the exclusive prefix sums
-// (one per run of groups, so at most one per group).
-static __device__ __align__(256) unsigned char g_fixed_scratch[COUNT_BYTES + OFFSET_BYTES];
+// 2 MiB on every GPU that loads the library, for the life of the process:
+// [0, COUNT_BYTES) survivor count of each group, then the list of groups that
+// have survivors, its length, and the exclusive prefix sums (one per run of
+// groups, so at most one per group).
+static __device__ __align__(256) unsigned char g_fixed_scratch[2 * COUNT_BYTES + LENGTH_BYTES + OFFSET_BYTES];
 
 constexpr int MAX_DEVICES = 64;
 std::mutex g_setup_lock;
@@ -97,8 +99,11 @@ extern "C" int ps_eval_compact_noalloc(ps_ctx* ctx, const ps_space* sp, uint64_t
   a.cap_bytes = filter->cap_bytes;
   a.host_cap = filter->host_cap;
   a.require_flags = filter->require_flags & ~(u32)PS_F_FEASIBLE;
-  a.tile_count = static_cast<u32*>(base);
-  a.tile_offset = reinterpret_cast<u64*>(static_cast<unsigned char*>(base) + COUNT_BYTES);
+  unsigned char* bytes = static_cast<unsigned char*>(base);
+  a.tile_count = reinterpret_cast<u32*>(bytes);
+  a.nonempty = reinterpret_cast<u32*>(bytes + COUNT_BYTES);
+  a.n_nonempty = reinterpret_cast<u32*>(bytes + 2 * COUNT_BYTES);
+  a.tile_offset = reinterpret_cast<u64*>(bytes + 2 * COUNT_BYTES + LENGTH_BYTES);
   eval_plan_runs(a);
   // The array still holds the previous call's numbers.  Every word this call
   // reads is written earlier in this call (the count pass stores a count for
@@ -106,6 +111,7 @@ extern "C" int ps_eval_compact_noalloc(ps_ctx* ctx, const ps_space* sp, uint64_t
   // into offsets); the counts are cleared anyway so that a stale value can
   // never be mistaken for a fresh one.
   if (cudaMemsetAsync(a.tile_count, 0, sizeof(u32) * n_groups, ctx->stream) != cudaSuccess) return PS_E_CUDA;
+  if (cudaMemsetAsync(a.n_nonempty, 0, sizeof(u32), ctx->stream) != cudaSuccess) return PS_E_CUDA;   // the list starts empty
   if (launch_eval_count(sp->dev, a, ctx->stream) != cudaSuccess) return PS_E_CUDA;
   if (launch_tile_scan(a, ctx->stream) != cudaSuccess) return PS_E_CUDA;
   if (launch_eval_write(sp->dev, a, ctx->stream) != cudaSuccess) return PS_E_CUDA;

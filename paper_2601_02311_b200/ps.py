@@ -47,7 +47,7 @@ EXPORTS = ("ps_create", "ps_destroy", "ps_status", "ps_strerror", "ps_space_crea
            "ps_space_destroy", "ps_space_set_models", "ps_space_rederive", "ps_space_size",
            "ps_space_points_per_model", "ps_space_decode", "ps_eval_batch", "ps_sweep_pareto",
            "ps_check_composition", "ps_int_peak", "ps_eval_compact_noalloc", "ps_select",
-           "ps_verify_batch")
+           "ps_verify_batch", "ps_select_compare")
 
 
 class _SpaceDesc(C.Structure):
@@ -78,6 +78,11 @@ class _VerifyShape(C.Structure):
                 ("rtol", C.c_double), ("atol", C.c_double)]
 
 
+SELECT_COMPARE_DTYPE = np.dtype([("alg_mem", "<u8"), ("alg_comm", "<u8"), ("alg_idx", "<u8"), ("best_mem", "<u8"),
+                                 ("best_comm", "<u8"), ("best_idx", "<u8"), ("branch", "<u4"), ("T", "<u4"),
+                                 ("code_dp", "<u4"), ("alg_flags", "<u4"), ("status", "<u4"), ("pad", "<u4")])
+SEL_IN_SPACE, SEL_SURVIVOR, SEL_ON_FRONTIER, SEL_DOMINATED, SEL_FRONTIER_EMPTY, SEL_FRONTIER_TRUNCATED = \
+    1, 2, 4, 8, 16, 32
 VERIFY_CASE_DTYPE = np.dtype([("code", "<u4"), ("D", "<u4"), ("data_offset", "<u8")])
 VERIFY_RESULT_DTYPE = np.dtype([("mem", "<u8"), ("comm", "<u8"), ("host", "<u8"), ("match", "<u4"),
                                 ("pad", "<u4"), ("max_rel_err", "<f8")])
@@ -116,6 +121,9 @@ _lib.ps_check_composition.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_ui
                                       C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p]
 _lib.ps_select.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32,
                            C.c_uint32, C.c_uint32, C.c_void_p]
+_lib.ps_select_compare.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint64, C.c_uint32, C.c_uint32,
+                                   C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32, C.POINTER(_Filter), C.c_void_p,
+                                   C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p]
 _lib.ps_verify_batch.argtypes = [C.c_void_p, C.POINTER(_VerifyShape), C.c_void_p, C.c_uint64, C.c_void_p,
                                  C.c_uint64, C.c_void_p, C.c_void_p]
 _lib.ps_int_peak.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_void_p,
@@ -354,6 +362,18 @@ class Space:
         _check(_lib.ps_sweep_pareto(self.ctx._h, self._h, C.byref(f), caps.ctypes.data, len(caps),
                                     kind, max_entries, _dptr(d_out), _dptr(d_counts)),
                "ps_sweep_pareto")
+
+    def select_compare(self, n_index: int, device_bytes: int, filt: dict, d_frontier: torch.Tensor,
+                       d_counts: torch.Tensor, n_caps: int, cap_index: int, max_entries: int, fast: int = 1,
+                       headroom=(7, 10), layer=(3, 10), tp_degree: int = 8) -> np.ndarray:
+        """ps_select_compare on the device outputs of a Pareto sweep; returns SELECT_COMPARE_DTYPE records."""
+        d_out = torch.zeros(self.n_models * 72, dtype=torch.uint8, device=self.ctx.torch_device)
+        f = _mk_filter(filt)
+        _check(_lib.ps_select_compare(self.ctx._h, self._h, n_index, device_bytes, fast, headroom[0], headroom[1],
+                                      layer[0], layer[1], tp_degree, C.byref(f), _dptr(d_frontier), _dptr(d_counts),
+                                      n_caps, cap_index, max_entries, _dptr(d_out)), "ps_select_compare")
+        self.ctx.check_status()
+        return d_out.cpu().numpy().view(SELECT_COMPARE_DTYPE)
 
     def alloc_sweep(self, n_caps: int, max_entries: int):
         dev = self.ctx.torch_device

@@ -1,7 +1,9 @@
 """Parity at the full sizes of the benchmark configurations, in the launch
 configuration bench.py times (whole shape table, same filters and capacities):
-sampled models and windows against the oracle, bit for bit, and properties of
-the complete outputs that hold at any size."""
+the complete top-64 and Pareto tables of every model and 64 windows of 2^20
+points against the oracle, bit for bit (marked slow: a few minutes of oracle
+time on all host cores), a quicker sampled version of the same, and properties
+of the complete outputs that hold at any size."""
 import numpy as np
 import pytest
 
@@ -97,3 +99,49 @@ def test_random_windows_of_the_full_space(ctx, name):
     got, want = gs.eval_batch(size - 1000, 1000), os_.eval_range(size - 1000, 1000)
     for k in want:
         assert np.array_equal(got[k], want[k])
+
+
+@pytest.mark.slow
+@pytest.mark.parametrize("name", ["C3", "C4"])
+def test_full_sweeps_every_model(ctx, ps, name):
+    """Every model's top-64 list and both capacities' Pareto frontiers, whole tables."""
+    space = synth.config(name)
+    gs, os_ = ctx.space(space), O.Space(space)
+    threads = O.hardware_threads()
+    topk_f = dict(require_flags=VALID)
+    par_f = dict(require_flags=VALID, host_cap=64 * GB)
+    caps = [80 * GB, 192 * GB]
+    te, tc = gs.sweep(topk_f, caps[1:], ps.REDUCE_TOPK, 64)
+    oe, oc = os_.sweep(topk_f, caps[1:], O.KIND_TOPK, 64, n_threads=threads)
+    assert np.array_equal(tc, oc)
+    assert te.tobytes() == oe.tobytes()
+    del oe
+    pe, pc = gs.sweep(par_f, caps, ps.REDUCE_PARETO, 64)
+    oe, oc = os_.sweep(par_f, caps, O.KIND_PARETO, 64, n_threads=threads)
+    assert np.array_equal(pc, oc)
+    assert pe.tobytes() == oe.tobytes()
+
+
+@pytest.mark.slow
+@pytest.mark.parametrize("name", ["C4", "C2"])
+def test_64_windows_of_a_million_points(ctx, name):
+    """ps_eval_batch on 64 pseudo-randomly placed windows of 2^20 points: every output word."""
+    import concurrent.futures as cf
+    space = synth.config(name)
+    gs, os_ = ctx.space(space), O.Space(space)
+    size, count = gs.size, 1 << 20
+    rng = np.random.default_rng(2020)
+    firsts = [int(rng.integers(0, size - count)) for _ in range(64)]
+    filt = dict(require_flags=VALID, cap_bytes=80 * GB)
+    # the oracle walks a window on one core (its C code releases the interpreter lock): windows side by side
+    with cf.ThreadPoolExecutor(max_workers=O.hardware_threads()) as pool:
+        wants = list(pool.map(lambda f: os_.eval_range(f, count), firsts))
+        compact_wants = list(pool.map(lambda f: os_.compact_range(f, count, filt), firsts[::8]))
+    for w, first in enumerate(firsts):
+        got = gs.eval_batch(first, count)
+        for k in wants[w]:
+            assert np.array_equal(got[k], wants[w][k]), (w, first, k)
+    for w, first in enumerate(firsts[::8]):
+        got = gs.compact(first, count, filt)
+        for k in compact_wants[w]:
+            assert np.array_equal(got[k], compact_wants[w][k]), (w, first, k)

@@ -416,3 +416,27 @@ def test_pareto_frontier_longer_than_the_fast_lists(ctx, ps):
     mixed["models"] = np.concatenate([synth.zoo(2, 6), space["models"], synth.zoo(2, 7)])
     gs, os_ = both(ctx, mixed)
     assert_same_sweep(gs.sweep(filt, caps, ps.REDUCE_PARETO, 192), os_.sweep(filt, caps, O.KIND_PARETO, 192, n_threads=8))
+
+
+def test_select_compare_matches_oracle(ctx, ps):
+    """Algorithm 1's choice beside the frontier, for every model of a single-N composition space."""
+    import torch
+    for n_value, mask in ((64, 0x1F), (512, 0b10111)):
+        space = synth.config("C3", n_models=40)
+        space["n_values"] = np.array([n_value], dtype=np.uint32)
+        space["mode_mask"] = mask
+        gs, os_ = both(ctx, space)
+        filt = dict(require_flags=VALID, host_cap=64 * synth.GB)
+        caps = [40 * synth.GB, 80 * synth.GB]
+        d_out, d_counts = gs.alloc_sweep(len(caps), 24)
+        gs.sweep_into(filt, caps, ps.REDUCE_PARETO, 24, d_out, d_counts)
+        oe, oc = os_.sweep(filt, caps, O.KIND_PARETO, 24, n_threads=8)
+        for cap_index in (0, 1):
+            got = gs.select_compare(0, caps[cap_index], filt, d_out, d_counts, len(caps), cap_index, 24)
+            want = O.select_compare(os_, 0, caps[cap_index], filt, oe, oc, cap_index)
+            names = ("alg_mem", "alg_comm", "alg_idx", "best_mem", "best_comm", "best_idx", "branch", "T",
+                     "code_dp", "alg_flags", "status")
+            for k, name in enumerate(names):
+                assert np.array_equal(got[name].astype(np.uint64), want[:, k]), (n_value, cap_index, name)
+        assert len(set(got["status"].tolist())) > 1            # more than one outcome occurs
+    ctx.check_status()

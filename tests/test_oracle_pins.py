@@ -455,3 +455,35 @@ def test_algorithm1_thresholds_are_strict_and_exact():
     # tensor parallelism divides the state before the data axis shards it (Remark 4)
     E2 = -(-big // 8)
     assert r[1, 0] == 16 * E2 + 2 * (-(-187_500_001 // 8))
+
+
+def test_algorithm1_beside_the_frontier_on_the_papers_example():
+    """70B parameters on 80 GB devices, data axis only.  Among the placements built
+    from R, S and S* Algorithm 1's ZeRO-3 is the whole frontier from N = 32 on:
+    16P/N bytes and 3 (N-1)/N |G| of traffic, 1.5x data parallelism's.  With all
+    five modes it is off the frontier: consuming gradients as they are produced
+    (S*, S, M, R) moves the same bytes and holds 2P/N less.  At N = 8 nothing fits."""
+    P, Md = GOLD["P"], 80 * synth.GB
+    filt = dict(require_flags=O.F_GI | O.F_SC, host_cap=0, comm_kind=O.COMM_PAPER_PLUS_EXT)
+    for N in (32, 64):
+        x = 2 * (P - P // N)                                   # ring volume of |G| = |Theta| = 2P bytes
+        for mask, on in ((0b00111, True), (0x1F, False)):
+            space = synth._space(synth.worked_example(False), [N], t_enum_max=1, k_enum_max=1, n_act=1, n_tpa=1,
+                                 mode_mask=mask)
+            sp = O.Space(space)
+            e, c = sp.sweep(filt, [Md], O.KIND_PARETO, 16)
+            r = O.select_compare(sp, 0, Md, filt, e, c, 0)[0]
+            assert (r[6], r[7], r[8]) == (1, 1, 32)            # branch 1: ZeRO-3
+            assert r[0] == 16 * P // N and r[1] == 3 * x and 2 * r[1] == 3 * (2 * x)
+            assert r[10] == (1 | 2 | 4 if on else 1 | 2 | 8)
+            if on:
+                assert c[0, 0] == 1 and (r[3], r[4], r[5]) == (r[0], r[1], r[2])
+            else:
+                assert (r[3], r[4]) == (14 * P // N, 3 * x)    # no gradient shard is kept
+                assert sp.decode(int(r[5]))["code_dp"] == code_of(SG, S, M, R)
+    space = synth._space(synth.worked_example(False), [8], t_enum_max=1, k_enum_max=1, n_act=1, n_tpa=1,
+                         mode_mask=0x1F)
+    sp = O.Space(space)
+    e, c = sp.sweep(filt, [Md], O.KIND_PARETO, 16)
+    r = O.select_compare(sp, 0, Md, filt, e, c, 0)[0]
+    assert r[6] == 3 and r[10] == (1 | 16) and r[0] == 16 * P // 8
