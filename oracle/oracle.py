@@ -42,7 +42,7 @@ class _Desc(C.Structure):
                 ("tp_max_valid", C.c_uint32), ("n_act_variants", C.c_uint32),
                 ("n_tpa_variants", C.c_uint32), ("mode_mask", C.c_uint32),
                 ("tp_coll_per_layer", C.c_uint32), ("sstar_units", C.c_uint32),
-                ("grad_accum_steps", C.c_uint32)]
+                ("grad_accum_steps", C.c_uint32), ("replication_k", C.c_uint32)]
 
 
 class _Filter(C.Structure):
@@ -98,7 +98,7 @@ class Space:
                           space["tp_max_valid"], space["n_act_variants"],
                           space["n_tpa_variants"], space["mode_mask"],
                           space["tp_coll_per_layer"], space.get("sstar_units", 1),
-                          space.get("grad_accum_steps", 1))
+                          space.get("grad_accum_steps", 1), space.get("replication_k", 1))
         self.params = {k: v for k, v in space.items() if k not in ("models", "n_values")}
 
     @property
@@ -202,11 +202,11 @@ def model_record(shape: np.ndarray) -> dict:
 
 
 def eval_record(rec: dict, N, T, K, D, v, tau, code, tp_max_valid=8, tp_coll_per_layer=4,
-                sstar_units=1, grad_accum_steps=1) -> dict:
+                sstar_units=1, grad_accum_steps=1, replication_k=1) -> dict:
     r = np.array([rec[k] for k in RECORD_FIELDS], dtype=np.uint64)
     out = np.zeros(5, dtype=np.uint64)
     lib().orc_eval_record(_ptr(r), N, T, K, D, v, tau, code, tp_max_valid, tp_coll_per_layer,
-                          sstar_units, grad_accum_steps, _ptr(out))
+                          sstar_units, grad_accum_steps, replication_k, _ptr(out))
     return dict(mem=int(out[0]), comm_paper=int(out[1]), comm_ext=int(out[2]), host=int(out[3]),
                 flags=int(out[4]))
 

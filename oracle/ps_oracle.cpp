@@ -68,6 +68,8 @@ struct ODesc {  // the design space
   u32 n_act_variants, n_tpa_variants, mode_mask, tp_coll_per_layer;
   u32 sstar_units;       // 0 or 1: Theorem 1 as stated; 2: overlapped gathers (the proof's note)
   u32 grad_accum_steps;  // 0 or 1: none; g: micro-batches per step ("Limitations")
+  u32 replication_k;     // 0 or 1: plain sharding; k: every shard is held k times (Section 1's
+                         // "k-way replication for 1 < k < N")
 };
 
 struct OFilter {
@@ -164,14 +166,22 @@ void mu_elems(int pi, u64 E, u64 u, u64 D, u64 gather_buffers, u64* persistent, 
   }
 }
 
+u64 gcd_u64(u64 a, u64 b) { while (b) { u64 t = a % b; a = b; b = t; } return a; }
+
 OResult eval_point(const ORecord& m, u64 N, u64 T, u64 K, u64 D, int v, int tau,
                    int pi_theta, int pi_omega, int pi_grad, int pi_act,
                    u32 tp_max_valid, u32 tp_coll_per_layer, bool axis_form_ok,
-                   u32 sstar_units = 1, u32 grad_accum_steps = 1) {
+                   u32 sstar_units = 1, u32 grad_accum_steps = 1, u32 replication_k = 1) {
   OResult out;
-  // the two extensions: unit buffers of a gathered state, micro-batches per step
+  // the extensions: unit buffers of a gathered state, micro-batches per step
   const u64 nbuf = sstar_units ? sstar_units : 1;
   const u64 g = grad_accum_steps ? grad_accum_steps : 1;
+  // k-way replication of the sharded modes: the D devices of the data axis form
+  // k shard groups of Gp = D / k devices; a sharded state is cut into Gp shards,
+  // each held by the k devices at the same position of their groups.  Where the
+  // requested k does not divide D the largest common divisor is used.
+  const u64 k = gcd_u64(replication_k ? replication_k : 1, D);
+  const u64 Gp = D / k;
   // Remark 4: tensor parallelism innermost, pipeline in the middle, data
   // outermost.  Table 2: both model axes shard Theta, Omega and G.
   u64 E1 = ceil_div(m.P, T);        // intra-layer split
@@ -185,14 +195,20 @@ OResult eval_point(const ORecord& m, u64 N, u64 T, u64 K, u64 D, int v, int tau,
 
   u64 p, t;
   out.mem = 0;
-  mu_elems(pi_theta, E2, u2, D, nbuf, &p, &t); out.mem += (u64)m.w_theta * (p + t);
-  mu_elems(pi_omega, E2, u2, D, nbuf, &p, &t); out.mem += (u64)m.w_omega * (p + t);
-  mu_elems(pi_grad,  E2, u2, D, nbuf, &p, &t); out.mem += (u64)m.w_grad  * (p + t);
-  mu_elems(pi_act,   EA, uA, D, nbuf, &p, &t); out.mem += p + t;   // already bytes
+  mu_elems(pi_theta, E2, u2, Gp, nbuf, &p, &t); out.mem += (u64)m.w_theta * (p + t);
+  mu_elems(pi_omega, E2, u2, Gp, nbuf, &p, &t); out.mem += (u64)m.w_omega * (p + t);
+  mu_elems(pi_grad,  E2, u2, Gp, nbuf, &p, &t); out.mem += (u64)m.w_grad  * (p + t);
+  mu_elems(pi_act,   EA, uA, Gp, nbuf, &p, &t); out.mem += p + t;   // already bytes
 
-  u64 sh = ceil_div(E2, D);       // largest shard of Theta / Omega / G
-  u64 x = ring_elems(E2, D);      // ring volume in elements
-  u64 xT = x * m.w_theta, xO = x * m.w_omega, xG = x * m.w_grad;
+  u64 sh = ceil_div(E2, Gp);      // largest shard of Theta / Omega / G
+  u64 x = ring_elems(E2, Gp);     // ring volume in elements of a gather or scatter inside a shard group
+  u64 xT = x * m.w_theta, xO = x * m.w_omega;
+  // a gradient reduced to shards: reduce-scatter inside the shard group, then an
+  // all-reduce of every shard across its k copies (the busiest device holds the
+  // largest shard); an all-reduce over all D devices
+  u64 to_shards = (x + 2 * ring_elems(sh, k)) * m.w_grad;
+  u64 all_reduce = 2 * ring_elems(E2, D) * m.w_grad;
+  u64 gatherG = x * m.w_grad;
 
   // Theorem 2: the three priced transitions, nothing else.  With gradient
   // accumulation ("Limitations") a step runs g micro-batches and synchronises
@@ -200,8 +216,8 @@ OResult eval_point(const ORecord& m, u64 N, u64 T, u64 K, u64 D, int v, int tau,
   // forward and backward need is paid g times.  Per micro-batch the gradient
   // terms are thus divided by g, as the paper says.
   out.comm_paper = 0;
-  if (pi_grad == R) out.comm_paper += 2 * xG;          // all-reduce, once per step
-  if (pi_grad == S) out.comm_paper += xG;              // reduce-scatter, once per step
+  if (pi_grad == R) out.comm_paper += all_reduce;      // all-reduce, once per step
+  if (pi_grad == S) out.comm_paper += to_shards;       // reduce-scatter (to shards), once per step
   if (pi_theta == SG) out.comm_paper += g * 2 * xT;    // gather for forward and backward of every micro-batch
 
   // the update is committed on a shard when Omega's home is a shard
@@ -211,9 +227,9 @@ OResult eval_point(const ORecord& m, u64 N, u64 T, u64 K, u64 D, int v, int tau,
   u64 ext_data = 0;
   if (pi_theta == O) ext_data += g * 2 * xT;                 // gather after each host load, every micro-batch
   if (pi_theta == R && update_on_shard) ext_data += xT;      // re-replicate updated shards
-  if (pi_grad == SG) ext_data += 2 * xG;                     // reduce-scatter, then gather
-  if (pi_grad == M) ext_data += (update_on_shard ? 1 : 2) * xG;
-  if (pi_grad == O) ext_data += xG;                          // reduce-scatter before offload
+  if (pi_grad == SG) ext_data += to_shards + gatherG;        // reduce-scatter, then gather
+  if (pi_grad == M) ext_data += update_on_shard ? to_shards : all_reduce;
+  if (pi_grad == O) ext_data += to_shards;                   // reduce-scatter before offload
   if (pi_omega == SG) ext_data += xO;                        // gather Omega for the update
   u64 layers_per_stage = ceil_div(m.L, K);
   u64 ext_tp = layers_per_stage * tp_coll_per_layer * 2 * ring_elems(m.Sbh, T) * m.w_act;
@@ -233,11 +249,14 @@ OResult eval_point(const ORecord& m, u64 N, u64 T, u64 K, u64 D, int v, int tau,
   if (pi_act == O)   out.host += g * 2 * EA;           // store after fwd, load for bwd, every micro-batch
 
   // Theorems 3 and 4 as static predicates over the placement
-  bool omega_full = (pi_omega == R) || (D == 1 && (pi_omega == S || pi_omega == SG));
+  // (a "shard" is the whole tensor when there is one shard position: one device, or
+  // as many copies as devices)
+  bool whole = (Gp == 1);
+  bool omega_full = (pi_omega == R) || (whole && (pi_omega == S || pi_omega == SG));
   bool theta_avail = (pi_theta == R || pi_theta == SG || pi_theta == O) ||
-                     (pi_theta == S && D == 1) || (pi_theta == M && omega_full);
-  bool act_avail = (pi_act == R || pi_act == M || pi_act == O) || D == 1;
-  bool grad_cover = update_on_shard || (pi_grad == R || pi_grad == SG || pi_grad == M) || D == 1;
+                     (pi_theta == S && whole) || (pi_theta == M && omega_full);
+  bool act_avail = (pi_act == R || pi_act == M || pi_act == O) || whole;
+  bool grad_cover = update_on_shard || (pi_grad == R || pi_grad == SG || pi_grad == M) || whole;
   bool gi = theta_avail && act_avail && grad_cover;
   bool sc = (pi_omega != M);
 
@@ -341,7 +360,8 @@ struct Space {
     Decoded p = decode(idx);
     ORecord rec = derive_record(d->models[p.model]);
     return eval_point(rec, p.N, p.T, p.K, p.D, p.v, p.tau, p.pi[0], p.pi[1], p.pi[2], p.pi[3],
-                      d->tp_max_valid, d->tp_coll_per_layer, true, d->sstar_units, d->grad_accum_steps);
+                      d->tp_max_valid, d->tp_coll_per_layer, true, d->sstar_units, d->grad_accum_steps,
+                      d->replication_k);
   }
 };
 
@@ -514,7 +534,7 @@ void orc_check_composition(const OShape* shape, u32 N, u32 T, u32 K, u32 D, u32 
 // UA1, Sbh, L, heads, w_theta, w_omega, w_grad, w_act as 13 u64.
 void orc_eval_record(const u64* rec, u32 N, u32 T, u32 K, u32 D, u32 v, u32 tau, u32 code,
                      u32 tp_max_valid, u32 tp_coll_per_layer, u32 sstar_units, u32 grad_accum_steps,
-                     u64* out5) {
+                     u32 replication_k, u64* out5) {
   ORecord m;
   m.P = rec[0]; m.unit = rec[1]; m.A[0] = rec[2]; m.A[1] = rec[3]; m.UA[0] = rec[4]; m.UA[1] = rec[5];
   m.Sbh = rec[6]; m.L = (u32)rec[7]; m.heads = (u32)rec[8];
@@ -522,7 +542,7 @@ void orc_eval_record(const u64* rec, u32 N, u32 T, u32 K, u32 D, u32 v, u32 tau,
   int pi[4];
   for (int s = 0; s < 4; ++s) { pi[s] = code % 5; code /= 5; }
   OResult r = eval_point(m, N, T, K, D, (int)v, (int)tau, pi[0], pi[1], pi[2], pi[3],
-                         tp_max_valid, tp_coll_per_layer, true, sstar_units, grad_accum_steps);
+                         tp_max_valid, tp_coll_per_layer, true, sstar_units, grad_accum_steps, replication_k);
   out5[0] = r.mem; out5[1] = r.comm_paper; out5[2] = r.comm_ext; out5[3] = r.host; out5[4] = r.flags;
 }
 
@@ -620,7 +640,7 @@ void orc_select_compare(const ODesc* d, u32 n_index, u64 Md, u32 fast, u32 hn, u
     int pi[4]; u32 c = code;
     for (int st = 0; st < 4; ++st) { pi[st] = c % 5; c /= 5; }
     OResult r = eval_point(rec, N, T, 1, N / T, 0, 0, pi[0], pi[1], pi[2], pi[3], d->tp_max_valid,
-                           d->tp_coll_per_layer, true, d->sstar_units, d->grad_accum_steps);
+                           d->tp_coll_per_layer, true, d->sstar_units, d->grad_accum_steps, d->replication_k);
     const u64 comm = objective_comm(r, *f);
     u32 fl;
     const bool survivor = passes(r, *f, Md, &fl);

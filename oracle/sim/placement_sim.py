@@ -183,19 +183,30 @@ def run_single(units, h, xs, ys, theta0, steps):
 
 
 class Placed:
-    """D devices executing one placement (pi_theta, pi_omega, pi_grad, pi_act)."""
+    """D devices executing one placement (pi_theta, pi_omega, pi_grad, pi_act).
 
-    def __init__(self, units, h, b, D, code, theta0, gather_buffers=1):
+    `copies` = k-way replication of the sharded modes: the D devices form k shard
+    groups of G = D / k devices each (k = gcd(copies, D)); device i sits at shard
+    position i mod G of group i div G.  A sharded state is cut into G shards
+    (eq. (2)) and shard p is held by the k devices at position p.  Gathers run
+    inside a shard group; a gradient is reduced to shards by a reduce-scatter
+    inside every shard group followed by an all-reduce of each shard across its
+    k copies.  copies = 1 is plain sharding over all D devices."""
+
+    def __init__(self, units, h, b, D, code, theta0, gather_buffers=1, copies=1):
         self.model = ToyModel(units, h)
         # unit buffers a gathered state holds: 2 when the next unit is fetched while
         # the current one is in use (only possible with at least two units)
         self.nbuf = min(gather_buffers, units)
         self.units, self.h, self.b, self.D = units, h, b, D
+        self.k = int(np.gcd(copies, D))
+        self.G = D // self.k
         self.pT, self.pO, self.pG, self.pA = code % 5, (code // 5) % 5, (code // 25) % 5, code // 125
         self.P = units * h
-        self.cut = bounds(self.P, D)
+        self.cut = bounds(self.P, self.G)          # shard positions
+        self.cutD = bounds(self.P, D)              # chunks of a ring over all D devices
         self.EA = units * b * h
-        self.cutA = bounds(self.EA, D)
+        self.cutA = bounds(self.EA, self.G)
         omega0 = np.stack([theta0.copy(), np.zeros_like(theta0), np.zeros_like(theta0)])
         # persistent homes; None = not held.  "host" is a separate arena.
         self.theta_gpu = [None] * D
@@ -203,7 +214,7 @@ class Placed:
         self.omega_gpu = [None] * D
         self.omega_host = [None] * D
         for i in range(D):
-            lo, hi = self.cut[i], self.cut[i + 1]
+            lo, hi = self.shard(i)
             if self.pT == R: self.theta_gpu[i] = theta0.copy()
             elif self.pT in (S, SG): self.theta_gpu[i] = theta0[lo:hi].copy()
             elif self.pT == O: self.theta_host[i] = theta0[lo:hi].copy()
@@ -211,6 +222,51 @@ class Placed:
             elif self.pO in (S, SG): self.omega_gpu[i] = omega0[:, lo:hi].copy()
             elif self.pO == O: self.omega_host[i] = omega0[:, lo:hi].copy()
         self.update_on_shard = self.pO in (S, SG, O)
+
+    def shard(self, i):
+        p = i % self.G
+        return self.cut[p], self.cut[p + 1]
+
+    def group_gather(self, pieces, width, sent):
+        """All-gather inside every shard group: pieces[i] is device i's piece; returns
+        per device the concatenation of its group's pieces (position order)."""
+        G, out = self.G, [None] * self.D
+        for c in range(self.k):
+            tmp = np.zeros(G, dtype=np.int64)
+            got = ring_all_gather([pieces[c * G + p] for p in range(G)], width, None, None, tmp)
+            for p in range(G):
+                out[c * G + p] = got[p]
+                sent[c * G + p] += tmp[p]
+        return out
+
+    def reduce_to_shards(self, vectors, lo, hi, width, sent_group, sent_rs, sent_ag):
+        """Sum over all D devices of vectors[i][lo:hi], delivered as shards: device i
+        ends with the part of [lo, hi) inside its shard.  A reduce-scatter inside
+        every shard group, then an all-reduce of each shard across its k copies
+        whose pieces follow the eq.-(2) cuts of the whole shard."""
+        G, k, D = self.G, self.k, self.D
+        ucut = [min(max(c, lo), hi) - lo for c in self.cut]
+        part = [None] * D
+        for c in range(k):
+            tmp = np.zeros(G, dtype=np.int64)
+            red = ring_reduce_scatter([vectors[c * G + p][lo:hi] for p in range(G)], ucut, width, None, None, tmp)
+            for p in range(G):
+                part[c * G + p] = red[p]
+                sent_group[c * G + p] += tmp[p]
+        if k > 1:
+            for p in range(G):
+                s_lo, s_hi = self.cut[p], self.cut[p + 1]
+                sub = [s_lo + (q * (s_hi - s_lo)) // k for q in range(k + 1)]      # cuts of the whole shard
+                a0 = min(max(s_lo, lo), hi)                                          # start of this part of it
+                rel = [min(max(x, lo), hi) - a0 for x in sub]
+                t1, t2 = np.zeros(k, dtype=np.int64), np.zeros(k, dtype=np.int64)
+                pieces = ring_reduce_scatter([part[c * G + p] for c in range(k)], rel, width, None, None, t1)
+                full = ring_all_gather(pieces, width, None, None, t2)
+                for c in range(k):
+                    part[c * G + p] = full[c]
+                    sent_rs[c * G + p] += t1[c]
+                    sent_ag[c * G + p] += t2[c]
+        return part
 
     # ---- Theta as seen by forward / backward on every device
     def theta_for_compute(self, books, tag):
@@ -222,7 +278,7 @@ class Placed:
                 out.append(self.theta_gpu[i].copy())
         elif self.pT == S:
             for i in range(D):
-                lo, hi = self.cut[i], self.cut[i + 1]
+                lo, hi = self.shard(i)
                 books.hold("theta", i, (hi - lo) * W_THETA)
                 full = np.zeros(P)
                 full[lo:hi] = self.theta_gpu[i]
@@ -230,7 +286,7 @@ class Placed:
         elif self.pT in (SG, O):
             shards = []
             for i in range(D):
-                lo, hi = self.cut[i], self.cut[i + 1]
+                lo, hi = self.shard(i)
                 if self.pT == SG:
                     books.hold("theta", i, (hi - lo) * W_THETA)
                     shards.append(self.theta_gpu[i])
@@ -244,10 +300,10 @@ class Placed:
                 a, b_ = l * h, (l + 1) * h
                 pieces = []
                 for i in range(D):
-                    lo, hi = self.cut[i], self.cut[i + 1]
+                    lo, hi = self.shard(i)
                     s0, s1 = max(a, lo), min(b_, hi)
                     pieces.append(shards[i][s0 - lo:s1 - lo] if s1 > s0 else np.zeros(0))
-                got = ring_all_gather(pieces, W_THETA, books, None, sent)
+                got = self.group_gather(pieces, W_THETA, sent)
                 if self.pT == SG:
                     books.unit_buffer("theta", self.nbuf * h * W_THETA)
                 for i in range(D):
@@ -261,7 +317,7 @@ class Placed:
                     if self.pO == R:
                         full[:] = self.omega_gpu[i][0]
                     else:
-                        lo, hi = self.cut[i], self.cut[i + 1]
+                        lo, hi = self.shard(i)
                         full[lo:hi] = self.omega_gpu[i][0]
                 books.unit_buffer("theta", h * W_THETA)
                 out.append(full)
@@ -299,18 +355,20 @@ class Placed:
         elif self.pA in (S, SG):
             slices = []
             for i in range(D):
-                lo, hi = self.cutA[i], self.cutA[i + 1]
+                p = i % self.G
+                lo, hi = self.cutA[p], self.cutA[p + 1]
                 books.hold("act", i, hi - lo)
                 slices.append(acts[i].reshape(-1)[lo:hi].copy())
             if self.pA == S:
                 for i in range(D):
+                    p = i % self.G
                     flat = np.zeros(self.EA)
-                    flat[self.cutA[i]:self.cutA[i + 1]] = slices[i]
+                    flat[self.cutA[p]:self.cutA[p + 1]] = slices[i]
                     kept.append(flat.reshape(acts[i].shape))
             else:
-                # gather from the peers: their slices belong to other samples
+                # gather from the peers of the shard group: their slices belong to other samples
                 sent = np.zeros(D, dtype=np.int64)
-                got = ring_all_gather(slices, 1, books, None, sent)
+                got = self.group_gather(slices, 1, sent)
                 books.unit_buffer("act", self.nbuf * b * h)
                 kept = [g.reshape(acts[0].shape) for g in got]
         # (3) Theta again for backward
@@ -324,60 +382,69 @@ class Placed:
         D, P, h, b = self.D, self.P, self.h, self.b
         # (4) synchronise / deliver gradients (mean over the D replicas)
         grad = [np.zeros(P) for _ in range(D)]     # what the update will read
-        cut = self.cut
+        zeros = lambda: np.zeros(D, dtype=np.int64)
         if self.pG == R:
-            red = ring_reduce_scatter(local, cut, W_GRAD, books, "grad reduce-scatter")
+            red = ring_reduce_scatter(local, self.cutD, W_GRAD, books, "grad reduce-scatter")
             full = ring_all_gather(red, W_GRAD, books, "grad all-gather")
             for i in range(D):
                 books.hold("grad", i, P * W_GRAD)
                 grad[i] = full[i] / D
-        elif self.pG in (S, O):
-            red = ring_reduce_scatter(local, cut, W_GRAD, books, "grad reduce-scatter")
-            for i in range(D):
-                n = cut[i + 1] - cut[i]
-                if self.pG == S:
-                    books.hold("grad", i, n * W_GRAD)
-                else:
-                    books.host[i] += 2 * n * W_GRAD              # offload, reload at the update
-                grad[i][cut[i]:cut[i + 1]] = red[i] / D
-        elif self.pG == SG:
-            red = ring_reduce_scatter(local, cut, W_GRAD, books, "grad reduce-scatter")
-            for i in range(D):
-                books.hold("grad", i, (cut[i + 1] - cut[i]) * W_GRAD)
-            sent = np.zeros(D, dtype=np.int64)
-            for l in range(self.units):
-                a, b_ = l * h, (l + 1) * h
-                pieces = []
+        elif self.pG in (S, O, SG):
+            s1, s2, s3 = zeros(), zeros(), zeros()
+            red = self.reduce_to_shards(local, 0, P, W_GRAD, s1, s2, s3)
+            books.phases += [("grad reduce-scatter in the shard group", s1), ("shard reduce-scatter across copies", s2),
+                             ("shard all-gather across copies", s3)]
+            if self.pG in (S, O):
                 for i in range(D):
-                    s0, s1 = max(a, cut[i]), min(b_, cut[i + 1])
-                    pieces.append(red[i][s0 - cut[i]:s1 - cut[i]] if s1 > s0 else np.zeros(0))
-                got = ring_all_gather(pieces, W_GRAD, books, None, sent)
-                books.unit_buffer("grad", self.nbuf * h * W_GRAD)
+                    lo, hi = self.shard(i)
+                    if self.pG == S:
+                        books.hold("grad", i, (hi - lo) * W_GRAD)
+                    else:
+                        books.host[i] += 2 * (hi - lo) * W_GRAD      # offload, reload at the update
+                    grad[i][lo:hi] = red[i] / D
+            else:
                 for i in range(D):
-                    grad[i][a:b_] = got[i] / D
-            books.phases.append(("grad all-gather before use", sent))
+                    lo, hi = self.shard(i)
+                    books.hold("grad", i, (hi - lo) * W_GRAD)
+                sent = zeros()
+                for l in range(self.units):
+                    a, b_ = l * h, (l + 1) * h
+                    pieces = []
+                    for i in range(D):
+                        lo, hi = self.shard(i)
+                        s0, s1_ = max(a, lo), min(b_, hi)
+                        pieces.append(red[i][s0 - lo:s1_ - lo] if s1_ > s0 else np.zeros(0))
+                    got = self.group_gather(pieces, W_GRAD, sent)
+                    books.unit_buffer("grad", self.nbuf * h * W_GRAD)
+                    for i in range(D):
+                        grad[i][a:b_] = got[i] / D
+                books.phases.append(("grad all-gather before use", sent))
         else:  # M: reduced unit by unit as produced, consumed at once
-            sent_rs = np.zeros(D, dtype=np.int64)
-            sent_ag = np.zeros(D, dtype=np.int64)
+            s1, s2, s3, sent_ag = zeros(), zeros(), zeros(), zeros()
             for l in range(self.units):
                 a, b_ = l * h, (l + 1) * h
-                ucut = [min(max(c, a), b_) - a for c in cut]
-                red = ring_reduce_scatter([g[a:b_] for g in local], ucut, W_GRAD, books, None, sent_rs)
                 books.unit_buffer("grad", h * W_GRAD)
                 if self.update_on_shard:
+                    red = self.reduce_to_shards(local, a, b_, W_GRAD, s1, s2, s3)
                     for i in range(D):
-                        grad[i][a + ucut[i]:a + ucut[i + 1]] = red[i] / D
+                        lo, hi = self.shard(i)
+                        s0, s1_ = min(max(lo, a), b_), min(max(hi, a), b_)
+                        grad[i][s0:s1_] = red[i] / D
                 else:
+                    ucut = [min(max(c, a), b_) - a for c in self.cutD]
+                    red = ring_reduce_scatter([g[a:b_] for g in local], ucut, W_GRAD, books, None, s1)
                     got = ring_all_gather(red, W_GRAD, books, None, sent_ag)
                     for i in range(D):
                         grad[i][a:b_] = got[i] / D
-            books.phases.append(("grad reduce per unit", sent_rs))
-            if not self.update_on_shard:
+            books.phases.append(("grad reduce per unit", s1))
+            if self.update_on_shard:
+                books.phases += [("unit shard reduce-scatter across copies", s2), ("unit shard all-gather across copies", s3)]
+            else:
                 books.phases.append(("grad gather per unit", sent_ag))
         # (5) update
         new_theta = [np.zeros(P) for _ in range(D)]   # valid on the committed range
         for i in range(D):
-            lo, hi = cut[i], cut[i + 1]
+            lo, hi = self.shard(i)
             if self.pO == R:
                 books.hold("omega", i, P * W_OMEGA)
                 self.omega_gpu[i] = adam(self.omega_gpu[i], grad[i], t)
@@ -395,27 +462,30 @@ class Placed:
                 new_theta[i] = lost[0]
         if self.pO == SG:
             # gather all of Omega unit by unit, use it, keep only the own shard's update
-            sent = np.zeros(D, dtype=np.int64)
+            sent = zeros()
             for l in range(self.units):
                 a, b_ = l * h, (l + 1) * h
                 pieces = []
                 for i in range(D):
-                    s0, s1 = max(a, cut[i]), min(b_, cut[i + 1])
-                    pieces.append(self.omega_gpu[i][0, s0 - cut[i]:s1 - cut[i]] if s1 > s0 else np.zeros(0))
+                    lo, hi = self.shard(i)
+                    s0, s1_ = max(a, lo), min(b_, hi)
+                    pieces.append(self.omega_gpu[i][0, s0 - lo:s1_ - lo] if s1_ > s0 else np.zeros(0))
                 for _row in range(3):          # master, m, v: 3 x 4 bytes per element
-                    ring_all_gather(pieces, W_OMEGA // 3, books, None, sent)
+                    self.group_gather(pieces, W_OMEGA // 3, sent)
                 books.unit_buffer("omega", self.nbuf * h * W_OMEGA)
             books.phases.append(("gather omega", sent))
             for i in range(D):
-                lo, hi = cut[i], cut[i + 1]
+                lo, hi = self.shard(i)
                 books.hold("omega", i, (hi - lo) * W_OMEGA)
                 self.omega_gpu[i] = adam(self.omega_gpu[i], grad[i][lo:hi], t)
                 new_theta[i][lo:hi] = self.omega_gpu[i][0]
         # (6) Theta back to its home
         if self.pT == R:
             if self.update_on_shard:
-                pieces = [new_theta[i][cut[i]:cut[i + 1]] for i in range(D)]
-                got = ring_all_gather(pieces, W_THETA, books, "re-replicate theta")
+                pieces = [new_theta[i][slice(*self.shard(i))] for i in range(D)]
+                sent = zeros()
+                got = self.group_gather(pieces, W_THETA, sent)
+                books.phases.append(("re-replicate theta", sent))
                 for i in range(D):
                     self.theta_gpu[i] = got[i]
             else:
@@ -423,43 +493,46 @@ class Placed:
                     self.theta_gpu[i] = new_theta[i].copy()
         elif self.pT in (S, SG):
             for i in range(D):
-                self.theta_gpu[i] = new_theta[i][cut[i]:cut[i + 1]].copy()
+                self.theta_gpu[i] = new_theta[i][slice(*self.shard(i))].copy()
         elif self.pT == O:
             for i in range(D):
-                books.host[i] += (cut[i + 1] - cut[i]) * W_THETA   # device -> host
-                self.theta_host[i] = new_theta[i][cut[i]:cut[i + 1]].copy()
+                lo, hi = self.shard(i)
+                books.host[i] += (hi - lo) * W_THETA   # device -> host
+                self.theta_host[i] = new_theta[i][lo:hi].copy()
 
     # ---- what the job as a whole holds after a step
     def reassemble(self):
-        """Returns (list of Theta views, list of Omega views): one per holder; a
-        placement is consistent only if every view equals the single-device
-        state.  An empty list means the state is held nowhere."""
-        D = self.D
+        """Returns (list of Theta views, list of Omega views): one per holder (one per
+        shard group for a sharded state); a placement is consistent only if every
+        view equals the single-device state.  An empty list means the state is
+        held nowhere."""
+        D, G, k = self.D, self.G, self.k
+        groups = [range(c * G, (c + 1) * G) for c in range(k)]
         if self.pO == R:
             omegas = [self.omega_gpu[i] for i in range(D)]
         elif self.pO in (S, SG):
-            omegas = [np.concatenate([self.omega_gpu[i] for i in range(D)], axis=1)]
+            omegas = [np.concatenate([self.omega_gpu[i] for i in g], axis=1) for g in groups]
         elif self.pO == O:
-            omegas = [np.concatenate([self.omega_host[i] for i in range(D)], axis=1)]
+            omegas = [np.concatenate([self.omega_host[i] for i in g], axis=1) for g in groups]
         else:
             omegas = []
         if self.pT == R:
             thetas = [self.theta_gpu[i] for i in range(D)]
         elif self.pT in (S, SG):
-            thetas = [np.concatenate([self.theta_gpu[i] for i in range(D)])]
+            thetas = [np.concatenate([self.theta_gpu[i] for i in g]) for g in groups]
         elif self.pT == O:
-            thetas = [np.concatenate([self.theta_host[i] for i in range(D)])]
+            thetas = [np.concatenate([self.theta_host[i] for i in g]) for g in groups]
         else:
             thetas = [om[0] for om in omegas]   # Theta exists only as the master copy
         return thetas, omegas
 
 
-def simulate_problem(units, h, b, D, code, theta0, xs, ys, steps=3, gather_buffers=1):
+def simulate_problem(units, h, b, D, code, theta0, xs, ys, steps=3, gather_buffers=1, copies=1):
     """As simulate(), on a given problem (theta0[P]; xs[j][i], ys[j][i] = micro-batch j of
     device i); also returns the parameters the job holds after the last step (first
     holder's view, None if they are held nowhere)."""
     ref = run_single(units, h, xs, ys, theta0, steps)
-    job = Placed(units, h, b, D, code, theta0, gather_buffers)
+    job = Placed(units, h, b, D, code, theta0, gather_buffers, copies)
     match = True
     books = None
     thetas = []
@@ -480,7 +553,7 @@ def simulate_problem(units, h, b, D, code, theta0, xs, ys, steps=3, gather_buffe
                 theta=thetas[0] if thetas else None, ref_theta=ref[-1][0])
 
 
-def simulate(units, h, b, D, code, steps=3, seed=0, accum=1, gather_buffers=1):
+def simulate(units, h, b, D, code, steps=3, seed=0, accum=1, gather_buffers=1, copies=1):
     """Run `steps` steps of `accum` micro-batches each; returns dict(match, mem,
     comm, host) where match says whether every step's reassembled Theta and Omega
     equal the single-device run to 1e-12 relative, and the byte figures are those
@@ -488,7 +561,7 @@ def simulate(units, h, b, D, code, steps=3, seed=0, accum=1, gather_buffers=1):
     unit while the current one is in use."""
     theta0, xs, ys = make_problem(units, h, b, D, seed, accum)
     ref = run_single(units, h, xs, ys, theta0, steps)
-    job = Placed(units, h, b, D, code, theta0, gather_buffers)
+    job = Placed(units, h, b, D, code, theta0, gather_buffers, copies)
     match = True
     books = None
     for t in range(1, steps + 1):

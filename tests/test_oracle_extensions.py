@@ -137,3 +137,69 @@ def test_simulator_with_micro_batches_and_prefetch(D):
             assert s["comm"] == r["comm_paper"] + r["comm_ext"], (code, D)
             assert s["host"] == r["host"], (code, D)
     assert n_valid == 171
+
+
+# ------------------------------------------------------------ k-way replication
+# Section 1 names "k-way replication for 1 < k < N" as a straightforward extension of
+# the replicated / sharded pair.  Reading: the sharded modes cut a state into D / k
+# shards and every shard is held by k devices; gathers stay inside a group of D / k
+# devices, a gradient is reduced to shards inside each group and then all-reduced
+# across the k copies of each shard.
+def test_k_way_replication_interpolates_between_sharded_and_replicated():
+    space = synth.config("C1", n_models=2)
+    n_values = space["n_values"].tolist()
+    plain = O.Space(space).eval_range(0, 625 * 2 * len(n_values))
+    for k in (2, 8, 1 << 10):
+        repl = O.Space(dict(space, replication_k=k)).eval_range(0, 625 * 2 * len(n_values))
+        for ni, N in enumerate(n_values):
+            base = ni * 2 * 625
+            if N == 1:
+                # one device: nothing to replicate
+                for name in plain:
+                    assert np.array_equal(plain[name][base:base + 1250], repl[name][base:base + 1250])
+            if k >= N:
+                # as many copies as devices: a "shard" is the whole tensor, so S costs what R costs
+                # (all three states sharded vs replicated: ZeRO-2-like code 30 + Theta S vs DP, code 0)
+                s_all = base + 1 + 5 + 25          # (S, S, S, R)
+                assert repl["mem"][s_all] == repl["mem"][base]
+                assert repl["comm_paper"][s_all] == repl["comm_paper"][base]
+                assert repl["flags"][s_all] & O.F_GI       # every device has all of Theta
+    # k = 1 is the plain space
+    same = O.Space(dict(space, replication_k=1)).eval_range(0, 1250)
+    for name in plain:
+        assert np.array_equal(plain[name][:1250], same[name])
+
+
+def test_k_way_replication_on_the_worked_example():
+    """70B parameters, N = 8, two copies of every shard (four shards): ZeRO-3 holds
+    16P/4 = 280 GB; its gradients cost a reduce-scatter over 4 devices, (3/4) 2P, plus
+    an all-reduce of the 2P/4 shard over 2 copies, 2 (1/2) 2P/4; its parameters two
+    gathers over 4 devices, 2 (3/4) 2P."""
+    space = dict(synth.config("C0"), replication_k=2)
+    res = O.Space(space).eval_range(0, 4375)
+    P = 70_000_000_000
+    z3 = 3 * 625 + 32                                      # N = 8
+    assert int(res["mem"][z3]) == 16 * P // 4
+    assert int(res["comm_paper"][z3]) == (3 * 2 * P // 4 + 2 * (2 * P // 4) // 2) + 2 * (3 * 2 * P // 4)
+    # data parallelism does not shard anything: unchanged
+    assert int(res["mem"][3 * 625]) == 16 * P and int(res["comm_paper"][3 * 625]) == 245_000_000_000
+    # N = 2 with two copies: ZeRO-3 is data parallelism in all but name
+    z3_2 = 1 * 625 + 32
+    assert int(res["mem"][z3_2]) == 16 * P and int(res["comm_paper"][z3_2]) == 2 * (2 * P // 2)
+
+
+@pytest.mark.parametrize("D,k", [(4, 2), (6, 3), (3, 3), (4, 3)])
+def test_k_way_replication_against_the_simulator(D, k):
+    """All 625 placements with every shard held k times (gcd(k, D) times where k does not
+    divide D): valid exactly when the run reproduces the single-device trajectory, and
+    then the bytes held, sent and moved over the host link are the simulator's."""
+    units, h, b = 3, 5, 2
+    rec = dict(P=units * h, unit=h, A0=units * b * h, A1=units * b * h, UA0=b * h, UA1=b * h, Sbh=b * h,
+               L=units, heads=1, w_theta=sim.W_THETA, w_omega=sim.W_OMEGA, w_grad=sim.W_GRAD, w_act=2)
+    for code in range(625):
+        r = O.eval_record(rec, D, 1, 1, D, 0, 0, code, replication_k=k)
+        valid = (r["flags"] & (O.F_GI | O.F_SC)) == (O.F_GI | O.F_SC)
+        s = sim.simulate(units, h, b, D, code, steps=3, seed=code % 5, copies=k)
+        assert valid == s["match"], (code, D, k)
+        if valid:
+            assert (s["mem"], s["comm"], s["host"]) == (r["mem"], r["comm_paper"] + r["comm_ext"], r["host"]), code
