@@ -133,7 +133,7 @@ typedef struct {
                                    2: {S, R}                                            */
   uint32_t mode_mask;           /* bit m set: mode m allowed on the data axis; != 0    */
   uint32_t tp_coll_per_layer;   /* all-reduces per layer per step on the tensor axis, <= 64 */
-  /* Two extensions the paper names without working them out.  Both apply to
+  /* Three extensions the paper names without working them out.  Each applies to
    * the whole space (sweep once per value to compare values); 0 means 1. */
   uint32_t sstar_units;         /* 1 or 2: unit buffers a gathered (S*) state holds.  Theorem 1
                                    charges one; its proof notes that an implementation which
@@ -152,6 +152,17 @@ typedef struct {
                                    per step for g times the samples: the paper's "reduced by a
                                    factor equal to the number of accumulation steps".  Memory
                                    and the predicates do not change. */
+  uint32_t replication_k;       /* 1 .. 2^24: copies of every shard ("k-way replication for
+                                   1 < k < N", Section 1).  The sharded modes S, S*, O of a data
+                                   axis of D devices cut a state into G = D / k shards, each held
+                                   by the k devices at the same position of k groups of G devices
+                                   (k = gcd(replication_k, D) where it does not divide D).  A shard
+                                   is ceil(E / G) elements; gathers run inside a group and move
+                                   E - floor(E / G); a gradient is reduced to shards inside every
+                                   group and then all-reduced across the copies of each shard.  With
+                                   G = 1 a shard is the whole tensor and the predicates treat the
+                                   sharded modes as they do on a single device.  Modes R and M and
+                                   the model axes are not affected. */
 } ps_space_desc;
 
 /* survivors of a filter: mem <= cap_bytes, host <= host_cap and every bit of
@@ -161,6 +172,13 @@ typedef struct {
   uint32_t require_flags;
   uint32_t comm_kind;     /* objective of the sweeps: PS_COMM_PAPER or ..._PLUS_EXT */
   uint64_t cap_bytes;     /* ps_eval_batch only; the sweeps take their own list     */
+  uint32_t skip_rejected; /* sweeps only.  0: every point is evaluated (its capacity compare is
+                             executed, then masked by the flags) -- what the throughput figures
+                             are quoted on.  1: a factorisation whose composition bits (T | heads,
+                             K | layers, T <= tp_max_valid) already miss a required flag is not
+                             evaluated at all; same results, less work when the filter requires
+                             PS_F_CV or one of its reasons */
+  uint32_t pad;
 } ps_filter;
 
 /* structure-of-arrays outputs of ps_eval_batch: device pointers, any may be

@@ -210,7 +210,7 @@ int ps_space_create(ps_ctx* ctx, const ps_space_desc* desc, ps_space** out) {
   if (desc->tp_coll_per_layer > 64) return PS_E_RANGE;
   for (u32 i = 0; i < desc->n_n; ++i)
     if (desc->n_values[i] < 1 || desc->n_values[i] > (1u << 24)) return PS_E_RANGE;
-  if (desc->sstar_units > 2 || desc->grad_accum_steps > 64) return PS_E_RANGE;
+  if (desc->sstar_units > 2 || desc->grad_accum_steps > 64 || desc->replication_k > (1u << 24)) return PS_E_RANGE;
   const u32 accum = desc->grad_accum_steps ? desc->grad_accum_steps : 1;
   for (u32 i = 0; i < desc->n_models; ++i)
     if (!shape_in_range(desc->models[i], desc->tp_coll_per_layer, accum)) return PS_E_RANGE;
@@ -265,6 +265,7 @@ int ps_space_create(ps_ctx* ctx, const ps_space_desc* desc, ps_space** out) {
   d.tp_coll = desc->tp_coll_per_layer;
   d.sstar_units = desc->sstar_units ? desc->sstar_units : 1;
   d.accum = accum;
+  d.repl = desc->replication_k ? desc->replication_k : 1;
   d.all_pow2 = 1;
   for (u32 i = 0; i < desc->n_n; ++i)
     if (desc->n_values[i] & (desc->n_values[i] - 1)) d.all_pow2 = 0;
@@ -441,6 +442,7 @@ int ps_sweep_pareto(ps_ctx* ctx, const ps_space* sp, const ps_filter* filter,
   s.require_flags = filter->require_flags & ~(u32)PS_F_FEASIBLE;
   s.comm_kind = filter->comm_kind;
   s.k_keep = reduce_kind == PS_REDUCE_TOPK ? max_entries : 0;
+  s.skip_rejected = filter->skip_rejected ? 1u : 0u;
   s.partial = static_cast<PartialEntry*>(ctx->scratch);
   s.partial_n = reinterpret_cast<uint2*>(static_cast<char*>(ctx->scratch) + partial_bytes);
   s.status = ctx->d_status;

@@ -45,6 +45,7 @@ struct SpaceDev {
   u32 tp_max_valid, tp_coll;
   u32 sstar_units;    // unit buffers a gathered (S*) state holds at a time: 1, or 2 when gathers overlap computation
   u32 accum;          // micro-batches per step (gradient accumulation), >= 1
+  u32 repl;           // copies of every shard (k-way replication of the sharded modes), >= 1
   u32 all_pow2;       // 1 if every device count of the space is a power of two (then every T, K, D is)
   u32 all_small;      // 1 if for every model (4 accum + 1) (w_T + w_O + w_G) (P + 2 unit) < 2^53: the device
                       // bytes, host bytes and data-axis volume of a (Theta, Omega, G) triple are then
@@ -85,26 +86,54 @@ __device__ __forceinline__ u64 div_ceil(u64 a, u32 d) { return div_floor(a + (d 
 // Quantities that depend on (model, T, K, D) only.  Remark 4: the tensor split
 // is innermost, the pipeline split next, the data axis outermost.  Both model
 // axes shard Theta, Omega and G (Table 2).
+// k-way replication: the D devices of the data axis form k = gcd(repl, D) shard
+// groups of G = D / k devices; a sharded state is cut into G shards, each held by
+// the k devices at the same position of their groups.  Gathers run inside a
+// group; a gradient is reduced to shards by a reduce-scatter inside every group
+// and an all-reduce of each shard across its copies.
+enum : u32 {
+  CLS_SHARDED = 0,    // several shard positions (G > 1)
+  CLS_ONE_DEVICE = 1, // D = 1: nothing moves, a shard is the tensor
+  CLS_ALL_COPIES = 2  // G = 1 < D: a "shard" is the tensor, held by every device
+};
 struct UnitBase {
   u64 E2;     // elements of Theta (= Omega = G) left on one (t, k) position
-  u64 sh;     // largest data-axis shard of them, ceil(E2 / D)   (eq. (2))
-  u64 x;      // ring volume over the data axis, E2 - floor(E2 / D)  (Section 2.3)
+  u64 sh;     // largest data-axis shard of them, ceil(E2 / G)   (eq. (2))
+  u64 x;      // ring volume inside a shard group, E2 - floor(E2 / G)  (Section 2.3)
+  u64 x2;     // all-reduce of the largest shard across its k copies, 2 (sh - floor(sh / k)); 0 if k = 1
+  u64 x3;     // what an all-reduce over all D devices moves beyond 2 x; 0 if k = 1
+  u32 G;      // shard positions
+  u32 cls;    // CLS_*
   u64 u;      // reconstruction unit after the tensor split
   u64 tp_x;   // ring volume of a boundary tensor over the tensor axis
   u64 sbh_t;  // ceil(Sbh / T)
   u32 lps;    // layers per pipeline stage, ceil(L / K)
   u32 cv;     // PS_F_CV and its reason bits (axis form assumed)
-  bool d1;    // D == 1
+  bool d1;    // one shard position (G == 1): a shard is the whole tensor
 };
 
+__device__ __forceinline__ u32 gcd_u32(u32 a, u32 b) {
+  while (b) { const u32 t = a % b; a = b; b = t; }
+  return a;
+}
+
 __device__ __forceinline__ UnitBase unit_base(const ModelRec& r, const Fact& f, u32 tp_max_valid,
-                                              bool axis_form) {
+                                              bool axis_form, u32 repl = 1) {
   UnitBase b;
   u64 E1 = div_ceil(r.P, f.T);
   b.E2 = div_ceil(E1, f.K);
-  u64 q = div_floor(b.E2, f.D);
-  b.sh = q + ((q * f.D != b.E2) ? 1 : 0);
+  const u32 k = repl > 1 ? gcd_u32(repl, f.D) : 1u;
+  b.G = f.D / k;
+  u64 q = div_floor(b.E2, b.G);
+  b.sh = q + ((q * b.G != b.E2) ? 1 : 0);
   b.x = b.E2 - q;
+  b.x2 = 0;
+  b.x3 = 0;
+  if (k > 1) {
+    b.x2 = 2 * (b.sh - div_floor(b.sh, k));
+    b.x3 = 2 * ((b.E2 - div_floor(b.E2, f.D)) - b.x);
+  }
+  b.cls = f.D == 1 ? CLS_ONE_DEVICE : (b.G == 1 ? CLS_ALL_COPIES : CLS_SHARDED);
   b.u = div_ceil(r.unit, f.T);
   u64 qs = div_floor(r.Sbh, f.T);
   b.tp_x = r.Sbh - qs;
@@ -120,7 +149,7 @@ __device__ __forceinline__ UnitBase unit_base(const ModelRec& r, const Fact& f, 
            (tp_le ? PS_F_TP_LE_MAX : 0) | (axis_form ? PS_F_AXIS_FORM : 0);
   if (t_heads && k_layers && tp_le && axis_form && whole) cv |= PS_F_CV;
   b.cv = cv;
-  b.d1 = (f.D == 1);
+  b.d1 = (b.G == 1);
   return b;
 }
 
@@ -128,14 +157,24 @@ __device__ __forceinline__ UnitBase unit_base(const ModelRec& r, const Fact& f, 
 // divisions become shifts.  Same values as unit_base / act_base.
 struct Pow2 {
   u32 sT, sK, sD;
+  u32 sC;     // log2 of the copies of a shard: gcd(repl, D) = the lowest set bit of repl, at most D
+  u32 sG;     // log2 of the shard positions, sD - sC
   bool all;
 };
-__device__ __forceinline__ Pow2 pow2_of(const Fact& f) {
+__device__ __forceinline__ Pow2 pow2_of(const Fact& f) {          // one copy of every shard
   Pow2 p;
   p.all = (((f.T & (f.T - 1)) | (f.K & (f.K - 1)) | (f.D & (f.D - 1))) == 0);
   p.sT = 31 - __clz(f.T);
   p.sK = 31 - __clz(f.K);
   p.sD = 31 - __clz(f.D);
+  p.sC = 0;
+  p.sG = p.sD;
+  return p;
+}
+__device__ __forceinline__ Pow2 pow2_of(const Fact& f, u32 repl) {
+  Pow2 p = pow2_of(f);
+  p.sC = min((u32)(__ffs(repl) - 1), p.sD);      // repl >= 1
+  p.sG = p.sD - p.sC;
   return p;
 }
 __device__ __forceinline__ u64 ceil_shift(u64 a, u32 s) { return (a + (((u64)1 << s) - 1)) >> s; }
@@ -144,8 +183,39 @@ __device__ __forceinline__ UnitBase unit_base_pow2(const ModelRec& r, const Fact
                                                    u32 tp_max_valid, bool axis_form) {
   UnitBase b;
   b.E2 = ceil_shift(ceil_shift(r.P, p.sT), p.sK);
+  b.G = 1u << p.sG;
+  b.sh = ceil_shift(b.E2, p.sG);
+  b.x = b.E2 - (b.E2 >> p.sG);
+  b.x2 = 2 * (b.sh - (b.sh >> p.sC));             // 0 when there is one copy
+  b.x3 = 2 * ((b.E2 - (b.E2 >> p.sD)) - b.x);
+  b.cls = f.D == 1 ? CLS_ONE_DEVICE : (p.sG == 0 ? CLS_ALL_COPIES : CLS_SHARDED);
+  b.u = ceil_shift(r.unit, p.sT);
+  b.tp_x = r.Sbh - (r.Sbh >> p.sT);
+  b.sbh_t = ceil_shift(r.Sbh, p.sT);
+  b.lps = (r.L + (f.K - 1)) >> p.sK;
+  const bool k_layers = (r.L & (f.K - 1)) == 0;
+  const bool t_heads = (r.heads & (f.T - 1)) == 0;
+  const bool tp_le = f.T <= tp_max_valid;
+  const bool whole = ((u64)f.T * f.K * f.D == (u64)f.N);
+  u32 cv = (t_heads ? PS_F_T_DIV_HEADS : 0) | (k_layers ? PS_F_K_DIV_LAYERS : 0) |
+           (tp_le ? PS_F_TP_LE_MAX : 0) | (axis_form ? PS_F_AXIS_FORM : 0);
+  if (t_heads && k_layers && tp_le && axis_form && whole) cv |= PS_F_CV;
+  b.cv = cv;
+  b.d1 = (p.sG == 0);
+  return b;
+}
+
+// the same with one copy of every shard (the shard positions are the D devices)
+__device__ __forceinline__ UnitBase unit_base_pow2_one_copy(const ModelRec& r, const Fact& f, const Pow2& p,
+                                                   u32 tp_max_valid, bool axis_form) {
+  UnitBase b;
+  b.E2 = ceil_shift(ceil_shift(r.P, p.sT), p.sK);
+  b.G = f.D;
   b.sh = ceil_shift(b.E2, p.sD);
   b.x = b.E2 - (b.E2 >> p.sD);
+  b.x2 = 0;
+  b.x3 = 0;
+  b.cls = f.D == 1 ? CLS_ONE_DEVICE : CLS_SHARDED;
   b.u = ceil_shift(r.unit, p.sT);
   b.tp_x = r.Sbh - (r.Sbh >> p.sT);
   b.sbh_t = ceil_shift(r.Sbh, p.sT);
@@ -168,15 +238,23 @@ __device__ __forceinline__ UnitBase unit_base_pow2(const ModelRec& r, const Fact
 struct ActBase {
   u64 EA, shA, uA;
 };
-__device__ __forceinline__ ActBase act_base(const ModelRec& r, const Fact& f, u32 v, u32 tau) {
+__device__ __forceinline__ ActBase act_base(const ModelRec& r, const Fact& f, u32 v, u32 tau, u32 G) {
   ActBase a;
   a.EA = tau == 0 ? div_ceil(r.A[v], f.T) : r.A[v];
   a.uA = tau == 0 ? div_ceil(r.UA[v], f.T) : r.UA[v];
-  a.shA = div_ceil(a.EA, f.D);
+  a.shA = div_ceil(a.EA, G);                      // G = shard positions of the data axis
   return a;
 }
 
 __device__ __forceinline__ ActBase act_base_pow2(const ModelRec& r, const Pow2& p, u32 v, u32 tau) {
+  ActBase a;
+  const u32 s = tau == 0 ? p.sT : 0;
+  a.EA = ceil_shift(r.A[v], s);
+  a.uA = ceil_shift(r.UA[v], s);
+  a.shA = ceil_shift(a.EA, p.sG);
+  return a;
+}
+__device__ __forceinline__ ActBase act_base_pow2_one_copy(const ModelRec& r, const Pow2& p, u32 v, u32 tau) {
   ActBase a;
   const u32 s = tau == 0 ? p.sT : 0;
   a.EA = ceil_shift(r.A[v], s);
@@ -251,23 +329,26 @@ __device__ __forceinline__ u32 point_flags(u32 th, u32 om, u32 gr, u32 ac, bool 
 __device__ __forceinline__ PointOut eval_point(const ModelRec& r, const Fact& f, u32 v, u32 tau,
                                                u32 th, u32 om, u32 gr, u32 ac, u32 tp_max_valid,
                                                u32 tp_coll, bool axis_form, u32 sstar_units = 1,
-                                               u32 accum = 1) {
-  UnitBase b = unit_base(r, f, tp_max_valid, axis_form);
-  ActBase a = act_base(r, f, v, tau);
+                                               u32 accum = 1, u32 repl = 1) {
+  UnitBase b = unit_base(r, f, tp_max_valid, axis_form, repl);
+  ActBase a = act_base(r, f, v, tau, b.G);
   PointOut o;
   o.mem = r.wT * mu_elems(th, b.E2, b.sh, b.u, sstar_units) + r.wO * mu_elems(om, b.E2, b.sh, b.u, sstar_units) +
           r.wG * mu_elems(gr, b.E2, b.sh, b.u, sstar_units) + mu_elems(ac, a.EA, a.shA, a.uA, sstar_units);
   u64 xT = b.x * r.wT, xO = b.x * r.wO, xG = b.x * r.wG;
+  // a gradient reduced to shards (inside the group, then across the copies of a shard), and
+  // all-reduced over all devices; with one copy of every shard these are xG and 2 xG
+  const u64 to_shards = xG + b.x2 * r.wG, all_reduce = 2 * xG + b.x3 * r.wG;
   // Theorem 2
-  o.comm_paper = (gr == PS_MODE_R ? 2 * xG : 0) + (gr == PS_MODE_S ? xG : 0) +
+  o.comm_paper = (gr == PS_MODE_R ? all_reduce : 0) + (gr == PS_MODE_S ? to_shards : 0) +
                  (th == PS_MODE_SG ? 2 * xT * accum : 0);
   bool on_shard = in_set(SET_UPDATE_ON_SHARD, om);
   u64 ext = 0;
   if (th == PS_MODE_O) ext += 2 * xT * accum;
   if (th == PS_MODE_R && on_shard) ext += xT;
-  if (gr == PS_MODE_SG) ext += 2 * xG;
-  if (gr == PS_MODE_M) ext += on_shard ? xG : 2 * xG;
-  if (gr == PS_MODE_O) ext += xG;
+  if (gr == PS_MODE_SG) ext += to_shards + xG;
+  if (gr == PS_MODE_M) ext += on_shard ? to_shards : all_reduce;
+  if (gr == PS_MODE_O) ext += to_shards;
   if (om == PS_MODE_SG) ext += xO;
   o.comm_ext = ext + model_axis_traffic(r, f, b, tau, tp_coll, accum);
   o.host = (th == PS_MODE_O ? (2 * accum + 1) * b.sh * r.wT : 0) + (om == PS_MODE_O ? 2 * b.sh * r.wO : 0) +
@@ -283,16 +364,23 @@ enum : u32 {
   T_M_OR_O = 1u << 4, T_EXT0 = 1u << 5
 };
 
-__device__ __forceinline__ u32 triple_bits(u32 th, u32 om, u32 gr, bool d1) {
+// cls: CLS_* of the factorisation (a shard is the whole tensor unless CLS_SHARDED)
+__device__ __forceinline__ u32 triple_bits(u32 th, u32 om, u32 gr, u32 cls) {
+  const bool d1 = cls != CLS_SHARDED;
   const bool on_shard = in_set(SET_UPDATE_ON_SHARD, om);
   const bool omega_full = (om == PS_MODE_R) || (d1 && in_set(SET_SHARDLIKE, om));
   const bool theta_avail = in_set(SET_THETA_ALWAYS, th) || (th == PS_MODE_S && d1) ||
                            (th == PS_MODE_M && omega_full);
   const bool grad_cover = d1 || on_shard || in_set(SET_GRAD_FULL, gr);
   const u32 seen = (1u << th) | (1u << om) | (1u << gr);
-  // data-axis traffic beyond Theorem 2: none with a single replica (nothing moves)
-  const bool ext0 = d1 || !((th == PS_MODE_O) || (th == PS_MODE_R && on_shard) ||
-                            in_set((1u << PS_MODE_SG) | SET_M_OR_O, gr) || om == PS_MODE_SG);
+  // data-axis traffic beyond Theorem 2: none with a single device (nothing moves); with
+  // every device holding every "shard" the gathers move nothing, the gradient modes that
+  // Theorem 2 does not price still do
+  const bool grad_unpriced = in_set((1u << PS_MODE_SG) | SET_M_OR_O, gr);
+  const bool ext0 = cls == CLS_ONE_DEVICE ||
+                    (cls == CLS_ALL_COPIES ? !grad_unpriced
+                                           : !((th == PS_MODE_O) || (th == PS_MODE_R && on_shard) ||
+                                               grad_unpriced || om == PS_MODE_SG));
   return (theta_avail ? T_THETA_AVAIL : 0) | (grad_cover ? T_GRAD_COVER : 0) |
          (om != PS_MODE_M ? T_SC : 0) | ((seen >> PS_MODE_O) & 1u ? T_HOST : 0) |
          ((seen & SET_M_OR_O) ? T_M_OR_O : 0) | (ext0 ? T_EXT0 : 0);

@@ -65,7 +65,8 @@ __device__ __forceinline__ u64 mad_small(u64 a, u32 k, u64 acc) {
   return r;
 }
 
-// static description of a triple for D > 1 (d1 = false) or D = 1
+// static description of a triple when the data axis has several shard positions (d1 = false)
+// or a single device (d1 = true)
 __device__ __forceinline__ u32 triple_static(u32 th, u32 om, u32 gr, bool d1) {
   const bool on_shard = in_set(SET_UPDATE_ON_SHARD, om);
   const bool omega_full = (om == PS_MODE_R) || (d1 && in_set(SET_SHARDLIKE, om));
@@ -80,6 +81,14 @@ __device__ __forceinline__ u32 triple_static(u32 th, u32 om, u32 gr, bool d1) {
   return (theta_avail ? PS_F_THETA_AVAIL : 0) | (grad_cover ? PS_F_GRAD_COVER : 0) |
          (om != PS_MODE_M ? PS_F_SC : 0) | (((seen >> PS_MODE_O) & 1u) ? X_HOST3 : 0) |
          ((seen & SET_M_OR_O) ? X_MO3 : 0) | (ext0 ? X_EXT0 : 0);
+}
+
+// the same for a factorisation whose shards are all held by every device (several copies,
+// one shard position): a shard is the whole tensor as on a single device, the gathers move
+// nothing, but the gradient modes Theorem 2 does not price still move data
+__device__ __forceinline__ u32 triple_static_all_copies(u32 th, u32 om, u32 gr) {
+  const u32 st = triple_static(th, om, gr, true) & ~X_EXT0;
+  return st | (in_set((1u << PS_MODE_SG) | SET_M_OR_O, gr) ? 0u : X_EXT0);
 }
 
 enum { MODE_MATERIALISE = 0, MODE_WRITE = 2 };
@@ -180,7 +189,8 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
   u32 model_cur = 0xffffffffu;
   ModelRec rec;
   u32 ka[R], kb[R], kc[R], kp[R], ke[R], kh[R];   // bytes (E, s, u), priced / unpriced comm (x), host (s)
-  u32 st_many[R], st_one[R];                      // static description for D > 1 and D = 1
+  u32 st_many[R], st_one[R];                      // static description of a triple by the class of the factorisation
+  u32 st_copies[POW2 ? 1 : R];                    // (the third class needs several copies of a shard)
 
   for (u32 it = it_begin; it < it_end; it += it_step) {
     const u32 seg = MODE == MODE_WRITE ? a.nonempty[it] : it;
@@ -226,15 +236,19 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
                 (gr[r] == PS_MODE_O ? 2 * rec.wG : 0);
         st_many[r] = triple_static(th[r], om[r], gr[r], false);
         st_one[r] = triple_static(th[r], om[r], gr[r], true);
+        if (!POW2) st_copies[r] = triple_static_all_copies(th[r], om[r], gr[r]);
       }
     }
 
     // ---- per group: shard quantities (all divisions), activation bytes per digit
     const Fact f = sp.facts[unit];
-    const Pow2 p2 = pow2_of(f);
-    const UnitBase ub = (POW2 || p2.all) ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
-                               : unit_base(rec, f, sp.tp_max_valid, true);
-    const ActBase ab = (POW2 || p2.all) ? act_base_pow2(rec, p2, v, tau) : act_base(rec, f, v, tau);
+    const u32 repl = POW2 ? 1u : sp.repl;        // the power-of-two case is compiled for one copy of every shard
+    const Pow2 p2 = POW2 ? pow2_of(f) : pow2_of(f, repl);
+    const UnitBase ub = POW2 ? unit_base_pow2_one_copy(rec, f, p2, sp.tp_max_valid, true)
+                        : p2.all ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
+                                 : unit_base(rec, f, sp.tp_max_valid, true, repl);
+    const ActBase ab = POW2 ? act_base_pow2_one_copy(rec, p2, v, tau)
+                       : p2.all ? act_base_pow2(rec, p2, v, tau) : act_base(rec, f, v, tau, ub.G);
     const u64 c_axis = model_axis_traffic(rec, f, ub, tau, sp.tp_coll, sp.accum);
     u64 act[NM];
 #pragma unroll
@@ -249,8 +263,18 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
       mem3[r] = mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0)));
       paper3[r] = mad_small(ub.x, kp[r], 0);
       ext3[r] = mad_small(ub.x, ke[r], 0);
+      if (repl > 1) {
+        // several copies of every shard: reducing gradients to shards costs x2 more, an
+        // all-reduce over all devices x3 more (both zero with one copy)
+        const bool on_shard = in_set(SET_UPDATE_ON_SHARD, om[r]);
+        paper3[r] += (u64)rec.wG * ((gr[r] == PS_MODE_S ? ub.x2 : 0) + (gr[r] == PS_MODE_R ? ub.x3 : 0));
+        ext3[r] += (u64)rec.wG * (((gr[r] == PS_MODE_SG || gr[r] == PS_MODE_O || (gr[r] == PS_MODE_M && on_shard)) ? ub.x2 : 0) +
+                                  ((gr[r] == PS_MODE_M && !on_shard) ? ub.x3 : 0));
+      }
       host3[r] = mad_small(ub.sh, kh[r], 0);
-      st[r] = ub.d1 ? st_one[r] : st_many[r];
+      // (with one copy of every shard a factorisation is sharded or a single device)
+      if (POW2) st[r] = ub.d1 ? st_one[r] : st_many[r];
+      else st[r] = ub.cls == CLS_SHARDED ? st_many[r] : (ub.cls == CLS_ONE_DEVICE ? st_one[r] : st_copies[POW2 ? 0 : r]);
     }
 
     // ---- the group's points inside the window
@@ -415,7 +439,7 @@ __global__ void __launch_bounds__(THREADS, 2) k_compact_count(SpaceDev sp, EvalA
     if (!in_set(SET_M_OR_O, ac)) not_mo |= 1u << d;
   }
   // the lane's triples: modes and the activation digits the required flags allow
-  // (bits 0..4 with several replicas, bits 8..12 with one), fixed for the kernel
+  // (bits 0..4, 8..12, 16..20 for the three classes of a factorisation), fixed for the kernel
   u32 th[R], om[R], gr[R], t_allowed[R];
 #pragma unroll
   for (int r = 0; r < R; ++r) {
@@ -425,9 +449,10 @@ __global__ void __launch_bounds__(THREADS, 2) k_compact_count(SpaceDev sp, EvalA
     th[r] = digit_mode(modemap, tt % NM);
     om[r] = digit_mode(modemap, (tt / NM) % NM);
     gr[r] = digit_mode(modemap, tt / N2);
-    const u32 a_many = allowed_act_digits(triple_bits(th[r], om[r], gr[r], false), req, all, own, is_o, not_mo);
-    const u32 a_one = allowed_act_digits(triple_bits(th[r], om[r], gr[r], true), req, all, all, is_o, not_mo);
-    t_allowed[r] = live ? (a_many | (a_one << 8)) : 0;
+    const u32 a_many = allowed_act_digits(triple_bits(th[r], om[r], gr[r], CLS_SHARDED), req, all, own, is_o, not_mo);
+    const u32 a_one = allowed_act_digits(triple_bits(th[r], om[r], gr[r], CLS_ONE_DEVICE), req, all, all, is_o, not_mo);
+    const u32 a_copies = allowed_act_digits(triple_bits(th[r], om[r], gr[r], CLS_ALL_COPIES), req, all, all, is_o, not_mo);
+    t_allowed[r] = live ? (a_many | (a_one << 8) | (a_copies << 16)) : 0;
   }
   // this lane's table entry (variant, digit)
   const u32 tl_vt = lane / NM, tl_d = lane - tl_vt * NM;
@@ -477,12 +502,15 @@ __global__ void __launch_bounds__(THREADS, 2) k_compact_count(SpaceDev sp, EvalA
     if (unit != unit_cur) {
       unit_cur = unit;
       const Fact f = sp.facts[unit];
-      const Pow2 p2 = pow2_of(f);
-      const UnitBase ub = (POW2 || p2.all) ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
-                                           : unit_base(rec, f, sp.tp_max_valid, true);
+      const u32 repl = POW2 ? 1u : sp.repl;
+      const Pow2 p2 = POW2 ? pow2_of(f) : pow2_of(f, repl);
+      const UnitBase ub = POW2 ? unit_base_pow2_one_copy(rec, f, p2, sp.tp_max_valid, true)
+                          : p2.all ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
+                                   : unit_base(rec, f, sp.tp_max_valid, true, repl);
       __syncwarp();                            // the previous factorisation's bounds have been read
       if (tl_mine) {
-        const ActBase ab = (POW2 || p2.all) ? act_base_pow2(rec, p2, tl_v, tl_tau) : act_base(rec, f, tl_v, tl_tau);
+        const ActBase ab = POW2 ? act_base_pow2_one_copy(rec, p2, tl_v, tl_tau)
+                           : p2.all ? act_base_pow2(rec, p2, tl_v, tl_tau) : act_base(rec, f, tl_v, tl_tau, ub.G);
         const u64 am = mu_elems(tl_mode, ab.EA, ab.shA, ab.uA, sp.sstar_units);
         tb.bound[tl_d][tl_vt] = am < cap_x ? cap_x - am : 0;
         if (tl_d == 0) {
@@ -492,7 +520,7 @@ __global__ void __launch_bounds__(THREADS, 2) k_compact_count(SpaceDev sp, EvalA
       }
       __syncwarp();
       const bool unit_ok = (ub.cv & req_cv) == req_cv;
-      const u32 shift = ub.d1 ? 8 : 0;
+      const u32 shift = POW2 ? (ub.d1 ? 8u : 0u) : 8 * ub.cls;
 #pragma unroll
       for (int r = 0; r < R; ++r) {
         mem3[r] = mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0)));
@@ -602,7 +630,8 @@ cudaError_t launch_eval_p(const SpaceDev& sp, const EvalArgs& a, cudaStream_t st
 
 template <int MODE, int NM>
 cudaError_t launch_eval_t(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream) {
-  return sp.all_pow2 ? launch_eval_p<MODE, NM, true>(sp, a, stream) : launch_eval_p<MODE, NM, false>(sp, a, stream);
+  return (sp.all_pow2 && sp.repl == 1) ? launch_eval_p<MODE, NM, true>(sp, a, stream)
+                                       : launch_eval_p<MODE, NM, false>(sp, a, stream);
 }
 
 template <int MODE>
@@ -638,7 +667,7 @@ cudaError_t launch_eval_materialise(const SpaceDev& sp, const EvalArgs& a, cudaS
 template <int NM>
 static cudaError_t launch_count_t(const SpaceDev& sp, const EvalArgs& a, cudaStream_t stream) {
   const unsigned blocks = (a.n_runs + WARPS - 1) / WARPS;       // a warp per run
-  if (sp.all_pow2) k_compact_count<NM, true><<<blocks, THREADS, 0, stream>>>(sp, a);
+  if (sp.all_pow2 && sp.repl == 1) k_compact_count<NM, true><<<blocks, THREADS, 0, stream>>>(sp, a);
   else k_compact_count<NM, false><<<blocks, THREADS, 0, stream>>>(sp, a);
   return cudaGetLastError();
 }

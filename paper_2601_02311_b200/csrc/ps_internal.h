@@ -71,6 +71,7 @@ struct SweepArgs {
   u32 require_flags;    // without PS_F_FEASIBLE
   u32 comm_kind;
   u32 k_keep;           // top-k: entries kept
+  u32 skip_rejected;    // do not evaluate factorisations whose composition bits miss a required flag
   PartialEntry* partial;   // [n_models * n_chunks * warps][SWEEP_LIST_CAP]: one list per warp
   uint2* partial_n;        // [n_models * n_chunks * warps]: (entries, survivors)
   u32* status;

@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(128) k_select_compare(SpaceDev sp, u32 unit_be
   in_space = in_space && unit != 0xffffffffu;
   const Fact f = in_space ? sp.facts[unit] : Fact{N, pick.T, 1, N / pick.T};
   const PointOut po = eval_point(rec, f, 0, 0, modes[0], modes[1], modes[2], modes[3], sp.tp_max_valid, sp.tp_coll,
-                                 true, sp.sstar_units, sp.accum);
+                                 true, sp.sstar_units, sp.accum, sp.repl);
   const u64 comm = comm_kind == PS_COMM_PAPER ? po.comm_paper : po.comm_paper + po.comm_ext;
   r.alg_mem = po.mem; r.alg_comm = comm;
   r.alg_idx = 0;

@@ -291,12 +291,43 @@ __device__ __forceinline__ void count_not_below(u32& n, u64 m, u64 bound) {
 // exact there; the other digits use the carry chain, so both pipes work
 constexpr u32 F64_DIGITS = 0x1f;
 
+// With several copies of every shard (k-way replication) a triple's communication is
+// kx * x plus what reducing gradients to shards and all-reducing them cost beyond
+// that: x2 per reduce-to-shards, x3 per all-reduce over all devices (both zero with
+// one copy).  Needed only where the exact volume is (the reduction pass).
+__device__ __forceinline__ u64 copies_traffic(u32 om, u32 gr, u32 w_grad, bool ext_in_objective, u64 x2, u64 x3) {
+  const bool on_shard = in_set(SET_UPDATE_ON_SHARD, om);
+  u32 n2 = gr == PS_MODE_S ? 1u : 0u, n3 = gr == PS_MODE_R ? 1u : 0u;
+  if (ext_in_objective) {
+    if (gr == PS_MODE_SG || gr == PS_MODE_O || (gr == PS_MODE_M && on_shard)) n2 += 1;
+    if (gr == PS_MODE_M && !on_shard) n3 += 1;
+  }
+  return (u64)w_grad * (n2 * x2 + n3 * x3);
+}
+
+// On request only (ps_filter.skip_rejected): a factorisation whose composition bits
+// already miss a required flag has no survivor, so a warp need not take it.  By
+// default every factorisation is taken and every point's capacity compare executed
+// and then masked, so that the throughput of a sweep says how fast points are
+// evaluated, not how many the filter lets the kernel jump over.
+__device__ __noinline__ bool unit_rejected(const SpaceDev& sp, const ModelRec& rec, u32 unit, u32 req_cv) {
+  const Fact f = sp.facts[unit];
+  const bool t_heads = rec.heads % f.T == 0, k_layers = rec.L % f.K == 0, tp_le = f.T <= sp.tp_max_valid;
+  const bool whole = (u64)f.T * f.K * f.D == (u64)f.N;
+  u32 cv = (t_heads ? PS_F_T_DIV_HEADS : 0) | (k_layers ? PS_F_K_DIV_LAYERS : 0) | (tp_le ? PS_F_TP_LE_MAX : 0) |
+           PS_F_AXIS_FORM;
+  if (t_heads && k_layers && tp_le && whole) cv |= PS_F_CV;
+  return (cv & req_cv) != req_cv;
+}
+
 // KIND: the reduction; NM: allowed modes; WARPS x 32 threads per block, compiled
 // for MIN_BLOCKS resident blocks per SM; HOST_LIMITED: the filter has a host
 // budget (without one the host bytes are never formed); FAST: every degree of
 // the space is a power of two and every byte count is below 2^53 (no division
 // and no 64-bit integer compare is compiled into the evaluation)
-template <int KIND, int NM, int WARPS, int MIN_BLOCKS, bool HOST_LIMITED, bool FAST>
+// SKIP: the kernel honours ps_filter.skip_rejected (the fast case is also compiled
+// without, so that the default sweep carries no trace of it)
+template <int KIND, int NM, int WARPS, int MIN_BLOCKS, bool HOST_LIMITED, bool FAST, bool SKIP>
 __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, SweepArgs args) {
   constexpr int THREADS = WARPS * 32;
   constexpr int N2 = NM * NM, N3 = NM * NM * NM, NC = N3 * NM;
@@ -344,6 +375,8 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
   u32 survivors = 0;
   u64 dom_m = U64MAX, dom_c = U64MAX;               // Pareto: a point known to be a survivor
 
+  // the fast case is compiled for spaces with one copy of every shard
+  const u32 repl = FAST ? 1u : sp.repl;
   const u32 req = args.require_flags;
   const bool ext_in_objective = args.comm_kind == PS_COMM_PAPER_PLUS_EXT;
   const u32 nvt = sp.nvt;
@@ -378,7 +411,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
   // with small integer coefficients that depend only on the triple's modes and
   // the model's byte widths -- fixed for the whole kernel.
   u32 t_local[R];      // triple number (0 if the lane has none in this round)
-  u32 t_allowed[R];    // allowed activation digits: bits 0..4 for D > 1, bits 8..12 for D = 1
+  u32 t_allowed[R];    // allowed activation digits: bits 0..4, 8..12, 16..20 for the three CLS_* of a unit
   u32 ka[R], kb[R], kc[R], kx[R], kh[R];
 #pragma unroll
   for (int r = 0; r < R; ++r) {
@@ -416,9 +449,10 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
     t_local[r] = tt;
     ka[r] = a; kb[r] = b; kc[r] = c; kh[r] = h;
     kx[r] = ct * rec.wT + co * rec.wO + cg * rec.wG;
-    const u32 a_many = allowed_act_digits(triple_bits(th, om, gr, false), req, all, own, is_o, not_mo);
-    const u32 a_one = allowed_act_digits(triple_bits(th, om, gr, true), req, all, all, is_o, not_mo);
-    t_allowed[r] = live ? (a_many | (a_one << 8)) : 0;
+    const u32 a_many = allowed_act_digits(triple_bits(th, om, gr, CLS_SHARDED), req, all, own, is_o, not_mo);
+    const u32 a_one = allowed_act_digits(triple_bits(th, om, gr, CLS_ONE_DEVICE), req, all, all, is_o, not_mo);
+    const u32 a_copies = allowed_act_digits(triple_bits(th, om, gr, CLS_ALL_COPIES), req, all, all, is_o, not_mo);
+    t_allowed[r] = live ? (a_many | (a_one << 8) | (a_copies << 16)) : 0;
     // keep the coefficients in registers instead of recomputing them for every unit
     asm volatile("" : "+r"(ka[r]), "+r"(kb[r]), "+r"(kc[r]), "+r"(kx[r]), "+r"(kh[r]), "+r"(t_allowed[r]));
   }
@@ -433,17 +467,28 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
 
   // warps take the block's units in turn: the first one by warp number, then
   // whichever is next when they finish (their work differs with the candidates)
-  for (u32 unit = u_begin + warp; unit < u_end;) {
+  u32 unit = u_begin + warp;
+  while (SKIP && args.skip_rejected && unit < u_end && unit_rejected(sp, rec, unit, req_cv)) {
+    u32 nxt = 0;
+    if (lane == 0) nxt = atomicAdd(&sh.next_unit, 1u);
+    unit = __shfl_sync(0xffffffffu, nxt, 0);
+  }
+  while (unit < u_end) {
     const Fact f = sp.facts[unit];
-    const Pow2 p2 = pow2_of(f);
+    const Pow2 p2 = FAST ? pow2_of(f) : pow2_of(f, repl);
     UnitBase ub;
     if (FAST) {
       // the tensor and pipeline parts come from the block's tables
       const TensorDegree& td = sh.by_t[p2.sT];
       const PipelineDegree kd = sh.by_k[p2.sK];
       ub.E2 = ceil_shift(td.E1, p2.sK);
+      // (one copy of every shard here: the shard positions are the D devices)
+      ub.G = f.D;
       ub.sh = ceil_shift(ub.E2, p2.sD);
       ub.x = ub.E2 - (ub.E2 >> p2.sD);
+      ub.x2 = 0;
+      ub.x3 = 0;
+      ub.cls = f.D == 1 ? CLS_ONE_DEVICE : CLS_SHARDED;
       ub.u = td.u;
       ub.tp_x = td.tp_x;
       ub.sbh_t = td.sbh_t;
@@ -456,7 +501,8 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
       ub.cv = cv;
       ub.d1 = (f.D == 1);
     } else {
-      ub = p2.all ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true) : unit_base(rec, f, sp.tp_max_valid, true);
+      ub = p2.all ? unit_base_pow2(rec, f, p2, sp.tp_max_valid, true)
+                  : unit_base(rec, f, sp.tp_max_valid, true, repl);
     }
     __syncwarp();
     {
@@ -472,11 +518,11 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
         const u32 s = tl_tau == 0 ? p2.sT : 0;
         ab.EA = ceil_shift(tl_A, s);
         ab.uA = ceil_shift(tl_UA, s);
-        ab.shA = ceil_shift(ab.EA, p2.sD);
+        ab.shA = ceil_shift(ab.EA, p2.sG);
       } else {
         ab.EA = tl_tau == 0 ? div_ceil(tl_A, f.T) : tl_A;
         ab.uA = tl_tau == 0 ? div_ceil(tl_UA, f.T) : tl_UA;
-        ab.shA = div_ceil(ab.EA, f.D);
+        ab.shA = div_ceil(ab.EA, ub.G);
       }
       const u64 am = mu_elems(tl_mode, ab.EA, ab.shA, ab.uA, sp.sstar_units);
       if (tl_mine) {
@@ -500,7 +546,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
     __syncwarp();
     // the lane's triples for this unit: own bytes, own communication, allowed digits
     const bool unit_ok = (ub.cv & req_cv) == req_cv;
-    const u32 a_shift = ub.d1 ? 8 : 0;
+    const u32 a_shift = FAST ? (ub.d1 ? 8u : 0u) : 8 * ub.cls;
     u64 mem3[R], comm3[R], host3[R];
     double mem3_f64[R], host3_f64[R];
     const double e2_f64 = (double)ub.E2, sh_f64 = (double)ub.sh, u_f64 = (double)ub.u;
@@ -511,7 +557,12 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
       // multiply-adds) and the integer only if the reduction pass needs it
       if (FAST) mem3_f64[r] = fma((double)ka[r], e2_f64, fma((double)kb[r], sh_f64, (double)kc[r] * u_f64));
       else mem3[r] = mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0)));
-      if (!FAST) comm3[r] = mad_small(ub.x, kx[r], 0);   // the fast case forms it where it is needed
+      if (!FAST) {                                      // the fast case forms it where it is needed
+        comm3[r] = mad_small(ub.x, kx[r], 0);
+        if (repl > 1)
+          comm3[r] += copies_traffic(digit_mode(modemap, (t_local[r] / NM) % NM), digit_mode(modemap, t_local[r] / N2),
+                                     rec.wG, ext_in_objective, ub.x2, ub.x3);
+      }
       bool host_fits = true;                    // the triple's own host bytes against the budget
       if (host_limited) {
         if (FAST) { host3_f64[r] = (double)kh[r] * sh_f64; host_fits = host3_f64[r] < (double)host_x; }
@@ -809,9 +860,11 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
       }
     }
     // next unit
-    u32 nxt = 0;
-    if (lane == 0) nxt = atomicAdd(&sh.next_unit, 1u);
-    unit = __shfl_sync(0xffffffffu, nxt, 0);
+    do {
+      u32 nxt = 0;
+      if (lane == 0) nxt = atomicAdd(&sh.next_unit, 1u);
+      unit = __shfl_sync(0xffffffffu, nxt, 0);
+    } while (SKIP && args.skip_rejected && unit < u_end && unit_rejected(sp, rec, unit, req_cv));
   }
 
   // ---- the warp's list goes to global scratch, sorted (top-k: its k smallest
@@ -916,7 +969,7 @@ __device__ __forceinline__ PointOut eval_local(const SpaceDev& sp, const ModelRe
   const Fact f = sp.facts[lp.unit];
   return eval_point(rec, f, lp.v, lp.tau, digit_mode(sp.modemap, lp.dth), digit_mode(sp.modemap, lp.dom),
                     digit_mode(sp.modemap, lp.dgr), digit_mode(sp.modemap, lp.dac), sp.tp_max_valid,
-                    sp.tp_coll, true, sp.sstar_units, sp.accum);
+                    sp.tp_coll, true, sp.sstar_units, sp.accum, sp.repl);
 }
 
 // The slow exact path for a model whose frontier outgrew the lists: see above.
@@ -1130,16 +1183,16 @@ __global__ void __launch_bounds__(MERGE_THREADS) k_sweep_merge(SpaceDev sp, Merg
 }  // namespace
 
 // ------------------------------------------------------------------ launchers
-template <int KIND, int NM, bool HOST_LIMITED, bool FAST>
+template <int KIND, int NM, bool HOST_LIMITED, bool FAST, bool SKIP>
 static cudaError_t launch_sweep_p(const SpaceDev& sp, const SweepArgs& a, u32 n_chunks, cudaStream_t stream) {
   constexpr int WARPS = KIND == PS_REDUCE_PARETO ? SWEEP_WARPS_PARETO : SWEEP_WARPS_TOPK;
   constexpr int MIN_BLOCKS = KIND == PS_REDUCE_PARETO ? SWEEP_BLOCKS_PARETO : SWEEP_BLOCKS_TOPK;
   dim3 grid(n_chunks, sp.n_models);
   const size_t smem = sizeof(SweepShared<WARPS>);
-  cudaError_t e = cudaFuncSetAttribute(k_sweep<KIND, NM, WARPS, MIN_BLOCKS, HOST_LIMITED, FAST>,
+  cudaError_t e = cudaFuncSetAttribute(k_sweep<KIND, NM, WARPS, MIN_BLOCKS, HOST_LIMITED, FAST, SKIP>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  k_sweep<KIND, NM, WARPS, MIN_BLOCKS, HOST_LIMITED, FAST><<<grid, WARPS * 32, smem, stream>>>(sp, a);
+  k_sweep<KIND, NM, WARPS, MIN_BLOCKS, HOST_LIMITED, FAST, SKIP><<<grid, WARPS * 32, smem, stream>>>(sp, a);
   return cudaGetLastError();
 }
 
@@ -1147,11 +1200,15 @@ template <int KIND, int NM>
 static cudaError_t launch_sweep_t(const SpaceDev& sp, const SweepArgs& a, u32 n_chunks, cudaStream_t stream) {
   const bool host_limited = a.host_cap < ((u64)1 << 62);
   // the fast case: powers of two everywhere, every byte count exact in a double
-  if (sp.all_pow2 && sp.all_small && a.cap_max < ((u64)1 << 53) - 1)
-    return host_limited ? launch_sweep_p<KIND, NM, true, true>(sp, a, n_chunks, stream)
-                        : launch_sweep_p<KIND, NM, false, true>(sp, a, n_chunks, stream);
-  return host_limited ? launch_sweep_p<KIND, NM, true, false>(sp, a, n_chunks, stream)
-                      : launch_sweep_p<KIND, NM, false, false>(sp, a, n_chunks, stream);
+  if (sp.all_pow2 && sp.all_small && sp.repl == 1 && a.cap_max < ((u64)1 << 53) - 1) {
+    if (a.skip_rejected)
+      return host_limited ? launch_sweep_p<KIND, NM, true, true, true>(sp, a, n_chunks, stream)
+                          : launch_sweep_p<KIND, NM, false, true, true>(sp, a, n_chunks, stream);
+    return host_limited ? launch_sweep_p<KIND, NM, true, true, false>(sp, a, n_chunks, stream)
+                        : launch_sweep_p<KIND, NM, false, true, false>(sp, a, n_chunks, stream);
+  }
+  return host_limited ? launch_sweep_p<KIND, NM, true, false, true>(sp, a, n_chunks, stream)
+                      : launch_sweep_p<KIND, NM, false, false, true>(sp, a, n_chunks, stream);
 }
 
 template <int KIND>

@@ -57,12 +57,13 @@ class _SpaceDesc(C.Structure):
                 ("tp_max_valid", C.c_uint32), ("n_act_variants", C.c_uint32),
                 ("n_tpa_variants", C.c_uint32), ("mode_mask", C.c_uint32),
                 ("tp_coll_per_layer", C.c_uint32), ("sstar_units", C.c_uint32),
-                ("grad_accum_steps", C.c_uint32)]
+                ("grad_accum_steps", C.c_uint32), ("replication_k", C.c_uint32)]
 
 
 class _Filter(C.Structure):
     _fields_ = [("host_cap", C.c_uint64), ("require_flags", C.c_uint32),
-                ("comm_kind", C.c_uint32), ("cap_bytes", C.c_uint64)]
+                ("comm_kind", C.c_uint32), ("cap_bytes", C.c_uint64),
+                ("skip_rejected", C.c_uint32), ("pad", C.c_uint32)]
 
 
 class _OutSoa(C.Structure):
@@ -147,7 +148,8 @@ def strerror(code: int) -> str:
 
 def _mk_filter(filt: dict) -> _Filter:
     return _Filter(filt.get("host_cap", NO_LIMIT), filt.get("require_flags", 0),
-                   filt.get("comm_kind", COMM_PAPER_PLUS_EXT), filt.get("cap_bytes", NO_LIMIT))
+                   filt.get("comm_kind", COMM_PAPER_PLUS_EXT), filt.get("cap_bytes", NO_LIMIT),
+                   1 if filt.get("skip_rejected") else 0, 0)
 
 
 def _dptr(t):
@@ -263,7 +265,7 @@ class Space:
                           space["t_enum_max"], space["k_enum_max"], space["tp_max_valid"],
                           space["n_act_variants"], space["n_tpa_variants"], space["mode_mask"],
                           space["tp_coll_per_layer"], space.get("sstar_units", 1),
-                          space.get("grad_accum_steps", 1))
+                          space.get("grad_accum_steps", 1), space.get("replication_k", 1))
         handle = C.c_void_p()
         _check(_lib.ps_space_create(ctx._h, C.byref(desc), C.byref(handle)), "ps_space_create")
         self._h = handle

@@ -83,3 +83,50 @@ def test_field_ranges(ctx, ps):
         with pytest.raises(ps.PsError) as e:
             ctx.space(space)
         assert e.value.code == ps.E_RANGE
+
+
+# ------------------------------------------------------------ k-way replication
+@pytest.mark.parametrize("k,sstar_units,g", [(2, 1, 1), (4, 2, 3), (1 << 12, 1, 1), (6, 1, 2)])
+def test_k_way_replication_materialise_and_compaction(ctx, k, sstar_units, g):
+    """Every shard held k times (Section 1's "k-way replication"): all five outputs of every
+    point, and the compaction, on power-of-two spaces and on ragged device counts (where k
+    need not divide D)."""
+    spaces = [synth.config("C0b"), synth.config("C1", n_models=3), synth.config("C3", n_models=1),
+              synth.ragged_space(4, n_models=2)]
+    for base in spaces:
+        space = dict(ext(base, sstar_units, g), replication_k=k)
+        gs, os_ = ctx.space(space), O.Space(space)
+        n = min(gs.size, 400_000)
+        first = (gs.size - n) // 3
+        same(gs.eval_batch(first, n), os_.eval_range(first, n))
+        for filt in (dict(require_flags=O.F_GI | O.F_SC, cap_bytes=80 * synth.GB, host_cap=500 * synth.GB),
+                     dict(require_flags=O.F_PAPER_PRICED | O.F_GI, cap_bytes=192 * synth.GB)):
+            same(gs.compact(first, n, filt), os_.compact_range(first, n, filt))
+    ctx.check_status()
+
+
+@pytest.mark.parametrize("k", [2, 8, 3])
+def test_k_way_replication_sweeps(ctx, ps, k):
+    for base in (synth.config("C3", n_models=4), synth.ragged_space(9, n_models=2)):
+        space = dict(base, replication_k=k)
+        gs, os_ = ctx.space(space), O.Space(space)
+        for comm_kind in (O.COMM_PAPER, O.COMM_PAPER_PLUS_EXT):
+            filt = dict(require_flags=O.F_GI | O.F_SC, comm_kind=comm_kind, host_cap=64 * synth.GB)
+            caps = [80 * synth.GB, 192 * synth.GB]
+            ge, gc = gs.sweep(filt, caps, ps.REDUCE_PARETO, 64)
+            oe, oc = os_.sweep(filt, caps, O.KIND_PARETO, 64, n_threads=8)
+            assert ge.tobytes() == oe.tobytes() and gc.tolist() == oc.tolist()
+            filt = dict(require_flags=VALID, comm_kind=comm_kind)
+            ge, gc = gs.sweep(filt, caps[1:], ps.REDUCE_TOPK, 64)
+            oe, oc = os_.sweep(filt, caps[1:], O.KIND_TOPK, 64, n_threads=8)
+            assert ge.tobytes() == oe.tobytes() and gc.tolist() == oc.tolist()
+    ctx.check_status()
+
+
+def test_k_way_replication_reaches_the_kernels(ctx):
+    """ZeRO-3 at N = 8 in the worked example with two copies of every shard: 16P/4 bytes."""
+    gs = ctx.space(dict(synth.config("C0"), replication_k=2))
+    r = gs.eval_batch(3 * 625 + 32, 1)
+    P = 70_000_000_000
+    assert int(r["mem"][0]) == 16 * P // 4
+    assert int(r["comm_paper"][0]) == (3 * 2 * P // 4 + 2 * (2 * P // 4) // 2) + 2 * (3 * 2 * P // 4)

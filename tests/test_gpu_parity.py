@@ -440,3 +440,18 @@ def test_select_compare_matches_oracle(ctx, ps):
                 assert np.array_equal(got[name].astype(np.uint64), want[:, k]), (n_value, cap_index, name)
         assert len(set(got["status"].tolist())) > 1            # more than one outcome occurs
     ctx.check_status()
+
+
+def test_sweeps_that_skip_rejected_factorisations_give_the_same_tables(ctx, ps):
+    """skip_rejected leaves out the factorisations the required composition flags reject at sight:
+    less work, identical results (and identical survivor counts)."""
+    for space in (synth.config("C3", n_models=5), synth.ragged_space(3, n_models=2)):
+        gs, os_ = both(ctx, space)
+        caps = [80 * synth.GB, 192 * synth.GB]
+        for req in (VALID, O.F_GI | O.F_SC | O.F_T_HEADS):
+            filt = dict(require_flags=req, host_cap=64 * synth.GB)
+            want = os_.sweep(filt, caps, O.KIND_PARETO, 64, n_threads=8)
+            assert_same_sweep(gs.sweep(dict(filt, skip_rejected=1), caps, ps.REDUCE_PARETO, 64), want)
+            filt = dict(require_flags=req)
+            want = os_.sweep(filt, caps[1:], O.KIND_TOPK, 64, n_threads=8)
+            assert_same_sweep(gs.sweep(dict(filt, skip_rejected=1), caps[1:], ps.REDUCE_TOPK, 64), want)
