@@ -159,9 +159,10 @@ int ps_create(ps_ctx** out, int device, void* cuda_stream) {
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return PS_E_CUDA; }
   ctx->sm_count = prop.multiProcessorCount;
-  if (cudaMalloc(&ctx->d_status, sizeof(u32)) != cudaSuccess ||
+  ctx->compact_calls = 0;
+  if (cudaMalloc(&ctx->d_status, 4 * sizeof(u32)) != cudaSuccess ||
       cudaMallocHost(&ctx->h_status, sizeof(u32)) != cudaSuccess ||
-      cudaMemsetAsync(ctx->d_status, 0, sizeof(u32), ctx->stream) != cudaSuccess) {
+      cudaMemsetAsync(ctx->d_status, 0, 4 * sizeof(u32), ctx->stream) != cudaSuccess) {
     ps_destroy(ctx);
     return PS_E_CUDA;
   }
@@ -404,10 +405,13 @@ int ps_eval_batch(ps_ctx* ctx, const ps_space* sp, uint64_t first, uint64_t coun
     char* base = static_cast<char*>(ctx->scratch);
     a.tile_count = reinterpret_cast<u32*>(base);
     a.nonempty = reinterpret_cast<u32*>(base + cnt_bytes);
-    a.n_nonempty = reinterpret_cast<u32*>(base + 2 * cnt_bytes);
     a.tile_offset = reinterpret_cast<u64*>(base + 2 * cnt_bytes + 16);
+    // the list's length: one of the context's two counters, zero by now (the previous
+    // compaction's scan cleared it); this call's scan clears the other
+    a.n_nonempty = ctx->d_status + 2 + (ctx->compact_calls & 1u);
+    a.n_nonempty_other = ctx->d_status + 2 + ((ctx->compact_calls + 1) & 1u);
+    ++ctx->compact_calls;
     eval_plan_runs(a);
-    CUDA_OK(cudaMemsetAsync(a.n_nonempty, 0, sizeof(u32), ctx->stream));
     CUDA_OK(launch_eval_count(sp->dev, a, ctx->stream));
     CUDA_OK(launch_tile_scan(a, ctx->stream));
     CUDA_OK(launch_eval_write(sp->dev, a, ctx->stream));

@@ -195,7 +195,8 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
   for (u32 it = it_begin; it < it_end; it += it_step) {
     const u32 seg = MODE == MODE_WRITE ? a.nonempty[it] : it;
     const u64 g = a.first_group + seg;
-    const u32 model = (u32)(g / groups_per_model);
+    // (a 32-bit division where the group number allows it: it is done once per group by every lane)
+    const u32 model = (g >> 32) == 0 ? (u32)g / groups_per_model : (u32)(g / groups_per_model);
     const u32 gl = (u32)(g - (u64)model * groups_per_model);
     const u32 unit = gl / sp.nvt, vt = gl - unit * sp.nvt;
     const u32 v = vt / sp.nt, tau = vt - v * sp.nt;
@@ -470,11 +471,17 @@ __global__ void __launch_bounds__(THREADS, 2) k_compact_count(SpaceDev sp, EvalA
   u32 with_survivors = 0;                  // bit j: group seg_begin + j has survivors
   const u64 window_end = a.first + a.count;
 
+  // the run's first group by division, the following ones by counting up
+  u32 model, unit, vt;
+  {
+    const u64 g0 = a.first_group + seg_begin;
+    model = (u32)(g0 / groups_per_model);
+    const u32 gl = (u32)(g0 - (u64)model * groups_per_model);
+    unit = gl / sp.nvt;
+    vt = gl - unit * sp.nvt;
+  }
   for (u32 seg = seg_begin; seg < seg_end; ++seg) {
     const u64 g = a.first_group + seg;
-    const u32 model = (u32)(g / groups_per_model);
-    const u32 gl = (u32)(g - (u64)model * groups_per_model);
-    const u32 unit = gl / sp.nvt, vt = gl - unit * sp.nvt;
     if (model != model_cur) {
       model_cur = model;
       unit_cur = 0xffffffffu;
@@ -553,6 +560,11 @@ __global__ void __launch_bounds__(THREADS, 2) k_compact_count(SpaceDev sp, EvalA
     if (lane == 0) a.tile_count[seg] = n;
     run_total += n;
     if (n) with_survivors |= 1u << (seg - seg_begin);
+    // the next group: next variant, else next factorisation, else next model
+    if (++vt == sp.nvt) {
+      vt = 0;
+      if (++unit == sp.n_facts) { unit = 0; ++model; }
+    }
   }
   if (lane == 0) a.tile_offset[run] = run_total;
   // the groups with survivors join the write pass's list (in any order: a group's place
@@ -606,7 +618,10 @@ __global__ void __launch_bounds__(SCAN_THREADS) k_tile_scan(EvalArgs a) {
     if (tid == SCAN_THREADS - 1) carry = before + incl;
     __syncthreads();
   }
-  if (tid == 0) *a.n_out = carry;
+  if (tid == 0) {
+    *a.n_out = carry;
+    *a.n_nonempty_other = 0;      // the next compaction's list starts empty
+  }
 }
 
 template <int MODE, int NM, bool POW2>

@@ -12,8 +12,9 @@ struct ps_ctx {
   cudaStream_t stream;
   void* scratch;
   size_t scratch_bytes;
-  u32* d_status;
+  u32* d_status;      // 16 bytes: the status word, then (at +2) the two list lengths of the compaction
   u32* h_status;      // pinned
+  u32 compact_calls;  // compactions enqueued so far (picks which list length a call uses)
   int sm_count;
 };
 
@@ -121,6 +122,8 @@ struct EvalArgs {
   u32* tile_count;          // [n_tiles] survivors of each group
   u32* nonempty;            // [n_tiles] the groups that have survivors, in any order
   u32* n_nonempty;          // how many (zero before the count pass)
+  u32* n_nonempty_other;    // the next compaction's counter: the scan kernel clears it, so that no
+                            // call needs a memset of its own (calls alternate between two counters)
   u64* tile_offset;         // [n_runs <= n_tiles] survivors of each run, then (scan) of all runs before it
   u32* status;
 };

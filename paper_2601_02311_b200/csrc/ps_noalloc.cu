@@ -102,7 +102,9 @@ extern "C" int ps_eval_compact_noalloc(ps_ctx* ctx, const ps_space* sp, uint64_t
   unsigned char* bytes = static_cast<unsigned char*>(base);
   a.tile_count = reinterpret_cast<u32*>(bytes);
   a.nonempty = reinterpret_cast<u32*>(bytes + COUNT_BYTES);
-  a.n_nonempty = reinterpret_cast<u32*>(bytes + 2 * COUNT_BYTES);
+  a.n_nonempty = ctx->d_status + 2 + (ctx->compact_calls & 1u);          // the context's alternating list lengths
+  a.n_nonempty_other = ctx->d_status + 2 + ((ctx->compact_calls + 1) & 1u);
+  ++ctx->compact_calls;
   a.tile_offset = reinterpret_cast<u64*>(bytes + 2 * COUNT_BYTES + LENGTH_BYTES);
   eval_plan_runs(a);
   // The array still holds the previous call's numbers.  Every word this call
@@ -111,7 +113,6 @@ extern "C" int ps_eval_compact_noalloc(ps_ctx* ctx, const ps_space* sp, uint64_t
   // into offsets); the counts are cleared anyway so that a stale value can
   // never be mistaken for a fresh one.
   if (cudaMemsetAsync(a.tile_count, 0, sizeof(u32) * n_groups, ctx->stream) != cudaSuccess) return PS_E_CUDA;
-  if (cudaMemsetAsync(a.n_nonempty, 0, sizeof(u32), ctx->stream) != cudaSuccess) return PS_E_CUDA;   // the list starts empty
   if (launch_eval_count(sp->dev, a, ctx->stream) != cudaSuccess) return PS_E_CUDA;
   if (launch_tile_scan(a, ctx->stream) != cudaSuccess) return PS_E_CUDA;
   if (launch_eval_write(sp->dev, a, ctx->stream) != cudaSuccess) return PS_E_CUDA;

@@ -1030,8 +1030,11 @@ __device__ __noinline__ void frontier_by_definition(const SpaceDev& sp, const Me
   }
 }
 
+// (compiled for eight resident blocks per SM: the kernel is a chain of short steps between
+// barriers, so it lives on many blocks in flight; the slow exact path, which is
+// rarely taken, must not cost the common path its registers)
 template <int KIND>
-__global__ void __launch_bounds__(MERGE_THREADS) k_sweep_merge(SpaceDev sp, MergeArgs args) {
+__global__ void __launch_bounds__(MERGE_THREADS, 8) k_sweep_merge(SpaceDev sp, MergeArgs args) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   MergeShared& sh = *reinterpret_cast<MergeShared*>(smem_raw);
   const int tid = threadIdx.x;
