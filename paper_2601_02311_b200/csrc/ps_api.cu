@@ -438,7 +438,8 @@ int ps_sweep_pareto(ps_ctx* ctx, const ps_space* sp, const ps_filter* filter,
   const u32 n_chunks = pick_chunks(ctx, sp, (int)reduce_kind);
   const size_t slots = (size_t)sp->dev.n_models * n_chunks * sweep_warps((int)reduce_kind);   // one list per warp
   const size_t partial_bytes = slots * SWEEP_LIST_CAP * sizeof(PartialEntry);
-  rc = ensure_scratch(ctx, partial_bytes + slots * sizeof(uint2));
+  const size_t lengths_bytes = (slots * sizeof(uint2) + 15) & ~size_t(15);
+  rc = ensure_scratch(ctx, partial_bytes + lengths_bytes + sizeof(u32) * (size_t)sp->dev.n_models);
   if (rc != PS_OK) return rc;
   SweepArgs s;
   memset(&s, 0, sizeof(s));
@@ -463,6 +464,7 @@ int ps_sweep_pareto(ps_ctx* ctx, const ps_space* sp, const ps_filter* filter,
   m.comm_kind = filter->comm_kind;
   m.out = d_out;
   m.counts = d_counts;
+  m.slow_path = reinterpret_cast<u32*>(static_cast<char*>(ctx->scratch) + partial_bytes + lengths_bytes);
   m.status = ctx->d_status;
   if (reduce_kind == PS_REDUCE_PARETO) {
     u64 cap_max = 0;

@@ -93,6 +93,7 @@ struct MergeArgs {
   u32 comm_kind;
   ps_front_entry* out;
   u32* counts;
+  u32* slow_path;       // Pareto, [n_models]: set by the merge for a model whose frontier outgrew the lists
   u32* status;
 };
 

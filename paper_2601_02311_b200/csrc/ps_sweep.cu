@@ -911,7 +911,6 @@ constexpr int MERGE_LISTS = 16;             // most lists a round takes (they ar
 constexpr int MERGE_MAX_LISTS = SWEEP_MAX_CHUNKS * (SWEEP_WARPS_PARETO > SWEEP_WARPS_TOPK ? SWEEP_WARPS_PARETO : SWEEP_WARPS_TOPK);
 
 struct MergeShared {
-  Key pass_best[MERGE_THREADS / 32];        // slow path: the warps' best candidates of a pass
   u64 in_a[MERGE_CAP], in_b[MERGE_CAP];     // the kept entries, then the round's lists
   u32 in_i[MERGE_CAP];
   u64 a[MERGE_CAP], b[MERGE_CAP];           // the sorted union; after the cut, the kept entries
@@ -973,8 +972,13 @@ __device__ __forceinline__ PointOut eval_local(const SpaceDev& sp, const ModelRe
 }
 
 // The slow exact path for a model whose frontier outgrew the lists: see above.
-__device__ __noinline__ void frontier_by_definition(const SpaceDev& sp, const MergeArgs& args, u32 model,
-                                                    const ModelRec& rec, MergeShared& sh) {
+// A kernel of its own, launched after every Pareto merge, so that the merge kernel does not
+// carry its registers; a block whose model needs no slow path returns at once.
+__global__ void __launch_bounds__(MERGE_THREADS) k_frontier_by_definition(SpaceDev sp, MergeArgs args) {
+  __shared__ Key pass_best[MERGE_THREADS / 32];    // the warps' best candidates of a pass
+  const u32 model = blockIdx.x;
+  if (args.slow_path[model] == 0) return;
+  const ModelRec rec = sp.recs[model];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   u32 found[PS_MAX_CAPS];
   for (u32 ci = 0; ci < PS_MAX_CAPS; ++ci) found[ci] = 0;
@@ -997,11 +1001,11 @@ __device__ __noinline__ void frontier_by_definition(const SpaceDev& sp, const Me
       const Key other = key_shfl_xor(best, o);
       if (key_less(other, best)) best = other;
     }
-    if (lane == 0) sh.pass_best[warp] = best;
+    if (lane == 0) pass_best[warp] = best;
     __syncthreads();
-    best = sh.pass_best[0];
+    best = pass_best[0];
     for (int w = 1; w < MERGE_THREADS / 32; ++w)
-      if (key_less(sh.pass_best[w], best)) best = sh.pass_best[w];
+      if (key_less(pass_best[w], best)) best = pass_best[w];
     __syncthreads();
     if (best.i == 0xffffffffu) break;                   // nothing beyond the last entry: done
     for (u32 ci = 0; ci < args.n_caps; ++ci) {
@@ -1030,11 +1034,13 @@ __device__ __noinline__ void frontier_by_definition(const SpaceDev& sp, const Me
   }
 }
 
-// (compiled for eight resident blocks per SM: the kernel is a chain of short steps between
-// barriers, so it lives on many blocks in flight; the slow exact path, which is
-// rarely taken, must not cost the common path its registers)
+// compiled for eight resident blocks per SM (64 registers): the kernel is a chain of
+// short steps between barriers, so it lives on many blocks in flight
+#ifndef SWEEP_MERGE_MIN_BLOCKS
+#define SWEEP_MERGE_MIN_BLOCKS 8
+#endif
 template <int KIND>
-__global__ void __launch_bounds__(MERGE_THREADS, 8) k_sweep_merge(SpaceDev sp, MergeArgs args) {
+__global__ void __launch_bounds__(MERGE_THREADS, SWEEP_MERGE_MIN_BLOCKS) k_sweep_merge(SpaceDev sp, MergeArgs args) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   MergeShared& sh = *reinterpret_cast<MergeShared*>(smem_raw);
   const int tid = threadIdx.x;
@@ -1140,9 +1146,10 @@ __global__ void __launch_bounds__(MERGE_THREADS, 8) k_sweep_merge(SpaceDev sp, M
   const u32 s_survivors = sh.survivors;
 
   const ModelRec rec = sp.recs[model];
-  if (KIND == PS_REDUCE_PARETO && overflowed) {
-    frontier_by_definition(sp, args, model, rec, sh);
-    return;
+  if (KIND == PS_REDUCE_PARETO) {
+    // a frontier that outgrew the lists is left to the slow exact kernel that follows
+    if (tid == 0) args.slow_path[model] = overflowed ? 1u : 0u;
+    if (overflowed) return;
   }
   for (u32 ci = 0; ci < args.n_caps; ++ci) {
     const u64 cap = args.caps[ci];
@@ -1238,6 +1245,7 @@ cudaError_t launch_sweep_merge(int kind, const SpaceDev& sp, const MergeArgs& a,
     e = cudaFuncSetAttribute(k_sweep_merge<PS_REDUCE_PARETO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     k_sweep_merge<PS_REDUCE_PARETO><<<sp.n_models, MERGE_THREADS, smem, stream>>>(sp, a);
+    k_frontier_by_definition<<<sp.n_models, MERGE_THREADS, 0, stream>>>(sp, a);
   } else {
     e = cudaFuncSetAttribute(k_sweep_merge<PS_REDUCE_TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
