@@ -542,18 +542,31 @@ __global__ void __launch_bounds__(THREADS, 2) k_compact_count(SpaceDev sp, EvalA
     const bool whole = code_lo == 0 && code_hi == (u32)NC;
     const u64 host_bound = tb.host_bound[vt];
     u32 n = 0;
+    if (whole) {
+      // the usual case: per point one compare, masked by the digit's bit
 #pragma unroll
-    for (int d = 0; d < NM; ++d) {
-      const u64 bound = tb.bound[d][vt];
-      const bool offload = (is_o >> d) & 1u;
+      for (int d = 0; d < NM; ++d) {
+        const u64 bound = tb.bound[d][vt];
+        const bool offload = (is_o >> d) & 1u;
 #pragma unroll
-      for (int r = 0; r < R; ++r) {
-        bool pass = ((allowed[r] >> d) & 1u) && mem3[r] < bound && (!offload || host3[r] < host_bound);
-        if (!whole) {
-          const u32 code = lane + 32 * r + d * N3;
-          pass = pass && code >= code_lo && code < code_hi;
+        for (int r = 0; r < R; ++r) {
+          const bool pass = mem3[r] < bound && (!offload || host3[r] < host_bound);
+          n += pass ? ((allowed[r] >> d) & 1u) : 0u;
         }
-        n += pass ? 1u : 0u;
+      }
+    } else {
+      // a group at the window's edge: only the codes inside it
+#pragma unroll 1
+      for (int d = 0; d < NM; ++d) {
+        const u64 bound = tb.bound[d][vt];
+        const bool offload = (is_o >> d) & 1u;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          const u32 code = lane + 32 * r + d * N3;
+          const bool pass = ((allowed[r] >> d) & 1u) && mem3[r] < bound && (!offload || host3[r] < host_bound) &&
+                            code >= code_lo && code < code_hi;
+          n += pass ? 1u : 0u;
+        }
       }
     }
     n = __reduce_add_sync(0xffffffffu, n);
