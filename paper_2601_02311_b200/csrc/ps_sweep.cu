@@ -696,7 +696,115 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
         }
       }
     }
-    if (__any_sync(0xffffffffu, matters)) {
+    if (KIND == PS_REDUCE_PARETO && __any_sync(0xffffffffu, matters)) {
+      // About one unit in ten comes here (every unit with a survivor), so this part is
+      // written for few instructions and independent chains: the lane's triples stay in
+      // registers and are handled side by side, only the variants are a rolled loop.
+      u64 l_mem[R], l_comm[R], l_host[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        l_mem[r] = FAST ? mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0))) : mem3[r];
+        l_comm[r] = FAST ? mad_small(ub.x, kx[r], 0) : comm3[r];
+        l_host[r] = (FAST && host_limited) ? mad_small(ub.sh, kh[r], 0) : host3[r];
+      }
+      {
+        // lane = a set of activation digits; which of them costs the least bytes
+        // (the variants side by side: four independent chains)
+        u64 least[4];
+        u32 which[4];
+#pragma unroll
+        for (int vt = 0; vt < 4; ++vt) { least[vt] = U64MAX; which[vt] = NM; }
+#pragma unroll
+        for (int d = NM - 1; d >= 0; --d) {
+#pragma unroll
+          for (int vt = 0; vt < 4; ++vt) {
+            const u64 am = tb.act[vt < (int)nvt ? vt : 0][d];
+            if (((lane >> d) & 1) && am <= least[vt]) { least[vt] = am; which[vt] = d; }
+          }
+        }
+#pragma unroll
+        for (int vt = 0; vt < 4; ++vt) tb.least[vt][lane] = (unsigned char)which[vt];
+      }
+      __syncwarp();
+
+      // Variants in an order in which later ones seldom beat earlier ones (the result
+      // does not depend on the order, the work does): the tensor axis that shards
+      // activations first, and full checkpointing before stored activations -- fewer
+      // bytes at the same communication.
+#pragma unroll 1
+      for (u32 vt_step = 0; vt_step < nvt; ++vt_step) {
+        const u32 vt = (sp.nv - 1 - vt_step % sp.nv) * sp.nt + vt_step / sp.nv;
+        const u64 c_axis = tb.c_axis[vt], host_bound = tb.host_bound[vt];
+        const u32 vt_first = unit_first + vt * NC;
+        u64 bound[NM];
+#pragma unroll
+        for (int d = 0; d < NM; ++d) bound[d] = tb.bound[d][vt];
+        // For a triple and variant the communication is the same for all NM activation
+        // digits, so of the surviving digits only the one with the least bytes (lowest
+        // digit on ties) can be on the frontier.  Digit d is a survivor if the triple's
+        // bytes are below the digit's bound and the flags allow the digit.
+        u64 m[R], c[R];
+        u32 idx[R];
+        bool cand[R];
+        bool some = false;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          u32 fit = 0;
+#pragma unroll
+          for (int d = 0; d < NM; ++d) fit |= (l_mem[r] < bound[d]) ? (1u << d) : 0u;
+          // offloading activations adds host bytes: drop that digit if they do not fit
+          const u32 allow_vt = (!host_limited || l_host[r] < host_bound) ? allowed[r] : (allowed[r] & ~is_o);
+          const u32 pass = fit & allow_vt;
+          const bool has = pass != 0;
+          const u32 d = has ? tb.least[vt][pass] : 0;
+          m[r] = l_mem[r] + tb.act[vt][d];
+          c[r] = l_comm[r] + c_axis;
+          idx[r] = vt_first + t_local[r] + d * N3;
+          // cheap tests: strictly dominated by a point already known to survive, or by
+          // the block's coarse staircase
+          const int bucket = stair_bucket(m[r]);
+          const u64 step = sh.stair[bucket > 0 ? bucket - 1 : 0];
+          cand[r] = has && !(dom_m <= m[r] && dom_c <= c[r] && (dom_m != m[r] || dom_c != c[r])) &&
+                    !(bucket > 0 && step <= c[r]);
+          some = some || cand[r];
+        }
+        if (!__any_sync(0xffffffffu, some)) continue;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          if (!__any_sync(0xffffffffu, cand[r])) continue;
+          bool offer = cand[r];
+          if (offer) {
+            int lo = 0, hi = list.n;
+            while (lo < hi) {               // entries with mem <= m
+              const int mid = (lo + hi) >> 1;
+              if (list.a[mid] <= m[r]) lo = mid + 1; else hi = mid;
+            }
+            if (lo > 0) {
+              const u64 em = list.a[lo - 1], ec = list.b[lo - 1];
+              if (ec < c[r] || (ec == c[r] && (em < m[r] || list.i[lo - 1] < idx[r]))) {
+                offer = false;
+                dom_m = em; dom_c = ec;
+              }
+            }
+          }
+          u32 pending = __ballot_sync(0xffffffffu, offer);
+          while (pending) {
+            const int src = __ffs(pending) - 1;
+            const u64 pm = __shfl_sync(0xffffffffu, m[r], src);
+            const u64 pc = __shfl_sync(0xffffffffu, c[r], src);
+            const u32 pi = __shfl_sync(0xffffffffu, idx[r], src);
+            pareto_insert(list, pm, pc, pi, lane, sh.stair);
+            // what the offered point strictly dominates need not be offered
+            if (lane == src || (pm <= m[r] && pc <= c[r] && (pm != m[r] || pc != c[r]))) {
+              if (offer && lane != src) { dom_m = pm; dom_c = pc; }
+              offer = false;
+            }
+            pending = __ballot_sync(0xffffffffu, offer);
+          }
+        }
+      }
+    }
+    if (KIND == PS_REDUCE_TOPK && __any_sync(0xffffffffu, matters)) {
       // This part runs for a few units in a hundred, so it is written as rolled
       // loops over the lane's triples, whose values it first copies to arrays that
       // can be indexed at run time: code that is rarely executed is not in the
@@ -711,25 +819,6 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
         l_host[r] = (FAST && host_limited) ? mad_small(ub.sh, kh[r], 0) : host3[r];
         l_allowed[r] = allowed[r]; l_triple[r] = t_local[r];
       }
-      if (KIND == PS_REDUCE_PARETO) {
-        // lane = a set of activation digits; which of them costs the least bytes
-        for (u32 vt = 0; vt < nvt; ++vt) {
-          u64 least = U64MAX;
-          u32 which = NM;
-#pragma unroll 1
-          for (int d = NM - 1; d >= 0; --d) {
-            const u64 am = tb.act[vt][d];
-            if (((lane >> d) & 1) && am <= least) { least = am; which = d; }
-          }
-          tb.least[vt][lane] = (unsigned char)which;
-        }
-        __syncwarp();
-      }
-
-      // Variants in an order in which later ones seldom beat earlier ones (the result
-      // does not depend on the order, the work does): the tensor axis that shards
-      // activations first, and full checkpointing before stored activations -- fewer
-      // bytes at the same communication.
 #pragma unroll 1
       for (u32 vt_step = 0; vt_step < nvt; ++vt_step) {
         const u32 vt = (sp.nv - 1 - vt_step % sp.nv) * sp.nt + vt_step / sp.nv;
@@ -749,52 +838,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
           some = some || l_pass[r] != 0;
         }
         if (!__any_sync(0xffffffffu, some)) continue;
-
-        if (KIND == PS_REDUCE_PARETO) {
-          // For a triple and variant the communication is the same for all NM
-          // activation digits, so of the surviving digits only the one with the
-          // least bytes (lowest digit on ties) can be on the frontier.
-#pragma unroll 1
-          for (int r = 0; r < R; ++r) {
-            const u32 pass = l_pass[r];
-            const bool has = pass != 0;
-            const u32 d = has ? tb.least[vt][pass] : 0;
-            const u64 m = l_mem[r] + tb.act[vt][d];
-            const u64 c = l_comm[r] + c_axis;
-            const u32 idx = vt_first + l_triple[r] + d * N3;
-            // cheap tests first: strictly dominated by a point already known to survive
-            bool cand = has && !(dom_m <= m && dom_c <= c && (dom_m != m || dom_c != c));
-            if (cand) {
-              const int bucket = stair_bucket(m);
-              if (bucket > 0 && sh.stair[bucket - 1] <= c) cand = false;
-            }
-            if (__any_sync(0xffffffffu, cand)) {
-              if (cand) {
-                int lo = 0, hi = list.n;
-                while (lo < hi) {               // entries with mem <= m
-                  const int mid = (lo + hi) >> 1;
-                  if (list.a[mid] <= m) lo = mid + 1; else hi = mid;
-                }
-                if (lo > 0) {
-                  const u64 em = list.a[lo - 1], ec = list.b[lo - 1];
-                  if (ec < c || (ec == c && (em < m || list.i[lo - 1] < idx))) {
-                    cand = false;
-                    dom_m = em; dom_c = ec;
-                  }
-                }
-              }
-              u32 pending = __ballot_sync(0xffffffffu, cand);
-              while (pending) {
-                const int src = __ffs(pending) - 1;
-                pending &= pending - 1;
-                const u64 pm = __shfl_sync(0xffffffffu, m, src);
-                const u64 pc = __shfl_sync(0xffffffffu, c, src);
-                const u32 pi = __shfl_sync(0xffffffffu, idx, src);
-                pareto_insert(list, pm, pc, pi, lane, sh.stair);
-              }
-            }
-          }
-        } else {
+        {
           // the k-th smallest communication known to this warp or to any warp of the block
           const u64 comm_limit = min(threshold.a, (u64)sh.block_comm_limit);
           // survivors that are below the threshold key, per triple as digit bits
