@@ -697,15 +697,18 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
       }
     }
     if (KIND == PS_REDUCE_PARETO && __any_sync(0xffffffffu, matters)) {
-      // About one unit in ten comes here (every unit with a survivor), so this part is
-      // written for few instructions and independent chains: the lane's triples stay in
-      // registers and are handled side by side, only the variants are a rolled loop.
+      // About one unit in ten comes here (every unit with a survivor).  Written as
+      // rolled loops over the lane's triples, whose values it first copies to arrays
+      // that can be indexed at run time, so that this part's registers do not weigh on
+      // the evaluation pass; only the digits of a point are tested side by side.
       u64 l_mem[R], l_comm[R], l_host[R];
+      u32 l_allowed[R], l_triple[R];
 #pragma unroll
       for (int r = 0; r < R; ++r) {
         l_mem[r] = FAST ? mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0))) : mem3[r];
         l_comm[r] = FAST ? mad_small(ub.x, kx[r], 0) : comm3[r];
         l_host[r] = (FAST && host_limited) ? mad_small(ub.sh, kh[r], 0) : host3[r];
+        l_allowed[r] = allowed[r]; l_triple[r] = t_local[r];
       }
       {
         // lane = a set of activation digits; which of them costs the least bytes
@@ -739,67 +742,55 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
         u64 bound[NM];
 #pragma unroll
         for (int d = 0; d < NM; ++d) bound[d] = tb.bound[d][vt];
-        // For a triple and variant the communication is the same for all NM activation
-        // digits, so of the surviving digits only the one with the least bytes (lowest
-        // digit on ties) can be on the frontier.  Digit d is a survivor if the triple's
-        // bytes are below the digit's bound and the flags allow the digit.
-        u64 m[R], c[R];
-        u32 idx[R];
-        bool cand[R];
-        bool some = false;
-#pragma unroll
+#pragma unroll 1
         for (int r = 0; r < R; ++r) {
+          // digit d of (triple, variant) is a survivor if the triple's bytes are below the
+          // digit's bound and the flags allow the digit
+          const u64 lm = l_mem[r];
           u32 fit = 0;
 #pragma unroll
-          for (int d = 0; d < NM; ++d) fit |= (l_mem[r] < bound[d]) ? (1u << d) : 0u;
+          for (int d = 0; d < NM; ++d) fit |= (lm < bound[d]) ? (1u << d) : 0u;
           // offloading activations adds host bytes: drop that digit if they do not fit
-          const u32 allow_vt = (!host_limited || l_host[r] < host_bound) ? allowed[r] : (allowed[r] & ~is_o);
+          const u32 allow_vt = (l_host[r] < host_bound) ? l_allowed[r] : (l_allowed[r] & ~is_o);
           const u32 pass = fit & allow_vt;
+          // For a triple and variant the communication is the same for all NM activation
+          // digits, so of the surviving digits only the one with the least bytes (lowest
+          // digit on ties) can be on the frontier.
           const bool has = pass != 0;
           const u32 d = has ? tb.least[vt][pass] : 0;
-          m[r] = l_mem[r] + tb.act[vt][d];
-          c[r] = l_comm[r] + c_axis;
-          idx[r] = vt_first + t_local[r] + d * N3;
-          // cheap tests: strictly dominated by a point already known to survive, or by
-          // the block's coarse staircase
-          const int bucket = stair_bucket(m[r]);
-          const u64 step = sh.stair[bucket > 0 ? bucket - 1 : 0];
-          cand[r] = has && !(dom_m <= m[r] && dom_c <= c[r] && (dom_m != m[r] || dom_c != c[r])) &&
-                    !(bucket > 0 && step <= c[r]);
-          some = some || cand[r];
-        }
-        if (!__any_sync(0xffffffffu, some)) continue;
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-          if (!__any_sync(0xffffffffu, cand[r])) continue;
-          bool offer = cand[r];
-          if (offer) {
+          const u64 m = lm + tb.act[vt][d];
+          const u64 c = l_comm[r] + c_axis;
+          const u32 idx = vt_first + l_triple[r] + d * N3;
+          // cheap tests first: strictly dominated by a point already known to survive,
+          // or by the block's coarse staircase
+          bool cand = has && !(dom_m <= m && dom_c <= c && (dom_m != m || dom_c != c));
+          if (cand) {
+            const int bucket = stair_bucket(m);
+            if (bucket > 0 && sh.stair[bucket - 1] <= c) cand = false;
+          }
+          if (!__any_sync(0xffffffffu, cand)) continue;
+          if (cand) {
             int lo = 0, hi = list.n;
             while (lo < hi) {               // entries with mem <= m
               const int mid = (lo + hi) >> 1;
-              if (list.a[mid] <= m[r]) lo = mid + 1; else hi = mid;
+              if (list.a[mid] <= m) lo = mid + 1; else hi = mid;
             }
             if (lo > 0) {
               const u64 em = list.a[lo - 1], ec = list.b[lo - 1];
-              if (ec < c[r] || (ec == c[r] && (em < m[r] || list.i[lo - 1] < idx[r]))) {
-                offer = false;
+              if (ec < c || (ec == c && (em < m || list.i[lo - 1] < idx))) {
+                cand = false;
                 dom_m = em; dom_c = ec;
               }
             }
           }
-          u32 pending = __ballot_sync(0xffffffffu, offer);
+          u32 pending = __ballot_sync(0xffffffffu, cand);
           while (pending) {
             const int src = __ffs(pending) - 1;
-            const u64 pm = __shfl_sync(0xffffffffu, m[r], src);
-            const u64 pc = __shfl_sync(0xffffffffu, c[r], src);
-            const u32 pi = __shfl_sync(0xffffffffu, idx[r], src);
+            const u64 pm = __shfl_sync(0xffffffffu, m, src);
+            const u64 pc = __shfl_sync(0xffffffffu, c, src);
+            const u32 pi = __shfl_sync(0xffffffffu, idx, src);
             pareto_insert(list, pm, pc, pi, lane, sh.stair);
-            // what the offered point strictly dominates need not be offered
-            if (lane == src || (pm <= m[r] && pc <= c[r] && (pm != m[r] || pc != c[r]))) {
-              if (offer && lane != src) { dom_m = pm; dom_c = pc; }
-              offer = false;
-            }
-            pending = __ballot_sync(0xffffffffu, offer);
+            pending &= pending - 1;
           }
         }
       }
@@ -826,32 +817,31 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
         const u32 vt_first = unit_first + vt * NC;
         // every point of (triple, variant): digit d is a survivor if the triple's
         // bytes are below the digit's bound and the flags allow the digit
-        bool some = false;
-#pragma unroll 1
-        for (int r = 0; r < R; ++r) {
-          u32 fit = 0;
-#pragma unroll 1
-          for (int d = 0; d < NM; ++d) fit |= (l_mem[r] < tb.bound[d][vt]) ? (1u << d) : 0u;
-          // offloading activations adds host bytes: drop that digit if they do not fit
-          const u32 allow_vt = (l_host[r] < host_bound) ? l_allowed[r] : (l_allowed[r] & ~is_o);
-          l_pass[r] = fit & allow_vt;
-          some = some || l_pass[r] != 0;
-        }
-        if (!__any_sync(0xffffffffu, some)) continue;
+        u64 bound[NM];
+#pragma unroll
+        for (int d = 0; d < NM; ++d) bound[d] = tb.bound[d][vt];
         {
           // the k-th smallest communication known to this warp or to any warp of the block
           const u64 comm_limit = min(threshold.a, (u64)sh.block_comm_limit);
-          // survivors that are below the threshold key, per triple as digit bits
+          // every point of (triple, variant): digit d is a survivor if the triple's bytes
+          // are below the digit's bound and the flags allow the digit; the survivors below
+          // the threshold key are candidates, per triple as digit bits
           u32 mine = 0;
 #pragma unroll 1
           for (int r = 0; r < R; ++r) {
+            const u64 lm = l_mem[r];
+            u32 fit = 0;
+#pragma unroll
+            for (int d = 0; d < NM; ++d) fit |= (lm < bound[d]) ? (1u << d) : 0u;
+            // offloading activations adds host bytes: drop that digit if they do not fit
+            const u32 allow_vt = (l_host[r] < host_bound) ? l_allowed[r] : (l_allowed[r] & ~is_o);
+            const u32 pass = fit & allow_vt;
             const u64 c = l_comm[r] + c_axis;
-            const u32 pass = l_pass[r];
             u32 cand = (c < threshold.a && c <= comm_limit) ? pass : 0u;
             if (c == threshold.a && pass != 0) {
 #pragma unroll 1
               for (int d = 0; d < NM; ++d) {
-                const Key key{c, l_mem[r] + tb.act[vt][d], vt_first + l_triple[r] + d * N3};
+                const Key key{c, lm + tb.act[vt][d], vt_first + l_triple[r] + d * N3};
                 if (((pass >> d) & 1u) && key_less(key, threshold)) cand |= 1u << d;
               }
             }
