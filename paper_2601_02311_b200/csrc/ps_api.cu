@@ -227,6 +227,7 @@ int ps_space_create(ps_ctx* ctx, const ps_space_desc* desc, ps_space** out) {
   sp->d_shapes = nullptr;
   sp->d_recs = nullptr;
   sp->d_facts = nullptr;
+  sp->d_order = nullptr;
   sp->n_values.assign(desc->n_values, desc->n_values + desc->n_n);
   // all (T, K) with T | N, K | N/T inside the enumeration limits: T ascending, then K
   for (u32 i = 0; i < desc->n_n; ++i) {
@@ -276,17 +277,47 @@ int ps_space_create(ps_ctx* ctx, const ps_space_desc* desc, ps_space** out) {
 
   bool ok = cudaMalloc(&sp->d_shapes, sizeof(ps_model_shape) * (size_t)desc->n_models) == cudaSuccess &&
             cudaMalloc(&sp->d_recs, sizeof(ModelRec) * (size_t)desc->n_models) == cudaSuccess &&
-            cudaMalloc(&sp->d_facts, sizeof(Fact) * sp->facts.size()) == cudaSuccess;
+            cudaMalloc(&sp->d_facts, sizeof(Fact) * sp->facts.size()) == cudaSuccess &&
+            cudaMalloc(&sp->d_order, sizeof(u32) * (size_t)desc->n_models) == cudaSuccess;
   ok = ok && cudaMemcpyAsync(sp->d_facts, sp->facts.data(), sizeof(Fact) * sp->facts.size(),
                              cudaMemcpyHostToDevice, ctx->stream) == cudaSuccess;
   if (!ok) { ps_space_destroy(sp); return PS_E_CUDA; }
   d.recs = sp->d_recs;
   d.facts = sp->d_facts;
+  d.order = sp->d_order;
   int rc = ps_space_set_models(sp, desc->models, desc->n_models);
   if (rc == PS_OK && cudaStreamSynchronize(ctx->stream) != cudaSuccess) rc = PS_E_CUDA;
   if (rc != PS_OK) { ps_space_destroy(sp); return rc; }
   *out = sp;
   return PS_OK;
+}
+
+// The order in which the sweeps' blocks take the models: most expected work first, so
+// that the blocks still running when the grid runs out are short ones.  A sweep block's
+// duration grows with the number of factorisations that pass the composition tests for
+// its model (T divides the heads, K divides the layers, T within the valid tensor
+// degree): only those have survivors under a filter that requires a valid composition,
+// and a unit with survivors costs several times one without.  The count is a sum over
+// the distinct (T, K) pairs of the space, weighted by how many device counts have them.
+static void sweep_order(ps_space* sp, const ps_model_shape* models, u32 n_models) {
+  std::vector<std::pair<u32, std::vector<std::pair<u32, u32>>>> by_t;   // T -> (K, number of factorisations)
+  for (const Fact& f : sp->facts) {
+    if (f.T > sp->dev.tp_max_valid) continue;
+    auto t = std::find_if(by_t.begin(), by_t.end(), [&](const auto& e) { return e.first == f.T; });
+    if (t == by_t.end()) { by_t.push_back({f.T, {}}); t = by_t.end() - 1; }
+    auto k = std::find_if(t->second.begin(), t->second.end(), [&](const auto& e) { return e.first == f.K; });
+    if (k == t->second.end()) t->second.push_back({f.K, 1u}); else ++k->second;
+  }
+  std::vector<u32> work(n_models, 0);
+  for (u32 i = 0; i < n_models; ++i)
+    for (const auto& t : by_t) {
+      if (models[i].heads % t.first) continue;
+      for (const auto& k : t.second)
+        if (models[i].layers % k.first == 0) work[i] += k.second;
+    }
+  sp->order.resize(n_models);
+  for (u32 i = 0; i < n_models; ++i) sp->order[i] = i;
+  std::stable_sort(sp->order.begin(), sp->order.end(), [&](u32 a, u32 b) { return work[a] > work[b]; });
 }
 
 int ps_space_set_models(ps_space* sp, const ps_model_shape* models, uint32_t n_models) {
@@ -298,9 +329,12 @@ int ps_space_set_models(ps_space* sp, const ps_model_shape* models, uint32_t n_m
     if (!shape_is_small(models[i], sp->dev.accum)) all_small = 0;
   }
   sp->dev.all_small = all_small;
+  sweep_order(sp, models, n_models);
   ps_ctx* ctx = sp->ctx;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return PS_E_CUDA;
+  CUDA_OK(cudaMemcpyAsync(sp->d_order, sp->order.data(), sizeof(u32) * (size_t)n_models, cudaMemcpyHostToDevice,
+                          ctx->stream));
   CUDA_OK(cudaMemcpyAsync(sp->d_shapes, models, sizeof(ps_model_shape) * (size_t)n_models,
                           cudaMemcpyHostToDevice, ctx->stream));
   CUDA_OK(launch_model_derive(sp->d_shapes, sp->d_recs, n_models, ctx->d_status, ctx->stream));
@@ -323,6 +357,7 @@ void ps_space_destroy(ps_space* sp) {
   if (sp->d_shapes) cudaFree(sp->d_shapes);
   if (sp->d_recs) cudaFree(sp->d_recs);
   if (sp->d_facts) cudaFree(sp->d_facts);
+  if (sp->d_order) cudaFree(sp->d_order);
   delete sp;
 }
 

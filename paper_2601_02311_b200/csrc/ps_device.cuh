@@ -34,6 +34,7 @@ struct __align__(16) Fact {
 struct SpaceDev {
   const ModelRec* recs;
   const Fact* facts;
+  const u32* order;   // the models in the order in which the sweeps' blocks take them (most work first)
   u64 ppm;            // points per model = n_facts * nvt * n_codes
   u32 n_models;
   u32 n_facts;        // factorisations of all N together ("units" per model)

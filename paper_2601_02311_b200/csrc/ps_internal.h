@@ -28,6 +28,8 @@ struct ps_space {
   ps_model_shape* d_shapes;
   ModelRec* d_recs;
   Fact* d_facts;
+  u32* d_order;                   // see SpaceDev::order
+  std::vector<u32> order;
   SpaceDev dev;
 };
 

@@ -335,7 +335,8 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
   extern __shared__ __align__(16) unsigned char smem_raw[];
   SweepShared<WARPS>& sh = *reinterpret_cast<SweepShared<WARPS>*>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const u32 model = blockIdx.y, chunk = blockIdx.x, n_chunks = gridDim.x;
+  // blocks are handed out in grid order: the models with the most expected work first
+  const u32 model = sp.order[blockIdx.y], chunk = blockIdx.x, n_chunks = gridDim.x;
 
   // stage the model record with 16-byte loads (6 x 16 B)
   if (tid < (int)(sizeof(ModelRec) / 16))
