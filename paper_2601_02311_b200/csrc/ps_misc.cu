@@ -77,26 +77,86 @@ __global__ void k_check_point(const ModelRec* rec, Fact f, u32 v, u32 tau, u32 c
   *out = e;
 }
 
+// Division of a device count by a small tensor degree t without dividing: with
+// magic[t] = ceil(2^32 / t) the high word of n * magic[t] is floor(n / t) whenever
+// n * t < 2^32 (the error of the magic, below t / 2^32 per unit of n, then stays
+// below 1 / t).  Filled on the host for t <= SELECT_MAGIC_MAX; device counts up to
+// 2^24 qualify.
+constexpr u32 SELECT_MAGIC_MAX = 64;
+struct SelectMagic {
+  u32 m[SELECT_MAGIC_MAX + 1];
+  double inv[SELECT_MAGIC_MAX + 1];   // 1 / t, correctly rounded
+};
+
+// floor(a / d) from a reciprocal of d that is correct to the last bit: for a < 2^52
+// the product is off by less than one, so its integer part is the quotient or a
+// neighbour of it, and the remainder says which.  One code path for every lane.
+__device__ __forceinline__ u64 div_by_reciprocal(u64 a, u32 d, double recip) {
+  if (a >= ((u64)1 << 52)) return a / d;
+  u64 q = (u64)__double2ll_rz((double)(long long)a * recip);
+  const long long rem = (long long)(a - q * d);
+  if (rem < 0) --q;
+  else if (rem >= (long long)d) ++q;
+  return q;
+}
+
+// the largest t <= tp_degree that divides n
+__device__ __forceinline__ u32 largest_tensor_degree(u32 n, u32 tp_degree, const SelectMagic& magic) {
+  const u32 top = min(tp_degree, n);
+  if (tp_degree <= SELECT_MAGIC_MAX && n <= (1u << 24)) {
+    u32 best = 1;
+    for (u32 t = 2; t <= tp_degree; ++t) {               // the same trip count for every lane
+      const u32 q = __umulhi(n, magic.m[t]);
+      if (q * t == n && t <= top) best = t;
+    }
+    return best;
+  }
+  for (u32 t = top; t > 1; --t)
+    if (n % t == 0) return t;
+  return 1;
+}
+
+// 128-bit unsigned integers as four 32-bit limbs, for products of a 64-bit count
+// with one or two factors of at most 32 bits (a generic 128 x 128 multiplication
+// costs several times more).
+struct Wide {
+  u32 w[4];
+};
+__device__ __forceinline__ Wide wide_mul(u64 a, u32 k) {
+  const u64 p0 = (u64)(u32)a * k;
+  const u64 p1 = (u64)(u32)(a >> 32) * k + (p0 >> 32);
+  return Wide{{(u32)p0, (u32)p1, (u32)(p1 >> 32), 0u}};
+}
+__device__ __forceinline__ Wide wide_mul(const Wide& a, u32 k) {      // a below 2^96
+  const u64 q0 = (u64)a.w[0] * k;
+  const u64 q1 = (u64)a.w[1] * k + (q0 >> 32);
+  const u64 q2 = (u64)a.w[2] * k + (q1 >> 32);
+  return Wide{{(u32)q0, (u32)q1, (u32)q2, (u32)(q2 >> 32)}};
+}
+__device__ __forceinline__ bool wide_less(const Wide& a, const Wide& b) {
+  const u64 ah = ((u64)a.w[3] << 32) | a.w[2], al = ((u64)a.w[1] << 32) | a.w[0];
+  const u64 bh = ((u64)b.w[3] << 32) | b.w[2], bl = ((u64)b.w[1] << 32) | b.w[0];
+  return ah < bh || (ah == bh && al < bl);
+}
+
 // Algorithm 1 for one query.  Thresholds are rationals; the comparisons are
 // carried out exactly in 128-bit integers.
 __device__ __forceinline__ ps_select_result select_one(const ps_select_query& s, u32 head_num,
                                                        u32 head_den, u32 layer_num, u32 layer_den,
-                                                       u32 tp_degree) {
-  typedef unsigned __int128 u128;
+                                                       u32 tp_degree, const SelectMagic& magic) {
   const u32 wsum = (u32)s.w_param + s.w_grad + s.w_opt;
-  const u128 m_model = (u128)wsum * s.param_elems;
-  const u128 budget = (u128)head_num * s.device_bytes;        // headroom * M_d, times head_den
+  const Wide m_model = wide_mul(wide_mul(s.param_elems, wsum), head_den);     // M_model * head_den
+  const Wide budget = wide_mul(s.device_bytes, head_num);                      // headroom * M_d, times head_den
   u32 branch, T = 1, code = 32;                                // ZeRO-3 unless data parallel fits
-  if (m_model * head_den < budget) {
+  if (wide_less(m_model, budget)) {
     branch = 0; code = 0;
-  } else if (m_model * head_den < budget * s.n_devices) {
+  } else if (wide_less(m_model, wide_mul(budget, s.n_devices))) {
     branch = 1;
   } else {
-    const u128 layer = (u128)wsum * s.layer_elems;
-    if (s.fast_interconnect && layer * layer_den > (u128)layer_num * s.device_bytes) {
+    const Wide layer = wide_mul(wide_mul(s.layer_elems, wsum), layer_den);
+    if (s.fast_interconnect && wide_less(wide_mul(s.device_bytes, layer_num), layer)) {
       branch = 2;
-      for (u32 t = min(tp_degree, s.n_devices); t >= 1; --t)
-        if (s.n_devices % t == 0) { T = t; break; }
+      T = largest_tensor_degree(s.n_devices, tp_degree, magic);
     } else {
       branch = 3;
     }
@@ -108,9 +168,22 @@ __device__ __forceinline__ ps_select_result select_one(const ps_select_query& s,
   //   ZeRO-3 (S*,S,S,R):               bytes (w_T + w_O + w_G) ceil(E / D) + w_T ceil(unit / T),
   //                                    volume x w_G + 2 x w_T
   // where x = E - floor(E / D) is the ring volume in elements (Section 2.3).
-  const u32 D = s.n_devices / T;
-  const u64 E = div_ceil(s.param_elems, T);
-  const u64 quot = div_floor(E, D);
+  // T is 1 or a small divisor of the device count: the divisions by it use the
+  // host's tables where they reach (one path for all lanes of a warp)
+  u32 D = s.n_devices;
+  u64 E = s.param_elems, unit_t = s.layer_elems;
+  if (T > 1) {
+    if (T <= SELECT_MAGIC_MAX && s.n_devices <= (1u << 24)) {
+      D = __umulhi(s.n_devices, magic.m[T]);
+      E = div_by_reciprocal(s.param_elems + (T - 1), T, magic.inv[T]);
+      unit_t = div_by_reciprocal(s.layer_elems + (T - 1), T, magic.inv[T]);
+    } else {
+      D = s.n_devices / T;
+      E = div_ceil(s.param_elems, T);
+      unit_t = div_ceil(s.layer_elems, T);
+    }
+  }
+  const u64 quot = div_by_reciprocal(E, D, __drcp_rn((double)D));
   const u64 x = E - quot;
   u64 mem, comm;
   if (code == 0) {
@@ -118,7 +191,7 @@ __device__ __forceinline__ ps_select_result select_one(const ps_select_query& s,
     comm = 2 * x * s.w_grad;
   } else {
     const u64 shard = quot + ((quot * D != E) ? 1 : 0);
-    mem = (u64)wsum * shard + (u64)s.w_param * div_ceil(s.layer_elems, T);
+    mem = (u64)wsum * shard + (u64)s.w_param * unit_t;
     comm = x * s.w_grad + 2 * x * s.w_param;
   }
   ps_select_result o;
@@ -127,37 +200,46 @@ __device__ __forceinline__ ps_select_result select_one(const ps_select_query& s,
   return o;
 }
 
-// Two queries per thread, SELECT_THREADS apart, so that four 16-byte loads are in
-// flight per thread before any arithmetic: the kernel streams 64 bytes per query.
-constexpr int SELECT_THREADS = 256;
-__global__ void __launch_bounds__(SELECT_THREADS) k_select(const ps_select_query* __restrict__ q, u64 n,
+// SELECT_PER_THREAD queries per thread, SELECT_THREADS apart, all of their 16-byte
+// loads in flight before any arithmetic: the kernel streams 64 bytes per query, read
+// once and written once (streaming loads and stores, nothing is reused).
+#ifndef SELECT_THREADS_PER_BLOCK
+#define SELECT_THREADS_PER_BLOCK 128
+#endif
+#ifndef SELECT_QUERIES_PER_THREAD
+#define SELECT_QUERIES_PER_THREAD 2
+#endif
+// resident blocks per SM the kernel is compiled for: 12 x 128 threads caps it at 40
+// registers, and a kernel that streams needs the warps more than the registers
+#ifndef SELECT_MIN_BLOCKS
+#define SELECT_MIN_BLOCKS 12
+#endif
+constexpr int SELECT_THREADS = SELECT_THREADS_PER_BLOCK;
+constexpr int SELECT_PER_THREAD = SELECT_QUERIES_PER_THREAD;
+__global__ void __launch_bounds__(SELECT_THREADS, SELECT_MIN_BLOCKS) k_select(const ps_select_query* __restrict__ q, u64 n,
                                                            u32 head_num, u32 head_den, u32 layer_num,
-                                                           u32 layer_den, u32 tp_degree,
+                                                           u32 layer_den, u32 tp_degree, SelectMagic magic,
                                                            ps_select_result* __restrict__ out) {
-  const u64 i0 = (u64)blockIdx.x * (2 * SELECT_THREADS) + threadIdx.x;
-  const u64 i1 = i0 + SELECT_THREADS;
-  ps_select_query s0, s1;
-  if (i0 < n) {
-    const uint4* src = reinterpret_cast<const uint4*>(q + i0);
-    uint4* dst = reinterpret_cast<uint4*>(&s0);
-    dst[0] = __ldg(src); dst[1] = __ldg(src + 1);
+  const u64 first = (u64)blockIdx.x * (SELECT_PER_THREAD * SELECT_THREADS) + threadIdx.x;
+  ps_select_query s[SELECT_PER_THREAD];
+#pragma unroll
+  for (int j = 0; j < SELECT_PER_THREAD; ++j) {
+    const u64 i = first + (u64)j * SELECT_THREADS;
+    if (i < n) {
+      const uint4* src = reinterpret_cast<const uint4*>(q + i);
+      uint4* dst = reinterpret_cast<uint4*>(&s[j]);
+      dst[0] = __ldcs(src); dst[1] = __ldcs(src + 1);
+    }
   }
-  if (i1 < n) {
-    const uint4* src = reinterpret_cast<const uint4*>(q + i1);
-    uint4* dst = reinterpret_cast<uint4*>(&s1);
-    dst[0] = __ldg(src); dst[1] = __ldg(src + 1);
-  }
-  if (i0 < n) {
-    const ps_select_result o = select_one(s0, head_num, head_den, layer_num, layer_den, tp_degree);
-    uint4* dst = reinterpret_cast<uint4*>(out + i0);
-    const uint4* src = reinterpret_cast<const uint4*>(&o);
-    dst[0] = src[0]; dst[1] = src[1];
-  }
-  if (i1 < n) {
-    const ps_select_result o = select_one(s1, head_num, head_den, layer_num, layer_den, tp_degree);
-    uint4* dst = reinterpret_cast<uint4*>(out + i1);
-    const uint4* src = reinterpret_cast<const uint4*>(&o);
-    dst[0] = src[0]; dst[1] = src[1];
+#pragma unroll
+  for (int j = 0; j < SELECT_PER_THREAD; ++j) {
+    const u64 i = first + (u64)j * SELECT_THREADS;
+    if (i < n) {
+      const ps_select_result o = select_one(s[j], head_num, head_den, layer_num, layer_den, tp_degree, magic);
+      uint4* dst = reinterpret_cast<uint4*>(out + i);
+      const uint4* src = reinterpret_cast<const uint4*>(&o);
+      __stcs(dst, src[0]); __stcs(dst + 1, src[1]);
+    }
   }
 }
 
@@ -165,7 +247,8 @@ __global__ void __launch_bounds__(SELECT_THREADS) k_select(const ps_select_query
 // the model's frontier (one thread per model).
 __global__ void __launch_bounds__(128) k_select_compare(SpaceDev sp, u32 unit_begin, u32 unit_end, u32 N,
                                                         u64 device_bytes, u32 fast, u32 head_num, u32 head_den,
-                                                        u32 layer_num, u32 layer_den, u32 tp_degree, u64 host_cap,
+                                                        u32 layer_num, u32 layer_den, u32 tp_degree,
+                                                        SelectMagic magic, u64 host_cap,
                                                         u32 require_flags, u32 comm_kind,
                                                         const ps_front_entry* __restrict__ frontier,
                                                         const u32* __restrict__ counts, u32 n_caps, u32 cap_index,
@@ -177,7 +260,7 @@ __global__ void __launch_bounds__(128) k_select_compare(SpaceDev sp, u32 unit_be
   q.param_elems = rec.P; q.layer_elems = rec.unit; q.device_bytes = device_bytes; q.n_devices = N;
   q.w_param = (uint8_t)rec.wT; q.w_grad = (uint8_t)rec.wG; q.w_opt = (uint8_t)rec.wO;
   q.fast_interconnect = (uint8_t)(fast ? 1 : 0);
-  const ps_select_result pick = select_one(q, head_num, head_den, layer_num, layer_den, tp_degree);
+  const ps_select_result pick = select_one(q, head_num, head_den, layer_num, layer_den, tp_degree, magic);
   ps_select_compare_result r;
   r.branch = pick.branch; r.T = pick.T; r.code_dp = pick.code_dp; r.pad = 0;
   u32 status = 0;
@@ -266,11 +349,22 @@ cudaError_t launch_check_point(const ModelRec* d_rec, Fact f, u32 v, u32 tau, u3
   return cudaGetLastError();
 }
 
+static SelectMagic select_magic() {
+  SelectMagic g;
+  g.m[0] = g.m[1] = 0;
+  g.inv[0] = g.inv[1] = 1.0;
+  for (u32 t = 2; t <= SELECT_MAGIC_MAX; ++t) {
+    g.m[t] = (u32)((((u64)1 << 32) + t - 1) / t);
+    g.inv[t] = 1.0 / (double)t;
+  }
+  return g;
+}
+
 cudaError_t launch_select(const ps_select_query* d_q, u64 n, u32 head_num, u32 head_den, u32 layer_num,
                           u32 layer_den, u32 tp_degree, ps_select_result* d_out, cudaStream_t stream) {
-  const u64 per_block = 2 * SELECT_THREADS;
+  const u64 per_block = (u64)SELECT_PER_THREAD * SELECT_THREADS;
   k_select<<<(unsigned)((n + per_block - 1) / per_block), SELECT_THREADS, 0, stream>>>(
-      d_q, n, head_num, head_den, layer_num, layer_den, tp_degree, d_out);
+      d_q, n, head_num, head_den, layer_num, layer_den, tp_degree, select_magic(), d_out);
   return cudaGetLastError();
 }
 
@@ -285,7 +379,8 @@ cudaError_t launch_select_compare(const SpaceDev& sp, u32 unit_begin, u32 unit_e
                                   const u32* d_counts, u32 n_caps, u32 cap_index, u32 max_entries,
                                   ps_select_compare_result* d_out, cudaStream_t stream) {
   k_select_compare<<<(sp.n_models + 127) / 128, 128, 0, stream>>>(
-      sp, unit_begin, unit_end, N, device_bytes, fast, head_num, head_den, layer_num, layer_den, tp_degree, host_cap,
+      sp, unit_begin, unit_end, N, device_bytes, fast, head_num, head_den, layer_num, layer_den, tp_degree,
+      select_magic(), host_cap,
       require_flags, comm_kind, d_frontier, d_counts, n_caps, cap_index, max_entries, d_out);
   return cudaGetLastError();
 }
