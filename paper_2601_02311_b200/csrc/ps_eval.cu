@@ -40,6 +40,9 @@ namespace {
 // many short blocks the stores of neighbouring groups are in flight together
 // (every point surviving: 0.56 of the copy bandwidth with 4 blocks per SM, 0.62
 // with 32).
+#ifndef EVAL_BULK_EVICT_FIRST
+#define EVAL_BULK_EVICT_FIRST 1
+#endif
 #ifndef EVAL_GRID_PER_SM_MATERIALISE
 #define EVAL_GRID_PER_SM_MATERIALISE 64
 #endif
@@ -133,9 +136,20 @@ __device__ __forceinline__ void warp_bulk_store(T* __restrict__ dst, const T* bu
   const int tail = n - head - body;
   if (lane < tail) dst[head + body + lane] = buf[skew + head + body + lane];
   if (lane == 0 && body > 0) {
+#if EVAL_BULK_EVICT_FIRST
+    // The output is written once and not read back by this kernel: with the evict-first
+    // policy the lines leave the L2 as whole lines.  (Without a policy the same stores
+    // cost 12 % more DRAM write traffic than the bytes stored.)
+    unsigned long long policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
+                 ::"l"(dst + head), "r"(smem_addr(buf + skew + head)), "r"(body * (int)sizeof(T)), "l"(policy)
+                 : "memory");
+#else
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                  ::"l"(dst + head), "r"(smem_addr(buf + skew + head)), "r"(body * (int)sizeof(T))
                  : "memory");
+#endif
   }
   if (lane == 0) asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
@@ -409,6 +423,7 @@ __global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
 // digits the required flags allow for its triple (fixed for the whole kernel).
 struct CountTables {
   u64 bound[5][4];       // [digit][variant]
+  __align__(16) double bound_f64[5][4];   // the same as doubles (exact below 2^53), 0 for variants the space lacks
   u64 host_bound[4];     // the triple's own host bytes must stay below this to offload activations
 };
 
@@ -466,6 +481,7 @@ __global__ void __launch_bounds__(THREADS, 2) k_compact_count(SpaceDev sp, EvalA
   ModelRec rec;
   u32 ka[R], kb[R], kc[R], kh[R];
   u64 mem3[R], host3[R];
+  bool small = false;                      // the factorisation's byte counts are exact as doubles
   u32 allowed[R];
   u64 run_total = 0;
   u32 with_survivors = 0;                  // bit j: group seg_begin + j has survivors
@@ -480,8 +496,8 @@ __global__ void __launch_bounds__(THREADS, 2) k_compact_count(SpaceDev sp, EvalA
     unit = gl / sp.nvt;
     vt = gl - unit * sp.nvt;
   }
-  for (u32 seg = seg_begin; seg < seg_end; ++seg) {
-    const u64 g = a.first_group + seg;
+  for (u32 seg = seg_begin; seg < seg_end;) {
+    const u64 g0 = a.first_group + seg;
     if (model != model_cur) {
       model_cur = model;
       unit_cur = 0xffffffffu;
@@ -519,11 +535,16 @@ __global__ void __launch_bounds__(THREADS, 2) k_compact_count(SpaceDev sp, EvalA
         const ActBase ab = POW2 ? act_base_pow2_one_copy(rec, p2, tl_v, tl_tau)
                            : p2.all ? act_base_pow2(rec, p2, tl_v, tl_tau) : act_base(rec, f, tl_v, tl_tau, ub.G);
         const u64 am = mu_elems(tl_mode, ab.EA, ab.shA, ab.uA, sp.sstar_units);
-        tb.bound[tl_d][tl_vt] = am < cap_x ? cap_x - am : 0;
+        const u64 bound = am < cap_x ? cap_x - am : 0;
+        tb.bound[tl_d][tl_vt] = bound;
+        tb.bound_f64[tl_d][tl_vt] = (double)bound;
         if (tl_d == 0) {
           const u64 ah = 2 * ab.EA * sp.accum;  // offloaded after forward, reloaded for backward, per micro-batch
           tb.host_bound[tl_vt] = ah < host_x ? host_x - ah : 0;
         }
+      } else if (tl_vt < 4) {
+        tb.bound_f64[tl_d][tl_vt] = 0.0;
+        if (tl_d == 0) tb.host_bound[tl_vt] = 0;
       }
       __syncwarp();
       const bool unit_ok = (ub.cv & req_cv) == req_cv;
@@ -534,50 +555,79 @@ __global__ void __launch_bounds__(THREADS, 2) k_compact_count(SpaceDev sp, EvalA
         host3[r] = mad_small(ub.sh, kh[r], 0);
         allowed[r] = (unit_ok && host3[r] < host_x) ? ((t_allowed[r] >> shift) & all) : 0;
       }
+      // Integers below 2^53 are exact as doubles: when the capacity and every triple's bytes
+      // are that small (one test for the warp), whole factorisations are counted with
+      // compares on the fp64 pipe and predicated fp32 adds (see below).
+      small = cap_x < ((u64)1 << 53) && (u64)(rec.wT + rec.wO + rec.wG) * (ub.E2 + 2 * ub.u) < ((u64)1 << 53);
     }
-    // the group's codes inside the window
-    const u64 group_first = g * NC;
-    const u32 code_lo = a.first > group_first ? (u32)(a.first - group_first) : 0u;
-    const u32 code_hi = window_end < group_first + NC ? (u32)(window_end - group_first) : (u32)NC;
-    const bool whole = code_lo == 0 && code_hi == (u32)NC;
-    const u64 host_bound = tb.host_bound[vt];
-    u32 n = 0;
-    if (whole) {
-      // the usual case: per point one compare, masked by the digit's bit
+    // the factorisation's groups inside this run: variants vt .. vt + n_here - 1
+    const u32 n_here = min(sp.nvt - vt, seg_end - seg);
+    u32 cnt[4] = {0, 0, 0, 0};             // this lane's survivors per variant
+    if (small && g0 * NC >= a.first && (g0 + n_here) * NC <= window_end) {
+      // The usual case, every group whole inside the window: all variants at once.  A
+      // triple's digit is tested for the four variants with one mask bit; a point costs a
+      // compare on the fp64 pipe and a predicated fp32 add.
+      float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
       for (int d = 0; d < NM; ++d) {
-        const u64 bound = tb.bound[d][vt];
+        double bound[4];
+        {
+          const double2 b01 = *reinterpret_cast<const double2*>(&tb.bound_f64[d][0]);
+          const double2 b23 = *reinterpret_cast<const double2*>(&tb.bound_f64[d][2]);
+          bound[0] = b01.x; bound[1] = b01.y; bound[2] = b23.x; bound[3] = b23.y;
+        }
         const bool offload = (is_o >> d) & 1u;
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-          const bool pass = mem3[r] < bound && (!offload || host3[r] < host_bound);
-          n += pass ? ((allowed[r] >> d) & 1u) : 0u;
+          const bool on = (allowed[r] >> d) & 1u;
+          const double m = (double)mem3[r];
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (on && m < bound[j] && (!offload || host3[r] < tb.host_bound[j])) c[j] += 1.0f;
         }
       }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) cnt[j] = (u32)c[j];
     } else {
-      // a group at the window's edge: only the codes inside it
 #pragma unroll 1
-      for (int d = 0; d < NM; ++d) {
-        const u64 bound = tb.bound[d][vt];
-        const bool offload = (is_o >> d) & 1u;
+      for (u32 k = 0; k < n_here; ++k) {
+        // a group at the window's edge (or byte counts beyond 2^53): only the codes inside the window
+        const u64 group_first = (g0 + k) * NC;
+        const u32 code_lo = a.first > group_first ? (u32)(a.first - group_first) : 0u;
+        const u32 code_hi = window_end < group_first + NC ? (u32)(window_end - group_first) : (u32)NC;
+        const u64 host_bound = tb.host_bound[vt + k];
+        u32 n = 0;
+#pragma unroll 1
+        for (int d = 0; d < NM; ++d) {
+          const u64 bound = tb.bound[d][vt + k];
+          const bool offload = (is_o >> d) & 1u;
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-          const u32 code = lane + 32 * r + d * N3;
-          const bool pass = ((allowed[r] >> d) & 1u) && mem3[r] < bound && (!offload || host3[r] < host_bound) &&
-                            code >= code_lo && code < code_hi;
-          n += pass ? 1u : 0u;
+          for (int r = 0; r < R; ++r) {
+            const u32 code = lane + 32 * r + d * N3;
+            const bool pass = ((allowed[r] >> d) & 1u) && mem3[r] < bound && (!offload || host3[r] < host_bound) &&
+                              code >= code_lo && code < code_hi;
+            n += pass ? 1u : 0u;
+          }
         }
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if ((u32)j == vt + k) cnt[j] = n;
       }
     }
-    n = __reduce_add_sync(0xffffffffu, n);
-    if (lane == 0) a.tile_count[seg] = n;
-    run_total += n;
-    if (n) with_survivors |= 1u << (seg - seg_begin);
-    // the next group: next variant, else next factorisation, else next model
-    if (++vt == sp.nvt) {
-      vt = 0;
-      if (++unit == sp.n_facts) { unit = 0; ++model; }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if ((u32)j >= vt && (u32)j < vt + n_here) {              // (the same for every lane)
+        const u32 n = __reduce_add_sync(0xffffffffu, cnt[j]);
+        const u32 at = seg + ((u32)j - vt);
+        if (lane == 0) a.tile_count[at] = n;
+        run_total += n;
+        if (n) with_survivors |= 1u << (at - seg_begin);
+      }
     }
+    // the next factorisation, else the next model
+    seg += n_here;
+    vt = 0;
+    if (++unit == sp.n_facts) { unit = 0; ++model; }
   }
   if (lane == 0) a.tile_offset[run] = run_total;
   // the groups with survivors join the write pass's list (in any order: a group's place
