@@ -507,7 +507,7 @@ def run_ours(args):
         hbm_peak = peaks.get("hbm_gbs", 6650.0)
         hbm_src = "measured" if "hbm_gbs" in peaks else "fallback"
         ncu = ncu_counters()
-        on_captured_workload = args.workload == "C4" and args.models is None and ncu is not None
+        captured = ncu["workloads"].get(args.workload) if (ncu is not None and args.models is None) else None
         ncu_commit = ncu["captured_at_commit"] if ncu else None
 
         def alu_roofline(kernel_key, label, ms):
@@ -517,7 +517,7 @@ def run_ours(args):
             utilisation (integer and logic instructions only) -- the figure to hold against
             an integer-ALU target.  Both come from the capture named in `counters_commit`
             and are given on the workload of that capture only."""
-            k = ncu["kernels"][kernel_key] if on_captured_workload else None
+            k = captured["kernels"].get(kernel_key) if captured else None
             ops = k["thread_instr_per_point"] if k else None
             achieved = ops * size / (ms * 1e-3) / 1e12 if k else None
             return {"bound": "alu", "kernel": label, "achieved": achieved, "peak": int_peak / 1e12,
@@ -559,9 +559,10 @@ def run_ours(args):
             "roofline_topk": alu_roofline("k_sweep_topk", "k_sweep<top-k> (+ merge)", phase_ms["topk"]),
             "roofline_hbm": {"bound": "hbm", "kernel": "k_eval<materialise>", "achieved": mat_gbs,
                              "peak": hbm_peak, "unit": "GB/s", "frac": mat_gbs / hbm_peak,
-                             "traffic": (int(ncu["kernels"]["k_eval_materialise"]["dram_bytes_per_point"] * count)
-                                         if on_captured_workload else None),
-                             "counters_commit": ncu_commit if on_captured_workload else None,
+                             "traffic": (int(captured["kernels"]["k_eval_materialise"]["dram_bytes_per_point"] * count)
+                                         if captured and "k_eval_materialise" in captured["kernels"] else None),
+                             "counters_commit": (ncu_commit if captured and "k_eval_materialise" in captured["kernels"]
+                                                 else None),
                              "peak_source": hbm_src + " (of measured)" if hbm_src == "measured" else hbm_src + " (of fallback)"},
         }
         dense_gbs = (BYTES_PER_POINT_MATERIALISE + 8) * dense_survivors / (dense_ms * 1e-3) / 1e9

@@ -672,9 +672,28 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
     }
     // ---- reduction pass, only if some survivor of this warp can matter
     bool matters = false;
+    u32 alive = 0;                         // Pareto: the lane's triples that may still add to the frontier
     if (KIND == PS_REDUCE_PARETO) {
+      // A triple with survivors matters unless every point of it is beaten already: its own
+      // bytes and its volume plus the least axis traffic bound its points from below, and a
+      // point known to survive (the cached one, or the block's coarse staircase) that beats
+      // the bounds strictly beats them all.
+      bool some = false;
 #pragma unroll
-      for (int r = 0; r < R; ++r) matters = matters || n_pass[r] != 0;
+      for (int r = 0; r < R; ++r) some = some || n_pass[r] != 0;
+      if (some) {
+        const u64 least_axis = tb.c_axis[0];   // tau = 0 sends the smaller boundary tensor; v does not matter
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          const u64 m_lb = FAST ? mad_small(ub.E2, ka[r], mad_small(ub.sh, kb[r], mad_small(ub.u, kc[r], 0))) : mem3[r];
+          const u64 c_lb = (FAST ? mad_small(ub.x, kx[r], 0) : comm3[r]) + least_axis;
+          const int bucket = stair_bucket(m_lb);
+          const bool beaten = (dom_m <= m_lb && dom_c <= c_lb && (dom_m != m_lb || dom_c != c_lb)) ||
+                              (bucket > 0 && sh.stair[bucket - 1] <= c_lb);
+          if (n_pass[r] != 0 && !beaten) alive |= 1u << r;
+        }
+      }
+      matters = alive != 0;
     } else {
       const u64 comm_limit = min(threshold.a, (u64)sh.block_comm_limit);
       const u64 least_axis = tb.c_axis[0];   // tau = 0 sends the smaller boundary tensor; v does not matter
@@ -730,6 +749,10 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
         for (int vt = 0; vt < 4; ++vt) tb.least[vt][lane] = (unsigned char)which[vt];
       }
       __syncwarp();
+      // rounds of triples in which some lane's triple is still alive
+      u32 rounds = 0;
+#pragma unroll
+      for (int r = 0; r < R; ++r) rounds |= __any_sync(0xffffffffu, (alive >> r) & 1u) ? (1u << r) : 0u;
 
       // Variants in an order in which later ones seldom beat earlier ones (the result
       // does not depend on the order, the work does): the tensor axis that shards
@@ -745,6 +768,7 @@ __global__ void __launch_bounds__(WARPS * 32, MIN_BLOCKS) k_sweep(SpaceDev sp, S
         for (int d = 0; d < NM; ++d) bound[d] = tb.bound[d][vt];
 #pragma unroll 1
         for (int r = 0; r < R; ++r) {
+          if (!((rounds >> r) & 1u)) continue;
           // digit d of (triple, variant) is a survivor if the triple's bytes are below the
           // digit's bound and the flags allow the digit
           const u64 lm = l_mem[r];
