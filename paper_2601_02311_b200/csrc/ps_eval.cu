@@ -31,26 +31,26 @@
 
 namespace {
 
-// Launch shapes (blocks per SM; two are resident at a time).  Materialise is
+// Launch shapes (blocks of four warps per SM; four are resident at a time).  Materialise is
 // fastest with about one group per warp: short-lived blocks keep the warps of an
 // SM at different stages (set-up, staging, draining stores) and the running
 // warps write neighbouring stretches of every output array.  The count pass
 // prefers long runs of groups per warp (what a model and a factorisation fix is
 // then computed once).  The write pass takes the listed groups round-robin; with
 // many short blocks the stores of neighbouring groups are in flight together
-// (every point surviving: 0.56 of the copy bandwidth with 4 blocks per SM, 0.62
-// with 32).
+// (every point surviving: 0.56 of the copy bandwidth with 32 warps in the grid per
+// SM, 0.62 with 256).
 #ifndef EVAL_BULK_EVICT_FIRST
 #define EVAL_BULK_EVICT_FIRST 1
 #endif
 #ifndef EVAL_GRID_PER_SM_MATERIALISE
-#define EVAL_GRID_PER_SM_MATERIALISE 64
+#define EVAL_GRID_PER_SM_MATERIALISE 128
 #endif
 #ifndef EVAL_GRID_PER_SM_COMPACT
 #define EVAL_GRID_PER_SM_COMPACT 2
 #endif
 #ifndef EVAL_GRID_PER_SM_WRITE
-#define EVAL_GRID_PER_SM_WRITE 32
+#define EVAL_GRID_PER_SM_WRITE 64
 #endif
 constexpr int THREADS = EVAL_THREADS;
 constexpr int WARPS = THREADS / 32;
@@ -156,7 +156,7 @@ __device__ __forceinline__ void warp_bulk_store(T* __restrict__ dst, const T* bu
 
 // POW2: every degree of the space is a power of two (no division is compiled in)
 template <int MODE, int NM, bool POW2>
-__global__ void __launch_bounds__(THREADS, 2) k_eval(SpaceDev sp, EvalArgs a) {
+__global__ void __launch_bounds__(THREADS, EVAL_MIN_BLOCKS) k_eval(SpaceDev sp, EvalArgs a) {
   constexpr int N2 = NM * NM, N3 = NM * NM * NM, NC = N3 * NM;
   constexpr int R = (N3 + 31) / 32;
   // materialise: two staging buffers per warp (dynamic shared memory, none in the other modes)
@@ -428,7 +428,7 @@ struct CountTables {
 };
 
 template <int NM, bool POW2>
-__global__ void __launch_bounds__(THREADS, 2) k_compact_count(SpaceDev sp, EvalArgs a) {
+__global__ void __launch_bounds__(THREADS, EVAL_MIN_BLOCKS) k_compact_count(SpaceDev sp, EvalArgs a) {
   constexpr int N2 = NM * NM, N3 = NM * NM * NM, NC = N3 * NM;
   constexpr int R = (N3 + 31) / 32;
   __shared__ CountTables tables[WARPS];
