@@ -35,24 +35,24 @@ struct ps_space {
 
 // ---- sweep
 // Block shapes of the sweep: warps per block and the resident blocks per SM the
-// kernel is compiled for (which caps its registers at 96 either way: 21 warps fit
-// an SM).  The top-k sweep is fastest with seven blocks of three warps: many
-// resident blocks (1036 at a time, so that a thousand models run as one wave and
-// four thousand as four full ones), few and long lists per model.  The Pareto
-// sweep is fastest with two blocks of ten warps: its warps share a block's coarse
-// staircase, so larger blocks reject more candidates early (3 x 7, 4 x 5 and 7 x 3
-// were 4 to 30 % slower).
+// kernel is compiled for (which sets its register budget).  The top-k sweep is
+// fastest with eight blocks of three warps (24 warps of 80 registers; 1184 resident
+// blocks, so that a thousand models run as one wave): few and long lists per model.
+// The Pareto sweep is fastest with four blocks of four warps (16 warps of 128
+// registers): since its reduction pass became short, what it gains from registers
+// outweighs what larger blocks gain from sharing a coarse staircase (2 x 10 warps of
+// 96 registers: +6 %; 2 x 8: +2.5 %; 3 x 5, 8 x 2, 1 x 16: +3 to +10 %).
 #ifndef SWEEP_WARPS_TOPK
 #define SWEEP_WARPS_TOPK 3
 #endif
 #ifndef SWEEP_BLOCKS_TOPK
-#define SWEEP_BLOCKS_TOPK 7
+#define SWEEP_BLOCKS_TOPK 8
 #endif
 #ifndef SWEEP_WARPS_PARETO
-#define SWEEP_WARPS_PARETO 10
+#define SWEEP_WARPS_PARETO 4
 #endif
 #ifndef SWEEP_BLOCKS_PARETO
-#define SWEEP_BLOCKS_PARETO 2
+#define SWEEP_BLOCKS_PARETO 4
 #endif
 static inline int sweep_warps(int kind) { return kind == PS_REDUCE_PARETO ? SWEEP_WARPS_PARETO : SWEEP_WARPS_TOPK; }
 static inline int sweep_blocks_per_sm(int kind) { return kind == PS_REDUCE_PARETO ? SWEEP_BLOCKS_PARETO : SWEEP_BLOCKS_TOPK; }
