@@ -376,6 +376,32 @@ def test_sweeps_around_the_exact_double_limit(ctx, ps, cap):
                       os_.sweep(filt, [cap], O.KIND_TOPK, 64, n_threads=8))
 
 
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("tp_degree", [1, 2, 63, 64, 65, 100, 4096])
+def test_select_divisor_search_paths(ctx, ps, tp_degree):
+    """The largest divisor of N not above tp_degree: degrees up to 64 go through the host's
+    tables, larger ones and device counts above 2^24 through the plain search; the extremes of
+    the documented ranges (P = 2^46, N = 2^24, a layer as large as the model) go through the
+    reciprocal divisions."""
+    q = synth.select_queries(3000, seed=900 + tp_degree)
+    q[:, 7] = 1                                   # fast interconnect: the tensor-parallel branch is open
+    q[::3, 2] = 1 << 30                           # small devices: many queries reach that branch
+    q[::3, 1] = q[::3, 0] // 3                    # with a layer too large for a device
+    odd = np.arange(len(q)) % 5 == 0
+    q[odd, 3] = (np.arange(odd.sum()) * 7919 + 1) % ((1 << 24) - 1) + 1     # any count up to 2^24
+    q[1, 3] = 1 << 24
+    q[2, 3] = (1 << 24) - 1
+    q[4, 0], q[4, 1], q[4, 3] = 1 << 46, 1 << 46, 1 << 24
+    q[5, 0], q[5, 1], q[5, 3] = 1 << 46, (1 << 46) - 1, 3 * 5 * 7 * 11 * 13 * 17
+    got = ctx.select(to_query_records(ps, q), tp_degree=tp_degree)
+    want = O.select(q, tp_degree=tp_degree)
+    for j, name in enumerate(("mem", "comm", "branch", "T", "code_dp", "flags")):
+        assert np.array_equal(got[name].astype(np.uint64), want[:, j]), name
+    assert (want[:, 2] == 2).sum() > 100          # the branch is exercised
+    if tp_degree > 2:
+        assert len(np.unique(want[want[:, 2] == 2, 3])) > 2      # with several degrees
+
 @pytest.mark.parametrize("host_cap", [0, 8 * synth.GB, 200 * synth.GB])
 def test_topk_with_a_host_budget_on_a_power_of_two_space(ctx, ps, host_cap):
     """The top-k kernels compiled for a host budget, in the power-of-two case."""
