@@ -162,6 +162,25 @@ def test_pareto_c3_sample(ctx, ps, comm_kind, host_cap):
     assert_same_sweep(got, want)
 
 
+def test_sweeps_after_the_model_table_is_replaced(ctx, ps):
+    """ps_space_set_models: the records, and the order in which the sweeps' blocks take the
+    models, follow the new table (the old table's models reversed, then shapes of another
+    seed: another order of expected work each time)."""
+    space = synth.config("C3", n_models=24)
+    gs = ctx.space(space)
+    filt = dict(require_flags=VALID, host_cap=64 * synth.GB)
+    caps = [80 * synth.GB, 192 * synth.GB]
+    other = synth.config("C4", n_models=24)["models"]
+    for models in (space["models"][::-1].copy(), other, space["models"]):
+        gs.set_models(models)
+        os_ = O.Space(dict(space, models=models))
+        assert_same_sweep(gs.sweep(filt, caps, ps.REDUCE_PARETO, 64), os_.sweep(filt, caps, O.KIND_PARETO, 64, n_threads=8))
+        assert_same_sweep(gs.sweep(dict(require_flags=VALID), caps[1:], ps.REDUCE_TOPK, 64),
+                          os_.sweep(dict(require_flags=VALID), caps[1:], O.KIND_TOPK, 64, n_threads=8))
+        first = 5 * gs.points_per_model + 777
+        assert_same_arrays(gs.eval_batch(first, 30_000), os_.eval_range(first, 30_000), "window")
+
+
 def test_pareto_many_caps_unsorted_and_truncated(ctx, ps):
     """Capacities in arbitrary order; an output shorter than the frontier still
     gets the true length in counts."""
