@@ -103,17 +103,17 @@ int enqueue_status_copy(ps_ctx* ctx) {
   return PS_OK;
 }
 
-u32 pick_chunks(const ps_ctx* ctx, const ps_space* sp, int kind) {
+u32 pick_chunks(const ps_ctx* ctx, const ps_space* sp, int kind, bool many) {
   // Blocks per model.  Every extra block of a model builds its lists from
   // scratch -- a top-k block takes every survivor as a candidate until it has
   // found its own first k -- so only as many as fill the GPU once (top-k) or
   // twice (Pareto, whose blocks are fewer and longer).
   const u64 waves = kind == PS_REDUCE_PARETO ? 2 : 1;
-  const u64 target = (u64)ctx->sm_count * sweep_blocks_per_sm(kind) * waves;
+  const u64 target = (u64)ctx->sm_count * sweep_blocks_per_sm(kind, many) * waves;
   u64 c = (target + sp->dev.n_models / 2) / sp->dev.n_models;       // to the nearest: one block too few is cheaper than a second list
   if (c < 1) c = 1;
   if (c > SWEEP_MAX_CHUNKS) c = SWEEP_MAX_CHUNKS;
-  const u64 by_units = (sp->dev.n_facts + sweep_warps(kind) - 1) / sweep_warps(kind);   // a unit per warp at least
+  const u64 by_units = (sp->dev.n_facts + sweep_warps(kind, many) - 1) / sweep_warps(kind, many);   // a unit per warp at least
   if (c > by_units) c = by_units;
   if (c < 1) c = 1;
   return (u32)c;
@@ -470,8 +470,14 @@ int ps_sweep_pareto(ps_ctx* ctx, const ps_space* sp, const ps_filter* filter,
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return PS_E_CUDA;
 
-  const u32 n_chunks = pick_chunks(ctx, sp, (int)reduce_kind);
-  const size_t slots = (size_t)sp->dev.n_models * n_chunks * sweep_warps((int)reduce_kind);   // one list per warp
+  // top-k over a table of many models, in the fast case (powers of two, byte counts exact in a
+  // double, every capacity below 2^53, nothing skipped): smaller blocks
+  bool many = reduce_kind == PS_REDUCE_TOPK && !filter->skip_rejected && sp->dev.all_pow2 && sp->dev.all_small &&
+              sp->dev.repl == 1 &&
+              (u64)sp->dev.n_models >= (u64)SWEEP_TOPK_MANY_WAVES * ctx->sm_count * SWEEP_BLOCKS_TOPK_MANY;
+  for (u32 c = 0; c < n_caps; ++c) many = many && caps_bytes[c] < ((u64)1 << 53) - 1;
+  const u32 n_chunks = pick_chunks(ctx, sp, (int)reduce_kind, many);
+  const size_t slots = (size_t)sp->dev.n_models * n_chunks * sweep_warps((int)reduce_kind, many);   // one list per warp
   const size_t partial_bytes = slots * SWEEP_LIST_CAP * sizeof(PartialEntry);
   const size_t lengths_bytes = (slots * sizeof(uint2) + 15) & ~size_t(15);
   rc = ensure_scratch(ctx, partial_bytes + lengths_bytes + sizeof(u32) * (size_t)sp->dev.n_models);
@@ -483,6 +489,7 @@ int ps_sweep_pareto(ps_ctx* ctx, const ps_space* sp, const ps_filter* filter,
   s.comm_kind = filter->comm_kind;
   s.k_keep = reduce_kind == PS_REDUCE_TOPK ? max_entries : 0;
   s.skip_rejected = filter->skip_rejected ? 1u : 0u;
+  s.many_models = many ? 1u : 0u;
   s.partial = static_cast<PartialEntry*>(ctx->scratch);
   s.partial_n = reinterpret_cast<uint2*>(static_cast<char*>(ctx->scratch) + partial_bytes);
   s.status = ctx->d_status;
@@ -490,7 +497,7 @@ int ps_sweep_pareto(ps_ctx* ctx, const ps_space* sp, const ps_filter* filter,
   memset(&m, 0, sizeof(m));
   m.partial = s.partial;
   m.partial_n = s.partial_n;
-  m.n_lists = n_chunks * sweep_warps((int)reduce_kind);
+  m.n_lists = n_chunks * sweep_warps((int)reduce_kind, many);
   m.host_cap = filter->host_cap;
   m.require_flags = s.require_flags;
   m.n_caps_total = n_caps;

@@ -54,8 +54,25 @@ struct ps_space {
 #ifndef SWEEP_BLOCKS_PARETO
 #define SWEEP_BLOCKS_PARETO 4
 #endif
-static inline int sweep_warps(int kind) { return kind == PS_REDUCE_PARETO ? SWEEP_WARPS_PARETO : SWEEP_WARPS_TOPK; }
-static inline int sweep_blocks_per_sm(int kind) { return kind == PS_REDUCE_PARETO ? SWEEP_BLOCKS_PARETO : SWEEP_BLOCKS_TOPK; }
+// A table of many models (at least SWEEP_TOPK_MANY_WAVES full waves of the smaller blocks) is
+// swept for top-k with blocks of two warps, nine resident per SM: -3.7 % on four thousand
+// models; on a thousand models the GPU is then short of warps (+10 %), so those keep three.
+// Compiled for the fast case without skipping only (see launch_sweep_t).
+#ifndef SWEEP_WARPS_TOPK_MANY
+#define SWEEP_WARPS_TOPK_MANY 2
+#endif
+#ifndef SWEEP_BLOCKS_TOPK_MANY
+#define SWEEP_BLOCKS_TOPK_MANY 9
+#endif
+#ifndef SWEEP_TOPK_MANY_WAVES
+#define SWEEP_TOPK_MANY_WAVES 2
+#endif
+static inline int sweep_warps(int kind, bool many = false) {
+  return kind == PS_REDUCE_PARETO ? SWEEP_WARPS_PARETO : (many ? SWEEP_WARPS_TOPK_MANY : SWEEP_WARPS_TOPK);
+}
+static inline int sweep_blocks_per_sm(int kind, bool many = false) {
+  return kind == PS_REDUCE_PARETO ? SWEEP_BLOCKS_PARETO : (many ? SWEEP_BLOCKS_TOPK_MANY : SWEEP_BLOCKS_TOPK);
+}
 #define SWEEP_LIST_CAP 128        /* entries of a warp's list and of a block's partial list */
 #define SWEEP_MAX_CHUNKS 16       /* blocks per model                                        */
 #define MERGE_CAP (5 * SWEEP_LIST_CAP)    /* entries the merge kernel combines at a time: what it
@@ -75,6 +92,8 @@ struct SweepArgs {
   u32 comm_kind;
   u32 k_keep;           // top-k: entries kept
   u32 skip_rejected;    // do not evaluate factorisations whose composition bits miss a required flag
+  u32 many_models;      // top-k: the blocks of two warps (the host has checked that the fast case applies)
+  u32 pad;
   PartialEntry* partial;   // [n_models * n_chunks * warps][SWEEP_LIST_CAP]: one list per warp
   uint2* partial_n;        // [n_models * n_chunks * warps]: (entries, survivors)
   u32* status;

@@ -1252,10 +1252,11 @@ __global__ void __launch_bounds__(MERGE_THREADS, SWEEP_MERGE_MIN_BLOCKS) k_sweep
 }  // namespace
 
 // ------------------------------------------------------------------ launchers
-template <int KIND, int NM, bool HOST_LIMITED, bool FAST, bool SKIP>
+template <int KIND, int NM, bool HOST_LIMITED, bool FAST, bool SKIP, bool MANY = false>
 static cudaError_t launch_sweep_p(const SpaceDev& sp, const SweepArgs& a, u32 n_chunks, cudaStream_t stream) {
-  constexpr int WARPS = KIND == PS_REDUCE_PARETO ? SWEEP_WARPS_PARETO : SWEEP_WARPS_TOPK;
-  constexpr int MIN_BLOCKS = KIND == PS_REDUCE_PARETO ? SWEEP_BLOCKS_PARETO : SWEEP_BLOCKS_TOPK;
+  constexpr int WARPS = KIND == PS_REDUCE_PARETO ? SWEEP_WARPS_PARETO : (MANY ? SWEEP_WARPS_TOPK_MANY : SWEEP_WARPS_TOPK);
+  constexpr int MIN_BLOCKS = KIND == PS_REDUCE_PARETO ? SWEEP_BLOCKS_PARETO
+                                                      : (MANY ? SWEEP_BLOCKS_TOPK_MANY : SWEEP_BLOCKS_TOPK);
   dim3 grid(n_chunks, sp.n_models);
   const size_t smem = sizeof(SweepShared<WARPS>);
   cudaError_t e = cudaFuncSetAttribute(k_sweep<KIND, NM, WARPS, MIN_BLOCKS, HOST_LIMITED, FAST, SKIP>,
@@ -1273,6 +1274,9 @@ static cudaError_t launch_sweep_t(const SpaceDev& sp, const SweepArgs& a, u32 n_
     if (a.skip_rejected)
       return host_limited ? launch_sweep_p<KIND, NM, true, true, true>(sp, a, n_chunks, stream)
                           : launch_sweep_p<KIND, NM, false, true, true>(sp, a, n_chunks, stream);
+    if (KIND == PS_REDUCE_TOPK && a.many_models)
+      return host_limited ? launch_sweep_p<KIND, NM, true, true, false, KIND == PS_REDUCE_TOPK>(sp, a, n_chunks, stream)
+                          : launch_sweep_p<KIND, NM, false, true, false, KIND == PS_REDUCE_TOPK>(sp, a, n_chunks, stream);
     return host_limited ? launch_sweep_p<KIND, NM, true, true, false>(sp, a, n_chunks, stream)
                         : launch_sweep_p<KIND, NM, false, true, false>(sp, a, n_chunks, stream);
   }

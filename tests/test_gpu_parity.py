@@ -162,6 +162,24 @@ def test_pareto_c3_sample(ctx, ps, comm_kind, host_cap):
     assert_same_sweep(got, want)
 
 
+@pytest.mark.parametrize("k,host_cap", [(64, O.NO_LIMIT), (7, 16 * synth.GB)])
+def test_topk_over_a_table_of_many_models(ctx, ps, k, host_cap):
+    """Enough models for two waves of the small top-k blocks (2 x 148 x 9 = 2664): the sweep then
+    runs in blocks of two warps.  Also with a budget that the same table does not take that
+    path with (skipping allowed), and with a capacity beyond 2^53 (the general kernels)."""
+    space = synth.config("C1", n_models=2700)
+    gs, os_ = both(ctx, space)
+    caps = [40 * synth.GB, 192 * synth.GB]
+    for filt in (dict(require_flags=VALID, host_cap=host_cap),
+                 dict(require_flags=VALID, host_cap=host_cap, skip_rejected=1)):
+        got = gs.sweep(filt, caps, ps.REDUCE_TOPK, k)
+        want = os_.sweep({f: v for f, v in filt.items() if f != "skip_rejected"}, caps, O.KIND_TOPK, k, n_threads=8)
+        assert_same_sweep(got, want)
+    big = [1 << 60]
+    filt = dict(require_flags=VALID, host_cap=host_cap)
+    assert_same_sweep(gs.sweep(filt, big, ps.REDUCE_TOPK, k), os_.sweep(filt, big, O.KIND_TOPK, k, n_threads=8))
+
+
 def test_sweeps_after_the_model_table_is_replaced(ctx, ps):
     """ps_space_set_models: the records, and the order in which the sweeps' blocks take the
     models, follow the new table (the old table's models reversed, then shapes of another
