@@ -317,7 +317,13 @@ static void sweep_order(ps_space* sp, const ps_model_shape* models, u32 n_models
     }
   sp->order.resize(n_models);
   for (u32 i = 0; i < n_models; ++i) sp->order[i] = i;
-  std::stable_sort(sp->order.begin(), sp->order.end(), [&](u32 a, u32 b) { return work[a] > work[b]; });
+  // (among models with the same count the smaller first: more of its points fit a capacity)
+  std::stable_sort(sp->order.begin(), sp->order.end(), [&](u32 a, u32 b) {
+    if (work[a] != work[b]) return work[a] > work[b];
+    const u64 pa = (u64)models[a].layers * models[a].hidden * models[a].hidden;
+    const u64 pb = (u64)models[b].layers * models[b].hidden * models[b].hidden;
+    return pa < pb;
+  });
 }
 
 int ps_space_set_models(ps_space* sp, const ps_model_shape* models, uint32_t n_models) {
